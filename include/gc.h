@@ -1,0 +1,179 @@
+/*
+ * gc.h - C ABI of the B200 fused-subgraph executor.
+ *
+ * The boundary follows the paper's statement of the problem (Sections II, V and VII): a framework
+ * hands over a *partition* - a list of ops over logical tensors with static shapes, dtypes, plain
+ * row-major layouts and per-tensor quantisation attributes -, the partition is *compiled once*, and
+ * the compiled object is *executed* many times on plain-layout inputs and outputs.  Constant
+ * weights may be unknown at compile time; they are preprocessed when they first arrive and the
+ * result is reused (Section V, "constant weight preprocessing").
+ *
+ * Two subgraph patterns are accepted; everything else fails at gc_compile with GC_ERR_UNSUPPORTED
+ * (there is no CPU fallback - the paper leaves fallback to the framework, Section VII):
+ *
+ *   MLP chain   (Section VII "MLP"; Fig. 5):  L >= 1 layers, each
+ *       MatMul(h, W) [-> Dequantize] [-> Add(bias)] [-> ReLU | GELU_TANH | Sigmoid]
+ *                    [-> Quantize | TypeCast]
+ *     h is the previous layer's result (graph input for the first layer), W a constant 2-D graph
+ *     input [K,N] (or [N,K] with transpose_b), bias a constant 1-D fp32 graph input [N].
+ *
+ *   Attention   (Section VII "MHA": two batch matmuls, a softmax and the binary ops between):
+ *       MatMul(Q, K, transpose_b) [-> Dequantize] [-> Mul(scalar)] [-> Add(mask)] -> SoftMax
+ *           [-> Quantize | TypeCast] -> MatMul(P, V) [-> Dequantize -> Quantize | -> TypeCast]
+ *     Q, K, V, O are [B,H,S,D] contiguous; mask is fp32 [B,1,1,S].
+ *
+ * Semantics of the ops (what an unfused, op-by-op evaluation gives, which the fused kernels must
+ * reproduce):
+ *   MatMul on u8/s8 operands: exact integer sum of zero-point-subtracted operands, s32 result whose
+ *     implied scale is the fp32 product scale_a * scale_b.  On bf16/f32 operands: fp32 accumulation
+ *     on tensor cores (f32 operands are consumed as tf32).
+ *   Dequantize: (float)(q - zero_point) * scale, fp32.          Quantize: saturate(rne(x * inv) + zp)
+ *     with inv = 1.0f / scale formed in fp32 (Section V: DQ scales and offsets, Q does the reverse).
+ *   On the integer paths every fp32 multiply/add is a separately rounded IEEE operation (no fused
+ *   multiply-add), so results are reproducible bit for bit.
+ *
+ * Conventions
+ *   - Every call returns a gc_status_t; out-parameters are untouched on error; gc_last_error()
+ *     returns a thread-local, library-owned message for the last failing call on this thread.
+ *   - Pointers named *_dev are CUDA device pointers on the device given to gc_compile; pointers
+ *     named *_host are host pointers.  The caller owns all tensor memory, the workspace and the
+ *     stream; the library owns only host-side plan objects.  Input and output device pointers must
+ *     be 16-byte aligned (GC_ERR_ALIGNMENT otherwise).
+ *   - in_*[i] corresponds to input_ids[i] given at gc_partition_create, out_*[i] to output_ids[i].
+ *   - gc_execute is asynchronous on the given stream.  One compiled object must not be executed
+ *     concurrently on two streams (it owns one workspace).
+ *   - Device-side waits are bounded: if one expires the kernel records an error in a status word
+ *     and returns; gc_query_status reports it as GC_ERR_TIMEOUT.  Nothing traps.
+ */
+#ifndef GC_B200_H_
+#define GC_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  GC_OK = 0,
+  GC_ERR_INVALID_ARG = 1,
+  GC_ERR_UNSUPPORTED = 2,
+  GC_ERR_SHAPE = 3,
+  GC_ERR_STATE = 4,
+  GC_ERR_CUDA = 5,
+  GC_ERR_OOM = 6,
+  GC_ERR_TIMEOUT = 7,
+  GC_ERR_ALIGNMENT = 8
+} gc_status_t;
+
+typedef enum { GC_F32 = 0, GC_BF16 = 1, GC_U8 = 2, GC_S8 = 3, GC_S32 = 4 } gc_dtype_t;
+
+typedef enum {
+  GC_OP_MATMUL = 0,
+  GC_OP_ADD = 1,
+  GC_OP_MUL = 2,
+  GC_OP_RELU = 3,
+  GC_OP_GELU_TANH = 4,
+  GC_OP_SIGMOID = 5,
+  GC_OP_SOFTMAX = 6,
+  GC_OP_QUANTIZE = 7,
+  GC_OP_DEQUANTIZE = 8,
+  GC_OP_TYPECAST = 9
+} gc_op_kind_t;
+
+#define GC_MAX_DIMS 6
+
+/* Logical tensor (Section II: dtype, shape, layout metadata).  Layout is always dense row-major. */
+typedef struct {
+  int64_t id;
+  int32_t dtype;          /* gc_dtype_t */
+  int32_t ndims;
+  int64_t dims[GC_MAX_DIMS];
+  float scale;            /* per-tensor quantisation scale; ignored for float dtypes */
+  int32_t zero_point;
+  int32_t is_constant;    /* 1: same pointer and contents on every execution (weights, biases) */
+} gc_logical_tensor_t;
+
+/* Op (Section II: kind, attributes, input and output logical tensors). */
+typedef struct {
+  int32_t kind;           /* gc_op_kind_t */
+  int32_t n_in;           /* 1 or 2 */
+  int64_t in[3];          /* logical tensor ids */
+  int64_t out;            /* logical tensor id */
+  int32_t transpose_b;    /* MATMUL: second operand stored [.., n, k] */
+  int32_t axis;           /* SOFTMAX: must address the last axis (-1 or ndims-1) */
+  float scalar;           /* MUL: the constant multiplier */
+  int32_t has_scalar;     /* MUL: must be 1 */
+} gc_op_t;
+
+/* Options for gc_compile; pass NULL for the defaults (all zero). */
+typedef struct {
+  int32_t force_generic;  /* 1: use the shape-generic CUDA-core kernels instead of the tcgen05 ones
+                             (ablation / debugging; results obey the same contracts) */
+  int32_t no_chain_fusion;/* 1: one launch per fused op with full stream ordering between them, the
+                             analogue of running with coarse-grain fusion disabled (Section VII) */
+  int32_t reserved[6];
+} gc_compile_options_t;
+
+typedef struct gc_partition gc_partition_t;
+typedef struct gc_compiled gc_compiled_t;
+
+/* Build a partition (Section II, graph of ops and logical tensors).  Host only; copies everything.
+ * ops must be in topological order.  Errors: INVALID_ARG (null pointers, unknown ids, duplicate
+ * ids, bad enum values), SHAPE (dims inconsistent with the op). */
+gc_status_t gc_partition_create(gc_partition_t** out, const gc_op_t* ops, int32_t n_ops,
+                                const gc_logical_tensor_t* tensors, int32_t n_tensors,
+                                const int64_t* input_ids, int32_t n_in,
+                                const int64_t* output_ids, int32_t n_out);
+void gc_partition_destroy(gc_partition_t* p);
+
+/* Pass as cuda_device to gc_compile to form the pattern and the plan for a nominal B200 (148 SMs)
+ * without touching a device; the result answers the query calls but gc_execute returns GC_ERR_STATE. */
+#define GC_DEVICE_PLAN_ONLY (-1)
+
+/* Compile a partition for one CUDA device (Section V: pattern formation, constant folding of the
+ * quantisation parameters, kernel/tile selection; Section VI: temporary buffers sized and reused
+ * at compile time).  Host only; touches the device only to query its properties. */
+gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, const gc_compile_options_t* opt,
+                       gc_compiled_t** out);
+void gc_compiled_destroy(gc_compiled_t* c);
+
+/* Scratch memory the compiled object needs (inter-layer activations, prepacked weights, padded
+ * input copies, a status word).  The caller allocates it on the device (256-byte aligned), hands
+ * it over once and keeps it alive until gc_compiled_destroy.  Contents need no initialisation. */
+gc_status_t gc_workspace_bytes(const gc_compiled_t* c, size_t* bytes);
+gc_status_t gc_set_workspace(gc_compiled_t* c, void* workspace_dev, size_t bytes);
+
+/* Execute (Section VII: "the compiled code only needs to be called once" per subgraph).  Enqueues
+ * all work on cuda_stream (a cudaStream_t, may be NULL for the default stream) and returns.  On
+ * the first call, or when a constant input arrives at a new address, the constant weights are
+ * prepacked on the same stream first and cached in the workspace (Section V). */
+gc_status_t gc_execute(gc_compiled_t* c, void* cuda_stream, const void* const* in_dev, int32_t n_in,
+                       void* const* out_dev, int32_t n_out);
+
+/* Same computation with HOST buffers: copies the inputs to a device staging area (constants only
+ * when their host pointer changes), executes, copies the outputs back and synchronises the stream.
+ * The staging area is caller-allocated device memory of gc_host_staging_bytes bytes. */
+gc_status_t gc_host_staging_bytes(const gc_compiled_t* c, size_t* bytes);
+gc_status_t gc_set_host_staging(gc_compiled_t* c, void* staging_dev, size_t bytes);
+gc_status_t gc_execute_host(gc_compiled_t* c, void* cuda_stream, const void* const* in_host,
+                            int32_t n_in, void* const* out_host, int32_t n_out);
+
+/* Synchronise the stream and read the device status word: GC_OK, GC_ERR_TIMEOUT (a bounded
+ * device-side wait expired) or GC_ERR_CUDA (the stream reported an error). */
+gc_status_t gc_query_status(gc_compiled_t* c, void* cuda_stream);
+
+/* Introspection: number of kernel launches one gc_execute enqueues after prepacking, and a short
+ * text description of the plan (pattern, per-layer kernel and tile).  The string is owned by the
+ * compiled object. */
+gc_status_t gc_launches_per_execute(const gc_compiled_t* c, int32_t* n);
+const char* gc_plan_description(const gc_compiled_t* c);
+
+const char* gc_last_error(void);
+const char* gc_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GC_B200_H_ */

@@ -1,0 +1,111 @@
+// Per-element post-op evaluation shared by the GEMM kernels (tcgen05 and CUDA-core variants).
+#pragma once
+#include <cuda_bf16.h>
+
+#include "gc_internal.h"
+
+namespace gc {
+
+__device__ __forceinline__ float tanh_approx(float x) {
+  float y;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ float apply_act(float t, int act) {
+  switch (act) {
+    case ACT_RELU:
+      return fmaxf(t, 0.0f);
+    case ACT_GELU_TANH: {
+      // 0.5 x (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3)))
+      const float u = 0.7978845608028654f * (t + 0.044715f * t * t * t);
+      return 0.5f * t * (1.0f + tanh_approx(u));
+    }
+    case ACT_SIGMOID:
+      return 1.0f / (1.0f + expf(-t));
+    default:
+      return t;
+  }
+}
+
+// Value after dequantize / bias / activation.  `raw` holds the accumulator bits (s32 or f32).
+__device__ __forceinline__ float epi_value(uint32_t raw, int n, const Epilogue& e) {
+  float t;
+  if (e.acc_is_int) {
+    t = __int2float_rn(static_cast<int>(raw));
+    t = __fmul_rn(t, e.dq);
+  } else {
+    t = __uint_as_float(raw);
+  }
+  if (e.bias) t = __fadd_rn(t, __ldg(e.bias + n));
+  return apply_act(t, e.act);
+}
+
+// saturate(rne(t * inv) + zp) to u8 / s8
+__device__ __forceinline__ int quantize_value(float t, float inv, int zp, int lo, int hi) {
+  int r = __float2int_rn(__fmul_rn(t, inv));      // cvt.rni.s32.f32 saturates
+  r = min(max(r, -(1 << 24)), 1 << 24);           // keep r + zp free of overflow
+  return min(max(r + zp, lo), hi);
+}
+
+// Store 16 consecutive outputs of one row (columns n0..n0+15) from 16 raw accumulator words.
+// `dst_row` points at column 0 of the row; n0 is a multiple of 16 and the row pitch keeps 16-byte
+// alignment of (dst_row + n0) for every supported dtype.
+__device__ __forceinline__ void epi_store16(const uint32_t* raw, void* dst_row, int n0, const Epilogue& e) {
+  if (e.acc_is_int && !e.has_dq) {   // raw s32 accumulators
+    int4* d = reinterpret_cast<int4*>(static_cast<int*>(dst_row) + n0);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) d[i] = make_int4(raw[4 * i], raw[4 * i + 1], raw[4 * i + 2], raw[4 * i + 3]);
+    return;
+  }
+  float t[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) t[i] = epi_value(raw[i], n0 + i, e);
+  if (e.out_dtype == GC_F32) {
+    float4* d = reinterpret_cast<float4*>(static_cast<float*>(dst_row) + n0);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) d[i] = make_float4(t[4 * i], t[4 * i + 1], t[4 * i + 2], t[4 * i + 3]);
+  } else if (e.out_dtype == GC_BF16) {
+    uint32_t w[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      __nv_bfloat162 h = __floats2bfloat162_rn(t[2 * i], t[2 * i + 1]);
+      w[i] = *reinterpret_cast<uint32_t*>(&h);
+    }
+    uint4* d = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(dst_row) + n0);
+    d[0] = make_uint4(w[0], w[1], w[2], w[3]);
+    d[1] = make_uint4(w[4], w[5], w[6], w[7]);
+  } else {
+    const int lo = e.out_dtype == GC_U8 ? 0 : -128, hi = e.out_dtype == GC_U8 ? 255 : 127;
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      uint32_t b0 = quantize_value(t[4 * i + 0], e.inv, e.zp, lo, hi) & 0xFF;
+      uint32_t b1 = quantize_value(t[4 * i + 1], e.inv, e.zp, lo, hi) & 0xFF;
+      uint32_t b2 = quantize_value(t[4 * i + 2], e.inv, e.zp, lo, hi) & 0xFF;
+      uint32_t b3 = quantize_value(t[4 * i + 3], e.inv, e.zp, lo, hi) & 0xFF;
+      w[i] = b0 | (b1 << 8) | (b2 << 16) | (b3 << 24);
+    }
+    *reinterpret_cast<uint4*>(static_cast<uint8_t*>(dst_row) + n0) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
+// Scalar store of one output (generic kernels).
+__device__ __forceinline__ void epi_store1(uint32_t raw, void* dst_row, int n, const Epilogue& e) {
+  if (e.acc_is_int && !e.has_dq) {
+    static_cast<int*>(dst_row)[n] = static_cast<int>(raw);
+    return;
+  }
+  const float t = epi_value(raw, n, e);
+  if (e.out_dtype == GC_F32) {
+    static_cast<float*>(dst_row)[n] = t;
+  } else if (e.out_dtype == GC_BF16) {
+    static_cast<__nv_bfloat16*>(dst_row)[n] = __float2bfloat16_rn(t);
+  } else if (e.out_dtype == GC_U8) {
+    static_cast<uint8_t*>(dst_row)[n] = static_cast<uint8_t>(quantize_value(t, e.inv, e.zp, 0, 255));
+  } else {
+    static_cast<int8_t*>(dst_row)[n] = static_cast<int8_t>(quantize_value(t, e.inv, e.zp, -128, 127));
+  }
+}
+
+}  // namespace gc

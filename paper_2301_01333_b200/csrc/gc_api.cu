@@ -1,0 +1,879 @@
+// Host side of the C ABI: partition bookkeeping, pattern formation (the fixed analogue of the paper's
+// fine-grain fusion: one Tunable op plus the Fusible ops that follow it, Section V), constant folding of
+// the quantisation parameters, kernel and tile selection (the role of the template heuristic, Section
+// III), compile-time buffer planning with reuse (Section VI) and the execute path that enqueues the
+// prepack (first call only) and the fused kernels on the caller's stream.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <string>
+#include <vector>
+
+#include "gc_internal.h"
+
+using namespace gc;
+
+// ------------------------------------------------------------------------------------------------
+// errors
+// ------------------------------------------------------------------------------------------------
+static thread_local char g_err[512] = "";
+
+static gc_status_t fail(gc_status_t st, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  return st;
+}
+#define CUDA_TRY(expr)                                                                          \
+  do {                                                                                          \
+    cudaError_t e__ = (expr);                                                                   \
+    if (e__ != cudaSuccess) return fail(GC_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e__)); \
+  } while (0)
+
+extern "C" const char* gc_last_error(void) { return g_err; }
+extern "C" const char* gc_version(void) { return "gc-b200 0.1 (sm_100a)"; }
+
+// ------------------------------------------------------------------------------------------------
+// partition
+// ------------------------------------------------------------------------------------------------
+struct gc_partition {
+  std::vector<gc_op_t> ops;
+  std::vector<gc_logical_tensor_t> tensors;
+  std::map<int64_t, int> index;   // tensor id -> position in `tensors`
+  std::vector<int64_t> in_ids, out_ids;
+  const gc_logical_tensor_t* lt(int64_t id) const {
+    auto it = index.find(id);
+    return it == index.end() ? nullptr : &tensors[it->second];
+  }
+  int input_pos(int64_t id) const {
+    for (size_t i = 0; i < in_ids.size(); ++i)
+      if (in_ids[i] == id) return static_cast<int>(i);
+    return -1;
+  }
+  int output_pos(int64_t id) const {
+    for (size_t i = 0; i < out_ids.size(); ++i)
+      if (out_ids[i] == id) return static_cast<int>(i);
+    return -1;
+  }
+  int consumers(int64_t id) const {
+    int n = 0;
+    for (const auto& op : ops)
+      for (int i = 0; i < op.n_in; ++i) n += op.in[i] == id;
+    return n;
+  }
+};
+
+static int dtype_bytes(int dt) { return dt == GC_F32 || dt == GC_S32 ? 4 : (dt == GC_BF16 ? 2 : 1); }
+static bool is_int8(int dt) { return dt == GC_U8 || dt == GC_S8; }
+static int64_t numel(const gc_logical_tensor_t& t) {
+  int64_t n = 1;
+  for (int i = 0; i < t.ndims; ++i) n *= t.dims[i];
+  return n;
+}
+static bool same_dims(const gc_logical_tensor_t& a, const gc_logical_tensor_t& b) {
+  if (a.ndims != b.ndims) return false;
+  for (int i = 0; i < a.ndims; ++i)
+    if (a.dims[i] != b.dims[i]) return false;
+  return true;
+}
+
+extern "C" gc_status_t gc_partition_create(gc_partition_t** out, const gc_op_t* ops, int32_t n_ops,
+                                           const gc_logical_tensor_t* tensors, int32_t n_tensors,
+                                           const int64_t* input_ids, int32_t n_in, const int64_t* output_ids,
+                                           int32_t n_out) {
+  if (!out || !ops || !tensors || !input_ids || !output_ids) return fail(GC_ERR_INVALID_ARG, "null argument");
+  if (n_ops <= 0 || n_tensors <= 0 || n_in <= 0 || n_out <= 0) return fail(GC_ERR_INVALID_ARG, "empty partition");
+  auto p = new gc_partition();
+  auto bail = [&](gc_status_t st) {
+    delete p;
+    return st;
+  };
+  for (int i = 0; i < n_tensors; ++i) {
+    const auto& t = tensors[i];
+    if (t.dtype < GC_F32 || t.dtype > GC_S32) return bail(fail(GC_ERR_INVALID_ARG, "tensor %lld: bad dtype", (long long)t.id));
+    if (t.ndims < 1 || t.ndims > GC_MAX_DIMS) return bail(fail(GC_ERR_INVALID_ARG, "tensor %lld: bad ndims", (long long)t.id));
+    for (int d = 0; d < t.ndims; ++d)
+      if (t.dims[d] <= 0) return bail(fail(GC_ERR_SHAPE, "tensor %lld: non-positive dimension", (long long)t.id));
+    if (p->index.count(t.id)) return bail(fail(GC_ERR_INVALID_ARG, "duplicate tensor id %lld", (long long)t.id));
+    if (is_int8(t.dtype) && !(t.scale > 0.f) ) return bail(fail(GC_ERR_INVALID_ARG, "tensor %lld: scale must be positive", (long long)t.id));
+    p->index[t.id] = static_cast<int>(p->tensors.size());
+    p->tensors.push_back(t);
+  }
+  std::map<int64_t, bool> defined;
+  for (int i = 0; i < n_in; ++i) {
+    if (!p->lt(input_ids[i])) return bail(fail(GC_ERR_INVALID_ARG, "unknown input id %lld", (long long)input_ids[i]));
+    if (defined.count(input_ids[i])) return bail(fail(GC_ERR_INVALID_ARG, "duplicate input id"));
+    defined[input_ids[i]] = true;
+    p->in_ids.push_back(input_ids[i]);
+  }
+  for (int i = 0; i < n_ops; ++i) {
+    const auto& op = ops[i];
+    if (op.kind < GC_OP_MATMUL || op.kind > GC_OP_TYPECAST) return bail(fail(GC_ERR_INVALID_ARG, "op %d: bad kind", i));
+    const int want_in = (op.kind == GC_OP_MATMUL || op.kind == GC_OP_ADD) ? 2 : 1;
+    if (op.n_in != want_in) return bail(fail(GC_ERR_INVALID_ARG, "op %d: expects %d inputs", i, want_in));
+    for (int k = 0; k < op.n_in; ++k) {
+      if (!p->lt(op.in[k])) return bail(fail(GC_ERR_INVALID_ARG, "op %d: unknown input tensor", i));
+      if (!defined.count(op.in[k])) return bail(fail(GC_ERR_INVALID_ARG, "op %d: input used before it is defined (ops must be in topological order)", i));
+    }
+    const auto* o = p->lt(op.out);
+    if (!o) return bail(fail(GC_ERR_INVALID_ARG, "op %d: unknown output tensor", i));
+    if (defined.count(op.out)) return bail(fail(GC_ERR_INVALID_ARG, "op %d: output tensor defined twice", i));
+    const auto* a = p->lt(op.in[0]);
+    // shape checks
+    if (op.kind == GC_OP_MATMUL) {
+      const auto* b = p->lt(op.in[1]);
+      if (a->ndims < 2 || b->ndims < 2 || o->ndims != a->ndims)
+        return bail(fail(GC_ERR_SHAPE, "op %d: matmul needs >= 2-D operands", i));
+      const int64_t m = a->dims[a->ndims - 2], k = a->dims[a->ndims - 1];
+      const int64_t kb = op.transpose_b ? b->dims[b->ndims - 1] : b->dims[b->ndims - 2];
+      const int64_t n = op.transpose_b ? b->dims[b->ndims - 2] : b->dims[b->ndims - 1];
+      if (k != kb || o->dims[o->ndims - 2] != m || o->dims[o->ndims - 1] != n)
+        return bail(fail(GC_ERR_SHAPE, "op %d: matmul shapes do not agree", i));
+      if (b->ndims > 2) {
+        if (b->ndims != a->ndims) return bail(fail(GC_ERR_SHAPE, "op %d: batched matmul rank mismatch", i));
+        for (int d = 0; d < a->ndims - 2; ++d)
+          if (a->dims[d] != b->dims[d] || a->dims[d] != o->dims[d])
+            return bail(fail(GC_ERR_SHAPE, "op %d: batch dimensions differ", i));
+      }
+    } else if (op.kind == GC_OP_ADD) {
+      const auto* b = p->lt(op.in[1]);
+      if (!same_dims(*a, *o)) return bail(fail(GC_ERR_SHAPE, "op %d: add output shape", i));
+      // second operand must broadcast onto the first (trailing alignment)
+      if (b->ndims > a->ndims) return bail(fail(GC_ERR_SHAPE, "op %d: add broadcast rank", i));
+      for (int d = 0; d < b->ndims; ++d) {
+        const int64_t bd = b->dims[b->ndims - 1 - d], ad = a->dims[a->ndims - 1 - d];
+        if (bd != 1 && bd != ad) return bail(fail(GC_ERR_SHAPE, "op %d: add operands do not broadcast", i));
+      }
+    } else {
+      if (!same_dims(*a, *o)) return bail(fail(GC_ERR_SHAPE, "op %d: elementwise output shape differs", i));
+      if (op.kind == GC_OP_MUL && !op.has_scalar) return bail(fail(GC_ERR_INVALID_ARG, "op %d: mul needs a scalar", i));
+      if (op.kind == GC_OP_SOFTMAX && !(op.axis == -1 || op.axis == a->ndims - 1))
+        return bail(fail(GC_ERR_UNSUPPORTED, "op %d: softmax over the last axis only", i));
+    }
+    defined[op.out] = true;
+    p->ops.push_back(op);
+  }
+  for (int i = 0; i < n_out; ++i) {
+    if (!p->lt(output_ids[i]) || !defined.count(output_ids[i]))
+      return bail(fail(GC_ERR_INVALID_ARG, "output id %lld is not produced by the partition", (long long)output_ids[i]));
+    p->out_ids.push_back(output_ids[i]);
+  }
+  *out = p;
+  return GC_OK;
+}
+
+extern "C" void gc_partition_destroy(gc_partition_t* p) { delete p; }
+
+// ------------------------------------------------------------------------------------------------
+// compiled object
+// ------------------------------------------------------------------------------------------------
+enum Pattern { PAT_MLP = 1, PAT_SDPA = 2, PAT_BATCHED_MATMUL = 3 };
+
+struct LayerPlan {
+  int M = 0, K = 0, N = 0;
+  int a_dtype = 0, w_dtype = 0, a_zp = 0;
+  int transposed_w = 0;
+  int a_input = -1;          // graph input position of the activation (first layer) or -1
+  int w_input = -1, bias_input = -1;
+  Epilogue epi = {};
+  int out_pos = -1;          // graph output position, or -1 for an intermediate
+  int out_elem = 0;          // bytes per stored element
+  int64_t out_pitch = 0;     // elements
+  size_t out_off = 0;        // workspace offset of an intermediate
+  size_t in_off = 0;         // workspace offset of the previous intermediate
+  int64_t a_pitch = 0;       // elements
+  bool use_tc = false;
+  int kind = 0, block_n = 0, grid = 0, m_tiles = 0, n_tiles = 0, nkb = 0;
+  bool need_pack = false;
+  size_t pack_off = 0;
+  int64_t pack_pitch = 0;    // elements
+  size_t wt_off = 0;
+  int Kp = 0;
+  // cached tensor maps
+  CUtensorMap tmA, tmB;
+  const void* tmA_ptr = nullptr;
+  bool tmB_valid = false;
+};
+
+struct SdpaPlan {
+  SdpaParams prm = {};
+  int q_input = -1, k_input = -1, v_input = -1, mask_input = -1, out_pos = 0;
+  bool use_tc = false;
+  CUtensorMap tmQ, tmK, tmV;
+  const void *q_ptr = nullptr, *k_ptr = nullptr, *v_ptr = nullptr;
+};
+
+struct gc_compiled {
+  int device = 0, num_sms = 148;
+  int pattern = 0;
+  gc_compile_options_t opt = {};
+  std::vector<LayerPlan> layers;
+  SdpaPlan sdpa;
+  GemmSimtParams bmm = {};   // PAT_BATCHED_MATMUL
+  int n_in = 0, n_out = 0;
+  std::vector<size_t> in_bytes, out_bytes;
+  std::vector<int> in_constant;
+  size_t ws_bytes = 0;
+  void* ws = nullptr;
+  bool status_cleared = false;
+  bool prepacked = false;
+  std::vector<const void*> const_ptrs;   // constant input pointers seen at the last prepack
+  int launches = 0;
+  std::string desc;
+  // host staging
+  size_t staging_bytes = 0;
+  void* staging = nullptr;
+  std::vector<size_t> in_stage_off, out_stage_off;
+  std::vector<const void*> host_const_seen;
+};
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// 2-D row-major tensor [rows][inner] with a row pitch in bytes; box = [box_rows][box_inner].
+static gc_status_t make_tmap(CUtensorMap* m, const void* ptr, int dtype, uint64_t inner, uint64_t rows,
+                             uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_rows, int swizzle_bytes) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return fail(GC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+  CUtensorMapDataType dt = dtype == GC_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                           : dtype == GC_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
+                                              : CU_TENSOR_MAP_DATA_TYPE_UINT8;
+  cuuint64_t gdim[2] = {inner, rows};
+  cuuint64_t gstr[1] = {pitch_bytes};
+  cuuint32_t box[2] = {box_inner, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUtensorMapSwizzle sw = swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                          : swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                                : CU_TENSOR_MAP_SWIZZLE_NONE;
+  CUresult r = enc(m, dt, 2, const_cast<void*>(ptr), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(GC_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+  return GC_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// pattern formation
+// ------------------------------------------------------------------------------------------------
+static int act_of(int kind) {
+  return kind == GC_OP_RELU ? ACT_RELU : kind == GC_OP_GELU_TANH ? ACT_GELU_TANH : kind == GC_OP_SIGMOID ? ACT_SIGMOID : -1;
+}
+
+static gc_status_t match_mlp(const gc_partition& p, gc_compiled& c) {
+  size_t i = 0;
+  int64_t cur = -1;
+  while (i < p.ops.size()) {
+    const gc_op_t& mm = p.ops[i];
+    if (mm.kind != GC_OP_MATMUL) return fail(GC_ERR_UNSUPPORTED, "op %zu: expected a matmul to start a fused op", i);
+    const auto* a = p.lt(mm.in[0]);
+    const auto* w = p.lt(mm.in[1]);
+    if (a->ndims != 2 || w->ndims != 2) return fail(GC_ERR_UNSUPPORTED, "MLP layers need 2-D operands");
+    LayerPlan L;
+    if (c.layers.empty()) {
+      L.a_input = p.input_pos(mm.in[0]);
+      if (L.a_input < 0) return fail(GC_ERR_UNSUPPORTED, "first matmul must read a graph input");
+    } else if (mm.in[0] != cur) {
+      return fail(GC_ERR_UNSUPPORTED, "op %zu: matmul does not consume the previous fused op (not a chain)", i);
+    }
+    L.w_input = p.input_pos(mm.in[1]);
+    if (L.w_input < 0 || !w->is_constant) return fail(GC_ERR_UNSUPPORTED, "op %zu: weights must be a constant graph input", i);
+    L.M = static_cast<int>(a->dims[0]);
+    L.K = static_cast<int>(a->dims[1]);
+    L.N = static_cast<int>(p.lt(mm.out)->dims[1]);
+    L.a_dtype = a->dtype;
+    L.w_dtype = w->dtype;
+    L.transposed_w = mm.transpose_b;
+    const bool int_path = is_int8(a->dtype) && is_int8(w->dtype);
+    const bool flt_path = (a->dtype == GC_BF16 && w->dtype == GC_BF16) || (a->dtype == GC_F32 && w->dtype == GC_F32);
+    if (!int_path && !flt_path) return fail(GC_ERR_UNSUPPORTED, "op %zu: unsupported matmul operand dtypes", i);
+    if (int_path && w->zero_point != 0) return fail(GC_ERR_UNSUPPORTED, "weights must be symmetric (zero point 0)");
+    if (p.lt(mm.out)->dtype != (int_path ? GC_S32 : GC_F32))
+      return fail(GC_ERR_UNSUPPORTED, "op %zu: matmul result must be %s", i, int_path ? "s32" : "f32");
+    L.a_zp = int_path ? a->zero_point : 0;
+    L.epi.acc_is_int = int_path;
+    L.epi.out_dtype = int_path ? GC_S32 : GC_F32;
+    int64_t t = mm.out;
+    ++i;
+    auto next_is = [&](int kind) { return i < p.ops.size() && p.ops[i].kind == kind && p.ops[i].in[0] == t; };
+    if (next_is(GC_OP_DEQUANTIZE)) {
+      if (!int_path) return fail(GC_ERR_UNSUPPORTED, "dequantize after a float matmul");
+      L.epi.has_dq = 1;
+      L.epi.dq = a->scale * w->scale;   // fp32 product, the scale of the s32 result
+      L.epi.out_dtype = GC_F32;
+      t = p.ops[i++].out;
+    }
+    if (i < p.ops.size() && p.ops[i].kind == GC_OP_ADD && (p.ops[i].in[0] == t || p.ops[i].in[1] == t)) {
+      const int64_t other = p.ops[i].in[0] == t ? p.ops[i].in[1] : p.ops[i].in[0];
+      const auto* b = p.lt(other);
+      const int pos = p.input_pos(other);
+      if (pos >= 0 && b->dtype == GC_F32 && numel(*b) == L.N && b->dims[b->ndims - 1] == L.N) {
+        if (int_path && !L.epi.has_dq) return fail(GC_ERR_UNSUPPORTED, "bias add on an s32 tensor");
+        L.bias_input = pos;
+        t = p.ops[i++].out;
+      } else {
+        return fail(GC_ERR_UNSUPPORTED, "op %zu: add operand is not a per-column fp32 bias", i);
+      }
+    }
+    if (i < p.ops.size() && act_of(p.ops[i].kind) >= 0 && p.ops[i].in[0] == t) {
+      if (int_path && !L.epi.has_dq) return fail(GC_ERR_UNSUPPORTED, "activation on an s32 tensor");
+      L.epi.act = act_of(p.ops[i].kind);
+      t = p.ops[i++].out;
+    }
+    if (next_is(GC_OP_QUANTIZE)) {
+      const auto* o = p.lt(p.ops[i].out);
+      if (!is_int8(o->dtype)) return fail(GC_ERR_UNSUPPORTED, "quantize must produce u8 or s8");
+      if (int_path && !L.epi.has_dq) return fail(GC_ERR_UNSUPPORTED, "quantize on an s32 tensor");
+      L.epi.out_dtype = o->dtype;
+      L.epi.inv = 1.0f / o->scale;
+      L.epi.zp = o->zero_point;
+      t = p.ops[i++].out;
+    } else if (next_is(GC_OP_TYPECAST)) {
+      const auto* o = p.lt(p.ops[i].out);
+      if (o->dtype != GC_BF16 && o->dtype != GC_F32) return fail(GC_ERR_UNSUPPORTED, "typecast target must be bf16 or f32");
+      if (int_path && !L.epi.has_dq) return fail(GC_ERR_UNSUPPORTED, "typecast on an s32 tensor");
+      L.epi.out_dtype = o->dtype;
+      t = p.ops[i++].out;
+    }
+    if (p.lt(t)->dtype != L.epi.out_dtype) return fail(GC_ERR_UNSUPPORTED, "fused op result dtype does not match its logical tensor");
+    const bool last = i == p.ops.size();
+    if (last) {
+      L.out_pos = p.output_pos(t);
+      if (L.out_pos < 0 || p.out_ids.size() != 1) return fail(GC_ERR_UNSUPPORTED, "the chain's last tensor must be the only graph output");
+    } else {
+      if (p.output_pos(t) >= 0 || p.consumers(t) != 1)
+        return fail(GC_ERR_UNSUPPORTED, "intermediate tensors must have exactly one consumer and not be outputs");
+      if (L.epi.out_dtype == GC_S32) return fail(GC_ERR_UNSUPPORTED, "an s32 tensor cannot feed the next matmul");
+    }
+    L.out_elem = dtype_bytes(L.epi.out_dtype);
+    cur = t;
+    c.layers.push_back(L);
+  }
+  return c.layers.empty() ? fail(GC_ERR_UNSUPPORTED, "no matmul found") : GC_OK;
+}
+
+static gc_status_t match_sdpa(const gc_partition& p, gc_compiled& c) {
+  SdpaPlan& s = c.sdpa;
+  SdpaParams& prm = s.prm;
+  size_t i = 0;
+  const gc_op_t& m1 = p.ops[0];
+  const auto *q = p.lt(m1.in[0]), *k = p.lt(m1.in[1]);
+  if (!m1.transpose_b || q->ndims != 4 || !same_dims(*q, *k)) return fail(GC_ERR_UNSUPPORTED, "attention: Q and K must be [B,H,S,D] with transpose_b");
+  s.q_input = p.input_pos(m1.in[0]);
+  s.k_input = p.input_pos(m1.in[1]);
+  if (s.q_input < 0 || s.k_input < 0) return fail(GC_ERR_UNSUPPORTED, "attention: Q and K must be graph inputs");
+  prm.B = static_cast<int>(q->dims[0]);
+  prm.H = static_cast<int>(q->dims[1]);
+  prm.S = static_cast<int>(q->dims[2]);
+  prm.D = static_cast<int>(q->dims[3]);
+  const bool i8 = is_int8(q->dtype) && is_int8(k->dtype);
+  if (!i8 && !(q->dtype == GC_BF16 && k->dtype == GC_BF16)) return fail(GC_ERR_UNSUPPORTED, "attention: operands must be bf16 or 8-bit");
+  prm.is_int8 = i8;
+  prm.zp_q = i8 ? q->zero_point : 0;
+  prm.zp_k = i8 ? k->zero_point : 0;
+  prm.q_signed = q->dtype == GC_S8;
+  prm.k_signed = k->dtype == GC_S8;
+  prm.dq1 = i8 ? q->scale * k->scale : 1.0f;
+  prm.scalar = 1.0f;
+  int64_t t = m1.out;
+  ++i;
+  auto next_is = [&](int kind) { return i < p.ops.size() && p.ops[i].kind == kind && p.ops[i].in[0] == t; };
+  if (i8) {
+    if (!next_is(GC_OP_DEQUANTIZE)) return fail(GC_ERR_UNSUPPORTED, "attention: int8 scores must be dequantized");
+    t = p.ops[i++].out;
+  }
+  if (next_is(GC_OP_MUL)) {
+    prm.scalar = p.ops[i].scalar;
+    t = p.ops[i++].out;
+  }
+  if (i < p.ops.size() && p.ops[i].kind == GC_OP_ADD && p.ops[i].in[0] == t) {
+    const auto* mk = p.lt(p.ops[i].in[1]);
+    s.mask_input = p.input_pos(p.ops[i].in[1]);
+    if (s.mask_input < 0 || mk->dtype != GC_F32 || mk->ndims != 4 || mk->dims[0] != prm.B || mk->dims[1] != 1 ||
+        mk->dims[2] != 1 || mk->dims[3] != prm.S)
+      return fail(GC_ERR_UNSUPPORTED, "attention: mask must be an fp32 graph input [B,1,1,S]");
+    t = p.ops[i++].out;
+  }
+  if (!next_is(GC_OP_SOFTMAX)) return fail(GC_ERR_UNSUPPORTED, "attention: expected softmax");
+  t = p.ops[i++].out;
+  if (i8) {
+    if (!next_is(GC_OP_QUANTIZE)) return fail(GC_ERR_UNSUPPORTED, "attention: int8 probabilities must be quantized");
+    const auto* pq = p.lt(p.ops[i].out);
+    if (pq->dtype != GC_U8) return fail(GC_ERR_UNSUPPORTED, "attention: quantized probabilities must be u8");
+    prm.p_is_quant = 1;
+    prm.inv_p = 1.0f / pq->scale;
+    prm.zp_p = pq->zero_point;
+    t = p.ops[i++].out;
+  } else {
+    if (!next_is(GC_OP_TYPECAST) || p.lt(p.ops[i].out)->dtype != GC_BF16)
+      return fail(GC_ERR_UNSUPPORTED, "attention: bf16 path expects the probabilities cast to bf16");
+    t = p.ops[i++].out;
+  }
+  if (!(i < p.ops.size() && p.ops[i].kind == GC_OP_MATMUL && p.ops[i].in[0] == t && !p.ops[i].transpose_b))
+    return fail(GC_ERR_UNSUPPORTED, "attention: expected the P.V matmul");
+  const auto* pt = p.lt(t);
+  const auto* v = p.lt(p.ops[i].in[1]);
+  s.v_input = p.input_pos(p.ops[i].in[1]);
+  if (s.v_input < 0 || !same_dims(*v, *q) || (i8 ? !is_int8(v->dtype) : v->dtype != GC_BF16))
+    return fail(GC_ERR_UNSUPPORTED, "attention: V must be a graph input shaped and typed like Q");
+  prm.zp_v = i8 ? v->zero_point : 0;
+  prm.v_signed = v->dtype == GC_S8;
+  prm.dq2 = i8 ? pt->scale * v->scale : 1.0f;
+  t = p.ops[i++].out;
+  if (i8) {
+    if (!next_is(GC_OP_DEQUANTIZE)) return fail(GC_ERR_UNSUPPORTED, "attention: int8 output must be dequantized");
+    t = p.ops[i++].out;
+    if (!next_is(GC_OP_QUANTIZE)) return fail(GC_ERR_UNSUPPORTED, "attention: int8 output must be requantized");
+    const auto* o = p.lt(p.ops[i].out);
+    if (!is_int8(o->dtype)) return fail(GC_ERR_UNSUPPORTED, "attention: output must be u8 or s8");
+    prm.out_dtype = o->dtype;
+    prm.inv_o = 1.0f / o->scale;
+    prm.zp_o = o->zero_point;
+    t = p.ops[i++].out;
+  } else {
+    if (!next_is(GC_OP_TYPECAST) || p.lt(p.ops[i].out)->dtype != GC_BF16)
+      return fail(GC_ERR_UNSUPPORTED, "attention: bf16 path expects a bf16 output");
+    prm.out_dtype = GC_BF16;
+    t = p.ops[i++].out;
+  }
+  if (i != p.ops.size() || p.out_ids.size() != 1 || p.output_pos(t) != 0)
+    return fail(GC_ERR_UNSUPPORTED, "attention: trailing ops or wrong outputs");
+  return GC_OK;
+}
+
+static void choose_tile(LayerPlan& L, int num_sms) {
+  const int esz = dtype_bytes(L.a_dtype);
+  const int k_elems = 128 / esz;
+  L.m_tiles = (L.M + 127) / 128;
+  L.nkb = (L.K + k_elems - 1) / k_elems;
+  const int cands[5] = {256, 128, 64, 32, 16};
+  int pick = 0;
+  for (int bn : cands) {
+    if (bn > 16 && bn > L.N) continue;
+    const int tiles = L.m_tiles * ((L.N + bn - 1) / bn);
+    if (tiles >= num_sms) {
+      pick = bn;
+      break;
+    }
+  }
+  if (!pick) pick = L.N >= 32 ? 32 : 16;
+  L.block_n = pick;
+  L.n_tiles = (L.N + pick - 1) / pick;
+  const int tiles = L.m_tiles * L.n_tiles;
+  L.grid = tiles < num_sms ? tiles : num_sms;
+}
+
+extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, const gc_compile_options_t* opt,
+                                  gc_compiled_t** out) {
+  if (!p || !out) return fail(GC_ERR_INVALID_ARG, "null argument");
+  cudaDeviceProp prop = {};
+  if (cuda_device == GC_DEVICE_PLAN_ONLY) {
+    // plan for a nominal B200 without touching any device; the result cannot be executed
+    prop.major = 10;
+    prop.multiProcessorCount = 148;
+    prop.sharedMemPerBlockOptin = 227 * 1024;
+  } else {
+    int ndev = 0;
+    CUDA_TRY(cudaGetDeviceCount(&ndev));
+    if (cuda_device < 0 || cuda_device >= ndev) return fail(GC_ERR_INVALID_ARG, "no such CUDA device %d", cuda_device);
+    CUDA_TRY(cudaGetDeviceProperties(&prop, cuda_device));
+    if (prop.major != 10) return fail(GC_ERR_UNSUPPORTED, "device %d is sm_%d%d; this library is built for sm_100a only", cuda_device, prop.major, prop.minor);
+  }
+  auto c = new gc_compiled();
+  auto bail = [&](gc_status_t st) {
+    delete c;
+    return st;
+  };
+  c->device = cuda_device;
+  c->num_sms = prop.multiProcessorCount;
+  if (opt) c->opt = *opt;
+  c->n_in = static_cast<int>(p->in_ids.size());
+  c->n_out = static_cast<int>(p->out_ids.size());
+  for (auto id : p->in_ids) {
+    c->in_bytes.push_back(static_cast<size_t>(numel(*p->lt(id))) * dtype_bytes(p->lt(id)->dtype));
+    c->in_constant.push_back(p->lt(id)->is_constant);
+  }
+  for (auto id : p->out_ids) c->out_bytes.push_back(static_cast<size_t>(numel(*p->lt(id))) * dtype_bytes(p->lt(id)->dtype));
+  c->const_ptrs.assign(c->n_in, nullptr);
+  c->host_const_seen.assign(c->n_in, nullptr);
+
+  size_t ws = 256;   // [0,4): status word
+  char line[256];
+  const gc_op_t& first = p->ops[0];
+  const bool batched = first.kind == GC_OP_MATMUL && p->lt(first.in[1])->ndims > 2;
+  if (batched && p->ops.size() == 1) {
+    // a bare batched matmul: the raw accumulator is the output
+    const auto *a = p->lt(first.in[0]), *b = p->lt(first.in[1]), *o = p->lt(first.out);
+    const bool i8 = is_int8(a->dtype) && is_int8(b->dtype);
+    if (!first.transpose_b) return bail(fail(GC_ERR_UNSUPPORTED, "batched matmul needs transpose_b"));
+    if (!i8 && !((a->dtype == GC_BF16 || a->dtype == GC_F32) && a->dtype == b->dtype))
+      return bail(fail(GC_ERR_UNSUPPORTED, "batched matmul operand dtypes"));
+    if (o->dtype != (i8 ? GC_S32 : GC_F32) || p->input_pos(first.in[0]) != 0 || p->input_pos(first.in[1]) != 1 ||
+        p->output_pos(first.out) != 0)
+      return bail(fail(GC_ERR_UNSUPPORTED, "batched matmul: inputs must be (A, B) and the result the output"));
+    c->pattern = PAT_BATCHED_MATMUL;
+    GemmSimtParams& g = c->bmm;
+    g.M = static_cast<int>(a->dims[a->ndims - 2]);
+    g.K = static_cast<int>(a->dims[a->ndims - 1]);
+    g.N = static_cast<int>(b->dims[b->ndims - 2]);
+    g.batch = static_cast<int>(numel(*a) / (static_cast<int64_t>(g.M) * g.K));
+    g.a_pitch = g.K;
+    g.w_pitch = g.K;
+    g.a_batch_stride = static_cast<int64_t>(g.M) * g.K;
+    g.w_batch_stride = static_cast<int64_t>(g.N) * g.K;
+    g.out_batch_stride = static_cast<int64_t>(g.M) * g.N;
+    g.out_pitch = g.N;
+    g.a_dtype = a->dtype;
+    g.w_dtype = b->dtype;
+    g.a_zp = i8 ? a->zero_point : 0;
+    g.w_zp = i8 ? b->zero_point : 0;
+    g.epi.acc_is_int = i8;
+    g.epi.out_dtype = o->dtype;
+    c->launches = 1;
+    c->desc = "pattern=batched_matmul kernel=cuda-core\n";
+  } else if (batched) {
+    gc_status_t st = match_sdpa(*p, *c);
+    if (st != GC_OK) return bail(st);
+    c->pattern = PAT_SDPA;
+    SdpaParams& s = c->sdpa.prm;
+    bool tc = !c->opt.force_generic && s.D == 64 && s.S % 128 == 0 && s.S <= 384 &&
+              sdpa_tc_smem_bytes(s.S, s.is_int8) <= static_cast<size_t>(prop.sharedMemPerBlockOptin);
+    if (s.is_int8)
+      tc = tc && s.zp_p == 0 && ((s.q_signed && s.zp_q == 0) || (!s.q_signed && s.zp_q == 128)) &&
+           ((s.k_signed && s.zp_k == 0) || (!s.k_signed && s.zp_k == 128));
+    if (!tc && s.S > 8192) return bail(fail(GC_ERR_UNSUPPORTED, "attention: sequence length %d not supported", s.S));
+    c->sdpa.use_tc = tc;
+    c->launches = 1;
+    snprintf(line, sizeof(line), "pattern=attention %s B=%d H=%d S=%d D=%d kernel=%s\n", s.is_int8 ? "int8" : "bf16", s.B,
+             s.H, s.S, s.D, tc ? "tcgen05" : "cuda-core");
+    c->desc = line;
+  } else {
+    gc_status_t st = match_mlp(*p, *c);
+    if (st != GC_OK) return bail(st);
+    c->pattern = PAT_MLP;
+    c->desc = "pattern=mlp_chain\n";
+    // prepacked weights
+    for (auto& L : c->layers) {
+      const int esz = dtype_bytes(L.w_dtype);
+      L.Kp = static_cast<int>(align_up(static_cast<size_t>(L.K) * esz, 128) / esz);
+      L.wt_off = ws;
+      ws = align_up(ws + static_cast<size_t>(L.N) * L.Kp * esz, 1024);
+    }
+    // temporaries between fused ops: two buffers reused alternately (life spans never overlap by
+    // more than one layer), each sized for the largest tensor it ever holds
+    size_t act_bytes[2] = {0, 0};
+    for (size_t l = 0; l + 1 < c->layers.size(); ++l) {
+      LayerPlan& L = c->layers[l];
+      L.out_pitch = static_cast<int64_t>(align_up(static_cast<size_t>(L.N), 16));
+      const size_t b = static_cast<size_t>(L.M) * L.out_pitch * L.out_elem;
+      if (b > act_bytes[l & 1]) act_bytes[l & 1] = b;
+    }
+    size_t act_off[2];
+    act_off[0] = ws;
+    ws = align_up(ws + act_bytes[0], 1024);
+    act_off[1] = ws;
+    ws = align_up(ws + act_bytes[1], 1024);
+    for (size_t l = 0; l < c->layers.size(); ++l) {
+      LayerPlan& L = c->layers[l];
+      const int esz = dtype_bytes(L.a_dtype);
+      if (l + 1 < c->layers.size()) L.out_off = act_off[l & 1];
+      else L.out_pitch = L.N;
+      if (l > 0) {
+        L.in_off = act_off[(l - 1) & 1];
+        L.a_pitch = c->layers[l - 1].out_pitch;
+      } else {
+        L.a_pitch = L.K;
+      }
+      const bool dt_ok = (is_int8(L.a_dtype) && L.w_dtype == GC_S8 && L.a_zp == 0) || L.a_dtype == GC_BF16 ||
+                         L.a_dtype == GC_F32;
+      L.use_tc = !c->opt.force_generic && dt_ok && L.N >= 16 && L.N % 16 == 0;
+      if (L.use_tc) {
+        L.kind = is_int8(L.a_dtype) ? 0 : (L.a_dtype == GC_BF16 ? 1 : 2);
+        choose_tile(L, c->num_sms);
+        if ((L.a_pitch * esz) % 16 != 0) {   // graph-entry reorder: TMA needs 16-byte row pitches
+          L.need_pack = true;
+          L.pack_pitch = static_cast<int64_t>(align_up(static_cast<size_t>(L.K) * esz, 16) / esz);
+          L.pack_off = ws;
+          ws = align_up(ws + static_cast<size_t>(L.M) * L.pack_pitch * esz, 1024);
+          c->launches += 1;
+        }
+      }
+      c->launches += 1;
+      snprintf(line, sizeof(line), "  layer %zu: M=%d K=%d N=%d kernel=%s block_n=%d grid=%d%s act=%d out=%d\n", l, L.M, L.K,
+               L.N, L.use_tc ? (L.kind == 0 ? "tcgen05.i8" : L.kind == 1 ? "tcgen05.bf16" : "tcgen05.tf32") : "cuda-core",
+               L.block_n, L.grid, L.need_pack ? " +pack" : "", L.epi.act, L.epi.out_dtype);
+      c->desc += line;
+    }
+  }
+  c->ws_bytes = align_up(ws, 1024);
+  // host staging layout
+  size_t so = 0;
+  for (int i = 0; i < c->n_in; ++i) {
+    c->in_stage_off.push_back(so);
+    so = align_up(so + c->in_bytes[i], 256);
+  }
+  for (int i = 0; i < c->n_out; ++i) {
+    c->out_stage_off.push_back(so);
+    so = align_up(so + c->out_bytes[i], 256);
+  }
+  c->staging_bytes = so;
+  *out = c;
+  return GC_OK;
+}
+
+extern "C" void gc_compiled_destroy(gc_compiled_t* c) { delete c; }
+
+extern "C" gc_status_t gc_workspace_bytes(const gc_compiled_t* c, size_t* bytes) {
+  if (!c || !bytes) return fail(GC_ERR_INVALID_ARG, "null argument");
+  *bytes = c->ws_bytes;
+  return GC_OK;
+}
+
+extern "C" gc_status_t gc_set_workspace(gc_compiled_t* c, void* ws, size_t bytes) {
+  if (!c || !ws) return fail(GC_ERR_INVALID_ARG, "null argument");
+  if (bytes < c->ws_bytes) return fail(GC_ERR_INVALID_ARG, "workspace too small: %zu < %zu", bytes, c->ws_bytes);
+  if (reinterpret_cast<uintptr_t>(ws) % 256) return fail(GC_ERR_ALIGNMENT, "workspace must be 256-byte aligned");
+  c->ws = ws;
+  c->prepacked = false;
+  c->status_cleared = false;
+  for (auto& L : c->layers) {
+    L.tmA_ptr = nullptr;
+    L.tmB_valid = false;
+  }
+  return GC_OK;
+}
+
+extern "C" gc_status_t gc_host_staging_bytes(const gc_compiled_t* c, size_t* bytes) {
+  if (!c || !bytes) return fail(GC_ERR_INVALID_ARG, "null argument");
+  *bytes = c->staging_bytes;
+  return GC_OK;
+}
+
+extern "C" gc_status_t gc_set_host_staging(gc_compiled_t* c, void* p, size_t bytes) {
+  if (!c || !p) return fail(GC_ERR_INVALID_ARG, "null argument");
+  if (bytes < c->staging_bytes) return fail(GC_ERR_INVALID_ARG, "staging area too small");
+  if (reinterpret_cast<uintptr_t>(p) % 256) return fail(GC_ERR_ALIGNMENT, "staging area must be 256-byte aligned");
+  c->staging = p;
+  std::fill(c->host_const_seen.begin(), c->host_const_seen.end(), nullptr);
+  return GC_OK;
+}
+
+extern "C" gc_status_t gc_launches_per_execute(const gc_compiled_t* c, int32_t* n) {
+  if (!c || !n) return fail(GC_ERR_INVALID_ARG, "null argument");
+  *n = c->launches;
+  return GC_OK;
+}
+
+extern "C" const char* gc_plan_description(const gc_compiled_t* c) { return c ? c->desc.c_str() : ""; }
+
+// ------------------------------------------------------------------------------------------------
+// execute
+// ------------------------------------------------------------------------------------------------
+static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* in, void* const* out) {
+  char* ws = static_cast<char*>(c.ws);
+  uint32_t* status = reinterpret_cast<uint32_t*>(ws);
+  // constant-weight preprocessing: once, and again only if a constant arrives at a new address
+  bool need = !c.prepacked;
+  for (auto& L : c.layers) need = need || c.const_ptrs[L.w_input] != in[L.w_input];
+  if (need) {
+    for (auto& L : c.layers) {
+      CUDA_TRY(launch_prepack_weight(in[L.w_input], ws + L.wt_off, L.K, L.N, L.Kp, L.transposed_w, L.w_dtype, st));
+      c.const_ptrs[L.w_input] = in[L.w_input];
+    }
+    c.prepacked = true;
+  }
+  for (size_t l = 0; l < c.layers.size(); ++l) {
+    LayerPlan& L = c.layers[l];
+    const int esz = dtype_bytes(L.a_dtype);
+    const void* A = l == 0 ? in[L.a_input] : ws + L.in_off;
+    int64_t a_pitch = L.a_pitch;
+    void* O = L.out_pos >= 0 ? out[L.out_pos] : ws + L.out_off;
+    Epilogue e = L.epi;
+    e.bias = L.bias_input >= 0 ? static_cast<const float*>(in[L.bias_input]) : nullptr;
+    if (L.use_tc) {
+      if (L.need_pack) {
+        CUDA_TRY(launch_pack_rows(A, ws + L.pack_off, L.M, L.a_pitch * esz, L.pack_pitch * esz, st));
+        A = ws + L.pack_off;
+        a_pitch = L.pack_pitch;
+      }
+      const int k_elems = 128 / esz;
+      if (L.tmA_ptr != A) {
+        gc_status_t s = make_tmap(&L.tmA, A, L.a_dtype, L.K, L.M, a_pitch * esz, k_elems, 128, 128);
+        if (s != GC_OK) return s;
+        L.tmA_ptr = A;
+      }
+      if (!L.tmB_valid) {
+        gc_status_t s = make_tmap(&L.tmB, ws + L.wt_off, L.w_dtype, L.Kp, L.N, static_cast<uint64_t>(L.Kp) * esz, k_elems,
+                                  L.block_n, 128);
+        if (s != GC_OK) return s;
+        L.tmB_valid = true;
+      }
+      GemmTcParams g = {};
+      g.M = L.M;
+      g.N = L.N;
+      g.K = L.K;
+      g.num_k_blocks = L.nkb;
+      g.m_tiles = L.m_tiles;
+      g.n_tiles = L.n_tiles;
+      g.out = O;
+      g.out_pitch = L.out_pitch;
+      g.epi = e;
+      g.status = status;
+      const bool pdl = !c.opt.no_chain_fusion && l > 0 && !L.need_pack;
+      CUDA_TRY(launch_gemm_tc(L.kind, L.block_n, L.a_dtype == GC_S8, L.tmA, L.tmB, g, L.grid, pdl, st));
+    } else {
+      GemmSimtParams g = {};
+      g.A = A;
+      g.Wt = ws + L.wt_off;
+      g.a_pitch = a_pitch;
+      g.w_pitch = L.Kp;
+      g.M = L.M;
+      g.N = L.N;
+      g.K = L.K;
+      g.batch = 1;
+      g.a_dtype = L.a_dtype;
+      g.w_dtype = L.w_dtype;
+      g.a_zp = L.a_zp;
+      g.w_zp = 0;
+      g.out = O;
+      g.out_pitch = L.out_pitch;
+      g.epi = e;
+      CUDA_TRY(launch_gemm_simt(g, st));
+    }
+  }
+  return GC_OK;
+}
+
+static gc_status_t run_sdpa(gc_compiled& c, cudaStream_t st, const void* const* in, void* const* out) {
+  SdpaPlan& s = c.sdpa;
+  SdpaParams prm = s.prm;
+  prm.Q = in[s.q_input];
+  prm.K = in[s.k_input];
+  prm.V = in[s.v_input];
+  prm.mask = s.mask_input >= 0 ? static_cast<const float*>(in[s.mask_input]) : nullptr;
+  prm.O = out[0];
+  prm.status = reinterpret_cast<uint32_t*>(c.ws);
+  if (!s.use_tc) {
+    CUDA_TRY(launch_sdpa_simt(prm, st));
+    return GC_OK;
+  }
+  const int dt = prm.is_int8 ? GC_U8 : GC_BF16;
+  const int esz = prm.is_int8 ? 1 : 2;
+  const uint64_t rows = static_cast<uint64_t>(prm.B) * prm.H * prm.S;
+  const int swz = prm.is_int8 ? 64 : 128;
+  if (s.q_ptr != prm.Q) {
+    gc_status_t r = make_tmap(&s.tmQ, prm.Q, dt, prm.D, rows, static_cast<uint64_t>(prm.D) * esz, prm.D, 128, swz);
+    if (r != GC_OK) return r;
+    s.q_ptr = prm.Q;
+  }
+  if (s.k_ptr != prm.K) {
+    gc_status_t r = make_tmap(&s.tmK, prm.K, dt, prm.D, rows, static_cast<uint64_t>(prm.D) * esz, prm.D, 128, swz);
+    if (r != GC_OK) return r;
+    s.k_ptr = prm.K;
+  }
+  if (s.v_ptr != prm.V) {
+    gc_status_t r = make_tmap(&s.tmV, prm.V, dt, prm.D, rows, static_cast<uint64_t>(prm.D) * esz, prm.D, 128, swz);
+    if (r != GC_OK) return r;
+    s.v_ptr = prm.V;
+  }
+  CUDA_TRY(launch_sdpa_tc(s.tmQ, s.tmK, s.tmV, prm, st));
+  return GC_OK;
+}
+
+extern "C" gc_status_t gc_execute(gc_compiled_t* c, void* cuda_stream, const void* const* in_dev, int32_t n_in,
+                                  void* const* out_dev, int32_t n_out) {
+  if (!c || !in_dev || !out_dev) return fail(GC_ERR_INVALID_ARG, "null argument");
+  if (n_in != c->n_in || n_out != c->n_out)
+    return fail(GC_ERR_INVALID_ARG, "expected %d inputs and %d outputs, got %d and %d", c->n_in, c->n_out, n_in, n_out);
+  if (c->device < 0) return fail(GC_ERR_STATE, "compiled with GC_DEVICE_PLAN_ONLY: cannot execute");
+  if (!c->ws) return fail(GC_ERR_STATE, "gc_set_workspace has not been called");
+  for (int i = 0; i < n_in; ++i) {
+    if (!in_dev[i]) return fail(GC_ERR_INVALID_ARG, "input %d is null", i);
+    if (reinterpret_cast<uintptr_t>(in_dev[i]) % 16) return fail(GC_ERR_ALIGNMENT, "input %d is not 16-byte aligned", i);
+  }
+  for (int i = 0; i < n_out; ++i) {
+    if (!out_dev[i]) return fail(GC_ERR_INVALID_ARG, "output %d is null", i);
+    if (reinterpret_cast<uintptr_t>(out_dev[i]) % 16) return fail(GC_ERR_ALIGNMENT, "output %d is not 16-byte aligned", i);
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int cur = -1;
+  CUDA_TRY(cudaGetDevice(&cur));
+  if (cur != c->device) CUDA_TRY(cudaSetDevice(c->device));
+  if (!c->status_cleared) {
+    CUDA_TRY(cudaMemsetAsync(c->ws, 0, 256, st));
+    c->status_cleared = true;
+  }
+  gc_status_t r;
+  if (c->pattern == PAT_MLP) {
+    r = run_mlp(*c, st, in_dev, out_dev);
+  } else if (c->pattern == PAT_SDPA) {
+    r = run_sdpa(*c, st, in_dev, out_dev);
+  } else {
+    GemmSimtParams g = c->bmm;
+    g.A = in_dev[0];
+    g.Wt = in_dev[1];
+    g.out = out_dev[0];
+    cudaError_t e = launch_gemm_simt(g, st);
+    r = e == cudaSuccess ? GC_OK : fail(GC_ERR_CUDA, "launch_gemm_simt: %s", cudaGetErrorString(e));
+  }
+  return r;
+}
+
+extern "C" gc_status_t gc_execute_host(gc_compiled_t* c, void* cuda_stream, const void* const* in_host, int32_t n_in,
+                                       void* const* out_host, int32_t n_out) {
+  if (!c || !in_host || !out_host) return fail(GC_ERR_INVALID_ARG, "null argument");
+  if (n_in != c->n_in || n_out != c->n_out) return fail(GC_ERR_INVALID_ARG, "wrong number of inputs or outputs");
+  if (!c->staging) return fail(GC_ERR_STATE, "gc_set_host_staging has not been called");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* sg = static_cast<char*>(c->staging);
+  std::vector<const void*> din(n_in);
+  std::vector<void*> dout(n_out);
+  for (int i = 0; i < n_in; ++i) {
+    if (!in_host[i]) return fail(GC_ERR_INVALID_ARG, "input %d is null", i);
+    din[i] = sg + c->in_stage_off[i];
+    if (!c->in_constant[i] || c->host_const_seen[i] != in_host[i]) {
+      CUDA_TRY(cudaMemcpyAsync(sg + c->in_stage_off[i], in_host[i], c->in_bytes[i], cudaMemcpyHostToDevice, st));
+      c->host_const_seen[i] = in_host[i];
+    }
+  }
+  for (int i = 0; i < n_out; ++i) {
+    if (!out_host[i]) return fail(GC_ERR_INVALID_ARG, "output %d is null", i);
+    dout[i] = sg + c->out_stage_off[i];
+  }
+  gc_status_t r = gc_execute(c, cuda_stream, din.data(), n_in, dout.data(), n_out);
+  if (r != GC_OK) return r;
+  for (int i = 0; i < n_out; ++i)
+    CUDA_TRY(cudaMemcpyAsync(out_host[i], sg + c->out_stage_off[i], c->out_bytes[i], cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaStreamSynchronize(st));
+  return GC_OK;
+}
+
+extern "C" gc_status_t gc_query_status(gc_compiled_t* c, void* cuda_stream) {
+  if (!c) return fail(GC_ERR_INVALID_ARG, "null argument");
+  if (!c->ws) return fail(GC_ERR_STATE, "gc_set_workspace has not been called");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  uint32_t word = 0;
+  CUDA_TRY(cudaMemcpyAsync(&word, c->ws, sizeof(word), cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaStreamSynchronize(st));
+  if (word != 0) return fail(GC_ERR_TIMEOUT, "a bounded device-side wait expired (code 0x%x)", word);
+  return GC_OK;
+}

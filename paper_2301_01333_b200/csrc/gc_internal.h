@@ -1,0 +1,95 @@
+// Internal declarations shared by the host-side planner (gc_api.cu) and the kernel translation units.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/gc.h"
+
+namespace gc {
+
+enum Act : int { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SIGMOID = 3 };
+
+// What a fused op does to each accumulator element before it is stored (the post-op anchor of the
+// fused-op template, Section IV).  Order is fixed:
+//   t = acc                      (float accumulator)            or
+//   t = (float)acc * dq          (s32 accumulator, has_dq)      or   raw s32 store (no has_dq)
+//   t = t + bias[n]              (bias != nullptr)
+//   t = act(t)
+//   out = t                      (f32)  |  bf16(t)  |  saturate(rne(t * inv) + zp)  (u8 / s8)
+// On the integer path every multiply/add is a separately rounded fp32 operation.
+struct Epilogue {
+  int acc_is_int;
+  int has_dq;
+  float dq;
+  const float* bias;
+  int act;
+  int out_dtype;   // gc_dtype_t
+  float inv;       // 1.0f / scale_out
+  int zp;          // zero point of the quantised output
+};
+
+struct GemmTcParams {
+  int M, N, K;
+  int num_k_blocks, m_tiles, n_tiles;
+  void* out;
+  int64_t out_pitch;   // elements
+  Epilogue epi;
+  uint32_t* status;
+};
+
+struct GemmSimtParams {
+  const void* A;       // [batch][M][a_pitch]
+  const void* Wt;      // [batch][N][w_pitch]   (reduction axis contiguous)
+  int64_t a_pitch, w_pitch, a_batch_stride, w_batch_stride, out_batch_stride;
+  int M, N, K, batch;
+  int a_dtype, w_dtype;  // gc_dtype_t
+  int a_zp, w_zp;
+  void* out;
+  int64_t out_pitch;
+  Epilogue epi;
+};
+
+struct SdpaParams {
+  const void* Q;
+  const void* K;
+  const void* V;
+  const float* mask;   // [B, S_kv] or nullptr
+  void* O;
+  int B, H, S, D;
+  int is_int8;         // u8/s8 operands (else bf16)
+  int zp_q, zp_k, zp_v;
+  float dq1;           // scale_q * scale_k   (int8)
+  float scalar;        // the Mul op's constant (1/sqrt(d)); 1 if absent
+  int p_is_quant;      // probabilities quantised (int8 path)
+  float inv_p;         // 1 / scale_p
+  int zp_p;
+  float dq2;           // scale_p * scale_v
+  float inv_o;         // 1 / scale_o
+  int zp_o;
+  int out_dtype;       // GC_BF16 or GC_U8 / GC_S8
+  int q_signed, k_signed, v_signed;   // s8 instead of u8 storage
+  uint32_t* status;
+};
+
+// ---- launchers (each enqueues exactly one kernel on the stream and returns cudaGetLastError) ----
+cudaError_t launch_pack_rows(const void* src, void* dst, int rows, int64_t src_pitch_bytes, int64_t dst_pitch_bytes,
+                             cudaStream_t s);
+// W given as [K,N] (transposed = 0) or [N,K] (transposed = 1), dense; writes Wt[N][Kp] with the
+// reduction axis contiguous and zero padded.  f32 weights are rounded to tf32 (nearest, ties away).
+cudaError_t launch_prepack_weight(const void* W, void* Wt, int K, int N, int Kp, int transposed, int dtype,
+                                  cudaStream_t s);
+cudaError_t launch_gemm_simt(const GemmSimtParams& p, cudaStream_t s);
+cudaError_t launch_sdpa_simt(const SdpaParams& p, cudaStream_t s);
+
+// kind: 0 = i8 (u8/s8 x s8 -> s32), 1 = bf16, 2 = tf32.  a_signed only matters for kind 0.
+bool gemm_tc_supported_block_n(int block_n);
+size_t gemm_tc_smem_bytes(int block_n);
+cudaError_t launch_gemm_tc(int kind, int block_n, int a_signed, const CUtensorMap& tmA, const CUtensorMap& tmB,
+                           const GemmTcParams& p, int grid, bool pdl, cudaStream_t s);
+
+size_t sdpa_tc_smem_bytes(int S, int is_int8);
+cudaError_t launch_sdpa_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const SdpaParams& p,
+                           cudaStream_t s);
+
+}  // namespace gc

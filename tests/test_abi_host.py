@@ -1,0 +1,117 @@
+"""Host-side checks that need no GPU: the C-ABI library loads and exports every symbol the header
+declares, argument validation, pattern formation and planning (plan-only compile)."""
+import os
+import re
+
+import pytest
+
+from paper_2301_01333_b200 import binding as B
+from paper_2301_01333_b200 import build as gc_build
+from paper_2301_01333_b200 import workloads as W
+from paper_2301_01333_b200.graph import Graph
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    gc_build.build()
+
+
+def test_library_exports_every_declared_symbol():
+    text = open(os.path.join(ROOT, "include", "gc.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    declared = set(re.findall(r"\b(gc_[a-z_]+)\s*\(", text))
+    assert declared == set(B.EXPORTS)
+    lib = B.load_library()
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert "sm_100a" in B.gc_version()
+
+
+def plan(g, **kw):
+    return B.CompiledPartition(g, device=B.GC_DEVICE_PLAN_ONLY, **kw)
+
+
+def test_plans_for_the_five_configs():
+    c1 = plan(W.mlp_f32().graph)
+    assert c1.plan.count("tcgen05.tf32") == 3 and "+pack" in c1.plan
+    c2 = plan(W.mlp_int8().graph)
+    assert c2.plan.count("tcgen05.i8") == 4 and c2.plan.count("cuda-core") == 1      # 256 -> 1 is a GEMV
+    c5 = plan(W.ffn_bf16().graph)
+    assert c5.plan.count("tcgen05.bf16") == 2 and c5.plan.count("block_n=256") == 2
+    assert c5.launches == 2
+    c3 = plan(W.mha_bf16().graph)
+    assert "attention bf16" in c3.plan and "tcgen05" in c3.plan
+    c4 = plan(W.mha_int8().graph)
+    assert "attention int8" in c4.plan and "S=384" in c4.plan and "tcgen05" in c4.plan
+    # workspace: prepacked weights + two reused activation buffers (+ padded input copy)
+    assert c5.workspace_bytes >= 16 * 2 ** 20 + 64 * 2 ** 20
+    assert c2.workspace_bytes < 4 * 2 ** 20
+    for c in (c1, c2, c3, c4, c5):
+        c.close()
+
+
+def test_force_generic_and_ragged_shapes_use_cuda_core_kernels():
+    c = plan(W.mlp_int8().graph, force_generic=True)
+    assert "tcgen05" not in c.plan
+    c = plan(W.mlp_f32(batch=3, dims=(5, 7, 3)).graph)
+    assert "tcgen05" not in c.plan           # N not a multiple of 16
+    c = plan(W.mha_bf16(batch=1, heads=1, seq=48, head_dim=32).graph)
+    assert "cuda-core" in c.plan
+
+
+def test_plan_only_cannot_execute():
+    c = plan(W.mlp_f32().graph)
+    with pytest.raises(B.GcError) as e:
+        B.gc_execute(c._comp, 0, [16] * 7, [16])
+    assert e.value.status == B.GC_ERR_STATE
+
+
+def test_partition_create_rejects_bad_graphs():
+    g = W.mlp_f32(batch=4, dims=(8, 16)).graph
+    g.ops[0].inputs = (g.ops[0].inputs[0], 999)
+    with pytest.raises(B.GcError) as e:
+        B.gc_partition_create(g)
+    assert e.value.status == B.GC_ERR_INVALID_ARG
+    g = W.mlp_f32(batch=4, dims=(8, 16)).graph
+    g.tensors[g.ops[0].output].dims = (4, 17)
+    with pytest.raises(B.GcError) as e:
+        B.gc_partition_create(g)
+    assert e.value.status == B.GC_ERR_SHAPE
+    g = W.mlp_f32(batch=4, dims=(8, 16)).graph
+    g.ops.reverse()                                  # not topological
+    with pytest.raises(B.GcError) as e:
+        B.gc_partition_create(g)
+    assert e.value.status == B.GC_ERR_INVALID_ARG
+    g = W.mlp_f32(batch=4, dims=(8, 16)).graph
+    g.outputs = [g.inputs[0] + 1000]
+    with pytest.raises(B.GcError):
+        B.gc_partition_create(g)
+
+
+def test_compile_rejects_unsupported_patterns():
+    # softmax alone
+    g = Graph()
+    x = g.input("f32", (4, 8))
+    g.mark_output(g.op("softmax", (x,), g.tensor("f32", (4, 8))))
+    with pytest.raises(B.GcError) as e:
+        plan(g)
+    assert e.value.status == B.GC_ERR_UNSUPPORTED
+    # weights that are not constant
+    w = W.mlp_f32(batch=4, dims=(8, 16))
+    w.graph.tensors[w.graph.inputs[1]].is_constant = False
+    with pytest.raises(B.GcError) as e:
+        plan(w.graph)
+    assert e.value.status == B.GC_ERR_UNSUPPORTED
+    # an intermediate that is also an output
+    w = W.mlp_f32(batch=4, dims=(8, 16, 16))
+    w.graph.outputs.append(w.graph.ops[2].output)
+    with pytest.raises(B.GcError) as e:
+        plan(w.graph)
+    assert e.value.status == B.GC_ERR_UNSUPPORTED
+    # no such device
+    p = B.gc_partition_create(W.mlp_f32().graph)
+    with pytest.raises(B.GcError):
+        B.gc_compile(p, 99)
+    B.gc_partition_destroy(p)
