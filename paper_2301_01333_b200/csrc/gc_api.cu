@@ -196,8 +196,9 @@ struct LayerPlan {
   size_t wt_off = 0;
   int Kp = 0;
   // cached tensor maps
-  CUtensorMap tmA, tmB;
+  CUtensorMap tmA, tmB, tmD;
   const void* tmA_ptr = nullptr;
+  const void* tmD_ptr = nullptr;
   bool tmB_valid = false;
 };
 
@@ -256,7 +257,8 @@ static gc_status_t make_tmap(CUtensorMap* m, const void* ptr, int dtype, uint64_
                              uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_rows, int swizzle_bytes) {
   EncodeTiledFn enc = get_encode();
   if (!enc) return fail(GC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
-  CUtensorMapDataType dt = dtype == GC_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+  CUtensorMapDataType dt = dtype == GC_F32    ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                           : dtype == GC_S32  ? CU_TENSOR_MAP_DATA_TYPE_INT32
                            : dtype == GC_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
                                               : CU_TENSOR_MAP_DATA_TYPE_UINT8;
   cuuint64_t gdim[2] = {inner, rows};
@@ -465,17 +467,17 @@ static void choose_tile(LayerPlan& L, int num_sms) {
   const int k_elems = 128 / esz;
   L.m_tiles = (L.M + 127) / 128;
   L.nkb = (L.K + k_elems - 1) / k_elems;
-  const int cands[5] = {256, 128, 64, 32, 16};
+  const int cands[4] = {256, 128, 64, 32};
   int pick = 0;
   for (int bn : cands) {
-    if (bn > 16 && bn > L.N) continue;
+    if (bn > 32 && bn > L.N) continue;
     const int tiles = L.m_tiles * ((L.N + bn - 1) / bn);
     if (tiles >= num_sms) {
       pick = bn;
       break;
     }
   }
-  if (!pick) pick = L.N >= 32 ? 32 : 16;
+  if (!pick) pick = 32;
   L.block_n = pick;
   L.n_tiles = (L.N + pick - 1) / pick;
   const int tiles = L.m_tiles * L.n_tiles;
@@ -657,6 +659,7 @@ extern "C" gc_status_t gc_set_workspace(gc_compiled_t* c, void* ws, size_t bytes
   c->status_cleared = false;
   for (auto& L : c->layers) {
     L.tmA_ptr = nullptr;
+    L.tmD_ptr = nullptr;
     L.tmB_valid = false;
   }
   return GC_OK;
@@ -738,8 +741,16 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
       g.out_pitch = L.out_pitch;
       g.epi = e;
       g.status = status;
+      const int box_cols = gemm_tc_store_box_cols(L.block_n, L.out_elem);
+      if (box_cols && L.tmD_ptr != O) {
+        gc_status_t s = make_tmap(&L.tmD, O, L.epi.out_dtype, L.N, L.M, static_cast<uint64_t>(L.out_pitch) * L.out_elem,
+                                  box_cols, 32, 128);
+        if (s != GC_OK) return s;
+        L.tmD_ptr = O;
+      }
       const bool pdl = !c.opt.no_chain_fusion && l > 0 && !L.need_pack;
-      CUDA_TRY(launch_gemm_tc(L.kind, L.block_n, L.a_dtype == GC_S8, L.tmA, L.tmB, g, L.grid, pdl, st));
+      CUDA_TRY(launch_gemm_tc(L.kind, L.block_n, L.a_dtype == GC_S8, L.tmA, L.tmB, box_cols ? L.tmD : L.tmA, g, L.grid,
+                              pdl, st));
     } else {
       GemmSimtParams g = {};
       g.A = A;

@@ -32,6 +32,7 @@ struct Epilogue {
 struct GemmTcParams {
   int M, N, K;
   int num_k_blocks, m_tiles, n_tiles;
+  uint32_t idesc;      // tcgen05 instruction descriptor (filled by the launcher)
   void* out;
   int64_t out_pitch;   // elements
   Epilogue epi;
@@ -85,8 +86,11 @@ cudaError_t launch_sdpa_simt(const SdpaParams& p, cudaStream_t s);
 // kind: 0 = i8 (u8/s8 x s8 -> s32), 1 = bf16, 2 = tf32.  a_signed only matters for kind 0.
 bool gemm_tc_supported_block_n(int block_n);
 size_t gemm_tc_smem_bytes(int block_n);
+// Columns per TMA-store box for this tile width and output element size, or 0 when the kernel stores
+// with plain vector stores (tile rows shorter than 128 bytes) and tmD is ignored.
+int gemm_tc_store_box_cols(int block_n, int out_elem_bytes);
 cudaError_t launch_gemm_tc(int kind, int block_n, int a_signed, const CUtensorMap& tmA, const CUtensorMap& tmB,
-                           const GemmTcParams& p, int grid, bool pdl, cudaStream_t s);
+                           const CUtensorMap& tmD, const GemmTcParams& p, int grid, bool pdl, cudaStream_t s);
 
 size_t sdpa_tc_smem_bytes(int S, int is_int8);
 cudaError_t launch_sdpa_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const SdpaParams& p,

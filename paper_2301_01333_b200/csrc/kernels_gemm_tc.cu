@@ -2,14 +2,20 @@
 // requantize  ->  store.  One kernel serves every layer of the MLP chains (Sections III-V: the Tunable op
 // with its post-ops fused at the innermost anchor).
 //
-// Structure (one persistent CTA per SM, 192 threads):
+// Structure (one persistent CTA per SM, 320 threads):
 //   warp 0     TMA producer: 128-byte-swizzled [128 x 128B] A tiles and [BLOCK_N x 128B] Wt tiles into a
 //              STAGES-deep shared-memory ring, completion on "full" mbarriers
 //   warp 1     MMA issuer: one thread issues tcgen05.mma (kind::i8 / f16 / tf32) into one of two TMEM
 //              accumulators; tcgen05.commit releases ring slots ("empty") and publishes accumulators
-//   warps 2-5  epilogue: tcgen05.ld the accumulator (lane = row), apply the post-ops, store; then hand
-//              the accumulator back, so the epilogue of tile i overlaps the main loop of tile i+1
-// K tails and M/N tails are zero-filled by TMA; every mbarrier wait is bounded (ptx.cuh).
+//   warps 2-9  epilogue: two warps per TMEM lane quarter, each taking alternate 128-byte-wide column
+//              groups: tcgen05.ld (lane = row), post-ops in registers, swizzled staging in shared memory,
+//              one TMA store per [32 rows x 128 B] box; then the accumulator is handed back, so the
+//              epilogue of tile i overlaps the main loop of tile i+1
+// K tails and M/N tails are zero-filled by TMA loads and clipped by TMA stores; every mbarrier wait is
+// bounded (ptx.cuh).  Narrow tiles whose rows are shorter than 128 bytes are stored with plain vector
+// stores instead of TMA.
+#include <cuda_bf16.h>
+
 #include "epilogue.cuh"
 #include "gc_internal.h"
 #include "ptx.cuh"
@@ -18,36 +24,131 @@ namespace gc {
 
 constexpr int GEMM_BLOCK_M = 128;
 constexpr int GEMM_TILE_K_BYTES = 128;   // one swizzle span: 128 i8 / 64 bf16 / 32 tf32 elements
-constexpr int GEMM_THREADS = 192;
+constexpr int GEMM_EPI_WARPS = 8;
+constexpr int GEMM_THREADS = 64 + 32 * GEMM_EPI_WARPS;
+constexpr int GEMM_STAGING_BYTES = GEMM_EPI_WARPS * 4096;
 
-__host__ __device__ constexpr int gemm_stages(int block_n) {
-  return block_n >= 256 ? 4 : (block_n >= 128 ? 6 : 8);
-}
+enum OutKind { OUT_F32 = 0, OUT_BF16 = 1, OUT_Q8 = 2, OUT_RAW32 = 3 };
+__host__ __device__ constexpr int out_bytes(int ok) { return ok == OUT_BF16 ? 2 : (ok == OUT_Q8 ? 1 : 4); }
+
 __host__ __device__ constexpr int gemm_stage_bytes(int block_n) {
   return GEMM_BLOCK_M * GEMM_TILE_K_BYTES + block_n * GEMM_TILE_K_BYTES;
 }
-
-bool gemm_tc_supported_block_n(int bn) { return bn == 16 || bn == 32 || bn == 64 || bn == 128 || bn == 256; }
-size_t gemm_tc_smem_bytes(int bn) {
-  return static_cast<size_t>(gemm_stages(bn)) * gemm_stage_bytes(bn) + 1024 /*alignment slack*/ + 256 /*barriers*/;
+__host__ __device__ constexpr int gemm_stages(int block_n) {
+  return block_n >= 256 ? 4 : (block_n >= 128 ? 5 : 8);
 }
 
-template <int KIND, int BLOCK_N, bool A_SIGNED>
+bool gemm_tc_supported_block_n(int bn) { return bn == 32 || bn == 64 || bn == 128 || bn == 256; }
+size_t gemm_tc_smem_bytes(int bn) {
+  return static_cast<size_t>(gemm_stages(bn)) * gemm_stage_bytes(bn) + GEMM_STAGING_BYTES + 1024 /*alignment slack*/ +
+         256 /*barriers*/;
+}
+int gemm_tc_store_box_cols(int block_n, int out_elem_bytes) {
+  return (block_n * out_elem_bytes) % 128 == 0 ? 128 / out_elem_bytes : 0;
+}
+
+// 32 accumulator words of one row -> 32 post-op values (fp32), columns n0 .. n0+31
+template <int KIND, int ACT>
+__device__ __forceinline__ void epi_values32(const uint32_t (&raw)[32], float (&t)[32], int n0, int n_end,
+                                             const Epilogue& e) {
+  float b[32];
+  if (e.bias) {
+    const float4* bp = reinterpret_cast<const float4*>(e.bias + n0);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      // columns at or beyond n_end belong to a clipped tile tail: never read the bias there
+      const float4 v = n0 + 4 * i < n_end ? __ldg(bp + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+      b[4 * i] = v.x; b[4 * i + 1] = v.y; b[4 * i + 2] = v.z; b[4 * i + 3] = v.w;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) b[i] = 0.f;
+  }
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    float x;
+    if constexpr (KIND == KIND_I8) {
+      x = __fmul_rn(__int2float_rn(static_cast<int>(raw[i])), e.dq);
+      x = e.bias ? __fadd_rn(x, b[i]) : x;                      // separately rounded on the integer path
+    } else {
+      x = __uint_as_float(raw[i]) + b[i];
+    }
+    if constexpr (ACT == ACT_RELU) {
+      x = fmaxf(x, 0.f);
+    } else if constexpr (ACT == ACT_GELU_TANH) {
+      // 0.5 x (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3))) = h + h tanh(x (c0 + c1 x^2)), h = x/2
+      const float x2 = x * x;
+      const float u = x * fmaf(x2, 0.7978845608028654f * 0.044715f, 0.7978845608028654f);
+      const float h = 0.5f * x;
+      x = fmaf(h, tanh_approx(u), h);
+    } else if constexpr (ACT == ACT_SIGMOID) {
+      x = 1.0f / (1.0f + expf(-x));
+    }
+    t[i] = x;
+  }
+}
+
+// post-op values -> packed output words (NW = 32 * out_bytes / 4)
+template <int OUT>
+__device__ __forceinline__ void epi_pack32(const float (&t)[32], uint32_t* w, const Epilogue& e) {
+  if constexpr (OUT == OUT_F32) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) w[i] = __float_as_uint(t[i]);
+  } else if constexpr (OUT == OUT_BF16) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      __nv_bfloat162 h = __floats2bfloat162_rn(t[2 * i], t[2 * i + 1]);
+      w[i] = *reinterpret_cast<uint32_t*>(&h);
+    }
+  } else {
+    const int lo = e.out_dtype == GC_U8 ? 0 : -128, hi = e.out_dtype == GC_U8 ? 255 : 127;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      uint32_t word = 0;
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        word |= static_cast<uint32_t>(quantize_value(t[4 * i + k], e.inv, e.zp, lo, hi) & 0xFF) << (8 * k);
+      w[i] = word;
+    }
+  }
+}
+
+template <int KIND, int OUT>
+__device__ __forceinline__ void epi_chunk32(const uint32_t (&raw)[32], uint32_t* w, int n0, int n_end,
+                                            const Epilogue& e) {
+  if constexpr (OUT == OUT_RAW32) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) w[i] = raw[i];
+  } else {
+    float t[32];
+    switch (e.act) {
+      case ACT_RELU: epi_values32<KIND, ACT_RELU>(raw, t, n0, n_end, e); break;
+      case ACT_GELU_TANH: epi_values32<KIND, ACT_GELU_TANH>(raw, t, n0, n_end, e); break;
+      case ACT_SIGMOID: epi_values32<KIND, ACT_SIGMOID>(raw, t, n0, n_end, e); break;
+      default: epi_values32<KIND, ACT_NONE>(raw, t, n0, n_end, e); break;
+    }
+    epi_pack32<OUT>(t, w, e);
+  }
+}
+
+template <int KIND, int BLOCK_N, int OUT>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmTcParams p) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmD, const GemmTcParams p) {
   constexpr int STAGES = gemm_stages(BLOCK_N);
   constexpr int STAGE_BYTES = gemm_stage_bytes(BLOCK_N);
   constexpr int A_BYTES = GEMM_BLOCK_M * GEMM_TILE_K_BYTES;
   constexpr int TMEM_COLS = 2 * BLOCK_N < 32 ? 32 : 2 * BLOCK_N;
   constexpr int K_ELEMS = KIND == KIND_I8 ? 128 : (KIND == KIND_BF16 ? 64 : 32);   // per 128-byte span
-  constexpr uint32_t IDESC =
-      KIND == KIND_I8   ? make_idesc(ACC_S32, A_SIGNED ? FMT_S8 : FMT_U8, FMT_S8, GEMM_BLOCK_M, BLOCK_N)
-      : KIND == KIND_BF16 ? make_idesc(ACC_F32, FMT_BF16, FMT_BF16, GEMM_BLOCK_M, BLOCK_N)
-                          : make_idesc(ACC_F32, FMT_TF32, FMT_TF32, GEMM_BLOCK_M, BLOCK_N);
+  constexpr int OUT_BYTES = out_bytes(OUT);
+  constexpr bool TMA_STORE = (BLOCK_N * OUT_BYTES) % 128 == 0;
+  constexpr int BOX_COLS = 128 / OUT_BYTES;                     // columns per 128-byte staging row
+  constexpr int NUM_BOXES = TMA_STORE ? BLOCK_N / BOX_COLS : 0;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+  uint8_t* staging = smem + STAGES * STAGE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(staging + GEMM_STAGING_BYTES);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   const uint32_t smem_base = smem_u32(smem);
   const uint32_t bar_full = smem_u32(bars);                       // [STAGES]
@@ -64,11 +165,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_tfull + 8 * a, 1);
-      mbar_init(bar_tempty + 8 * a, 4);
+      mbar_init(bar_tempty + 8 * a, GEMM_EPI_WARPS);
     }
     fence_mbar_init();
     tma_prefetch_desc(&tmA);
     tma_prefetch_desc(&tmB);
+    if (TMA_STORE) tma_prefetch_desc(&tmD);
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
@@ -137,7 +239,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const uint64_t b_desc = make_smem_desc(sB, 16, 1024, SWZ_128B);
 #pragma unroll
           for (int k = 0; k < 4; ++k)
-            umma_ss<KIND>(d_tmem, a_desc + 2 * k, b_desc + 2 * k, IDESC, (kb | k) != 0 ? 1u : 0u);
+            umma_ss<KIND>(d_tmem, a_desc + 2 * k, b_desc + 2 * k, p.idesc, (kb | k) != 0 ? 1u : 0u);
           umma_commit(bar_empty + 8 * stage);
           if (++stage == STAGES) {
             stage = 0;
@@ -152,11 +254,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   } else {
     // ------------------------------------------------------------------ epilogue warps
-    const int q = warp & 3;   // TMEM lane quarter this warp may access
+    const int ew = warp - 2;          // 0..7
+    const int q = warp & 3;           // TMEM lane quarter this warp may access
+    const int half = ew >> 2;         // which alternate column groups this warp takes
     int acc = 0;
     uint32_t acc_phase = 0;
-    const int out_elem = (p.epi.acc_is_int && !p.epi.has_dq) ? 4
-                         : (p.epi.out_dtype == GC_F32 ? 4 : (p.epi.out_dtype == GC_BF16 ? 2 : 1));
+    uint8_t* my_stage = staging + ew * 4096;
+    const uint32_t my_stage_u32 = smem_u32(my_stage);
+    const uint32_t row_off = (lane >> 3) * 1024 + (lane & 7) * 128;
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
       const int m_blk = tile / p.n_tiles, n_blk = tile % p.n_tiles;
       if (!mbar_wait(bar_tfull + 8 * acc, acc_phase)) {
@@ -165,12 +270,38 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         break;
       }
       tc_fence_after();
-      const int row = m_blk * GEMM_BLOCK_M + q * 32 + lane;
-      char* dst_row = static_cast<char*>(p.out) + static_cast<int64_t>(row) * p.out_pitch * out_elem;
       const uint32_t t_row = tmem_base + acc * BLOCK_N + (static_cast<uint32_t>(q * 32) << 16);
-      if constexpr (BLOCK_N >= 32) {
+      if constexpr (TMA_STORE) {
+        for (int box = half; box < NUM_BOXES; box += 2) {
+          // the previous store out of this warp's staging buffer must have read it completely
+          if (lane == 0) tma_store_wait_read<0>();
+          __syncwarp();
 #pragma unroll 1
-        for (int c = 0; c < BLOCK_N / 32; ++c) {
+          for (int sub = 0; sub < BOX_COLS / 32; ++sub) {
+            uint32_t r[32];
+            tmem_ld32(t_row + box * BOX_COLS + sub * 32, r);
+            tmem_wait_ld();
+            constexpr int NW = 32 * OUT_BYTES / 4;              // packed words for 32 columns
+            uint32_t w[NW];
+            epi_chunk32<KIND, OUT>(r, w, n_blk * BLOCK_N + box * BOX_COLS + sub * 32, p.N, p.epi);
+            const int c0 = sub * (NW / 4);                      // first 16-byte chunk of this sub-block
+#pragma unroll
+            for (int i = 0; i < NW / 4; ++i)
+              *reinterpret_cast<uint4*>(my_stage + row_off + (((c0 + i) ^ (lane & 7)) * 16)) =
+                  make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+          }
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_2d(&tmD, n_blk * BLOCK_N + box * BOX_COLS, m_blk * GEMM_BLOCK_M + q * 32, my_stage_u32);
+            tma_store_commit();
+          }
+        }
+      } else {
+        // rows shorter than 128 bytes: 16-column groups stored straight from registers
+        const int row = m_blk * GEMM_BLOCK_M + q * 32 + lane;
+        char* dst_row = static_cast<char*>(p.out) + static_cast<int64_t>(row) * p.out_pitch * OUT_BYTES;
+        for (int c = half; c < BLOCK_N / 32; c += 2) {
           uint32_t r[32];
           tmem_ld32(t_row + c * 32, r);
           tmem_wait_ld();
@@ -180,12 +311,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (n0 + 16 < p.N) epi_store16(r + 16, dst_row, n0 + 16, p.epi);
           }
         }
-      } else {
-        uint32_t r[16];
-        tmem_ld16(t_row, r);
-        tmem_wait_ld();
-        const int n0 = n_blk * BLOCK_N;
-        if (row < p.M && n0 < p.N) epi_store16(r, dst_row, n0, p.epi);
       }
       tc_fence_before();
       __syncwarp();
@@ -193,6 +318,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1;
     }
+    if (TMA_STORE && lane == 0) tma_store_wait_all<0>();
   }
 
   // ---------------------------------------------------------------------- teardown
@@ -210,13 +336,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
 }
 
-template <int KIND, int BLOCK_N, bool A_SIGNED>
-static cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmTcParams& p, int grid, bool pdl,
-                              cudaStream_t s) {
+template <int KIND, int BLOCK_N, int OUT>
+static cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmD,
+                              const GemmTcParams& p, int grid, bool pdl, cudaStream_t s) {
   const size_t smem = gemm_tc_smem_bytes(BLOCK_N);
-  auto kern = gemm_tc_kernel<KIND, BLOCK_N, A_SIGNED>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-  if (e != cudaSuccess) return e;
+  auto kern = gemm_tc_kernel<KIND, BLOCK_N, OUT>;
+  static bool attr_set[64] = {};     // per instantiation and device
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (!attr_set[dev & 63]) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    attr_set[dev & 63] = true;
+  }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
   cfg.blockDim = dim3(GEMM_THREADS);
@@ -227,29 +359,55 @@ static cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, co
   attr[0].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, p);
+  return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmD, p);
 }
 
-template <int KIND, bool A_SIGNED>
-static cudaError_t launch_bn(int bn, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmTcParams& p, int grid,
-                             bool pdl, cudaStream_t s) {
+template <int KIND, int OUT>
+static cudaError_t launch_bn(int bn, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmD,
+                             const GemmTcParams& p, int grid, bool pdl, cudaStream_t s) {
   switch (bn) {
-    case 16: return launch_one<KIND, 16, A_SIGNED>(tmA, tmB, p, grid, pdl, s);
-    case 32: return launch_one<KIND, 32, A_SIGNED>(tmA, tmB, p, grid, pdl, s);
-    case 64: return launch_one<KIND, 64, A_SIGNED>(tmA, tmB, p, grid, pdl, s);
-    case 128: return launch_one<KIND, 128, A_SIGNED>(tmA, tmB, p, grid, pdl, s);
-    case 256: return launch_one<KIND, 256, A_SIGNED>(tmA, tmB, p, grid, pdl, s);
+    case 32: return launch_one<KIND, 32, OUT>(tmA, tmB, tmD, p, grid, pdl, s);
+    case 64: return launch_one<KIND, 64, OUT>(tmA, tmB, tmD, p, grid, pdl, s);
+    case 128: return launch_one<KIND, 128, OUT>(tmA, tmB, tmD, p, grid, pdl, s);
+    case 256: return launch_one<KIND, 256, OUT>(tmA, tmB, tmD, p, grid, pdl, s);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+template <int KIND>
+static cudaError_t launch_out(int out, int bn, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmD,
+                              const GemmTcParams& p, int grid, bool pdl, cudaStream_t s) {
+  switch (out) {
+    case OUT_F32: return launch_bn<KIND, OUT_F32>(bn, tmA, tmB, tmD, p, grid, pdl, s);
+    case OUT_BF16: return launch_bn<KIND, OUT_BF16>(bn, tmA, tmB, tmD, p, grid, pdl, s);
+    case OUT_Q8: return launch_bn<KIND, OUT_Q8>(bn, tmA, tmB, tmD, p, grid, pdl, s);
+    case OUT_RAW32:
+      if constexpr (KIND == KIND_I8) return launch_bn<KIND, OUT_RAW32>(bn, tmA, tmB, tmD, p, grid, pdl, s);
+      return launch_bn<KIND, OUT_F32>(bn, tmA, tmB, tmD, p, grid, pdl, s);
     default: return cudaErrorInvalidValue;
   }
 }
 
 cudaError_t launch_gemm_tc(int kind, int block_n, int a_signed, const CUtensorMap& tmA, const CUtensorMap& tmB,
-                           const GemmTcParams& p, int grid, bool pdl, cudaStream_t s) {
-  if (kind == KIND_I8)
-    return a_signed ? launch_bn<KIND_I8, true>(block_n, tmA, tmB, p, grid, pdl, s)
-                    : launch_bn<KIND_I8, false>(block_n, tmA, tmB, p, grid, pdl, s);
-  if (kind == KIND_BF16) return launch_bn<KIND_BF16, false>(block_n, tmA, tmB, p, grid, pdl, s);
-  if (kind == KIND_TF32) return launch_bn<KIND_TF32, false>(block_n, tmA, tmB, p, grid, pdl, s);
+                           const CUtensorMap& tmD, const GemmTcParams& p_in, int grid, bool pdl, cudaStream_t s) {
+  GemmTcParams p = p_in;
+  const Epilogue& e = p.epi;
+  const int out = (e.acc_is_int && !e.has_dq) ? OUT_RAW32
+                  : e.out_dtype == GC_F32    ? OUT_F32
+                  : e.out_dtype == GC_BF16   ? OUT_BF16
+                                             : OUT_Q8;
+  if (kind == KIND_I8) {
+    p.idesc = make_idesc(ACC_S32, a_signed ? FMT_S8 : FMT_U8, FMT_S8, GEMM_BLOCK_M, block_n);
+    return launch_out<KIND_I8>(out, block_n, tmA, tmB, tmD, p, grid, pdl, s);
+  }
+  if (kind == KIND_BF16) {
+    p.idesc = make_idesc(ACC_F32, FMT_BF16, FMT_BF16, GEMM_BLOCK_M, block_n);
+    return launch_out<KIND_BF16>(out, block_n, tmA, tmB, tmD, p, grid, pdl, s);
+  }
+  if (kind == KIND_TF32) {
+    p.idesc = make_idesc(ACC_F32, FMT_TF32, FMT_TF32, GEMM_BLOCK_M, block_n);
+    return launch_out<KIND_TF32>(out, block_n, tmA, tmB, tmD, p, grid, pdl, s);
+  }
   return cudaErrorInvalidValue;
 }
 
