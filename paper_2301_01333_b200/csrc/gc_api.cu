@@ -560,8 +560,9 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
     bool tc = !c->opt.force_generic && s.D == 64 && s.S % 128 == 0 && s.S <= 384 &&
               sdpa_tc_smem_bytes(s.S, s.is_int8) <= static_cast<size_t>(prop.sharedMemPerBlockOptin);
     if (s.is_int8)
-      tc = tc && s.zp_p == 0 && ((s.q_signed && s.zp_q == 0) || (!s.q_signed && s.zp_q == 128)) &&
-           ((s.k_signed && s.zp_k == 0) || (!s.k_signed && s.zp_k == 128));
+      // Q must be exactly centred (s8 / zero point 0, or u8 / zero point 128); a zero point on K only
+      // shifts every score of a row by the same amount, which softmax cancels
+      tc = tc && s.zp_p == 0 && ((s.q_signed && s.zp_q == 0) || (!s.q_signed && s.zp_q == 128));
     if (!tc && s.S > 8192) return bail(fail(GC_ERR_UNSUPPORTED, "attention: sequence length %d not supported", s.S));
     c->sdpa.use_tc = tc;
     c->launches = 1;
@@ -806,7 +807,7 @@ static gc_status_t run_sdpa(gc_compiled& c, cudaStream_t st, const void* const* 
     if (r != GC_OK) return r;
     s.v_ptr = prm.V;
   }
-  CUDA_TRY(launch_sdpa_tc(s.tmQ, s.tmK, s.tmV, prm, st));
+  CUDA_TRY(launch_sdpa_tc(s.tmQ, s.tmK, s.tmV, prm, c.num_sms, st));
   return GC_OK;
 }
 

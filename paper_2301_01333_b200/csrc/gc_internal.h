@@ -94,6 +94,6 @@ cudaError_t launch_gemm_tc(int kind, int block_n, int a_signed, const CUtensorMa
 
 size_t sdpa_tc_smem_bytes(int S, int is_int8);
 cudaError_t launch_sdpa_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const SdpaParams& p,
-                           cudaStream_t s);
+                           int num_sms, cudaStream_t s);
 
 }  // namespace gc
