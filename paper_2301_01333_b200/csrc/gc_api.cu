@@ -206,8 +206,8 @@ struct SdpaPlan {
   SdpaParams prm = {};
   int q_input = -1, k_input = -1, v_input = -1, mask_input = -1, out_pos = 0;
   bool use_tc = false;
-  CUtensorMap tmQ, tmK, tmV;
-  const void *q_ptr = nullptr, *k_ptr = nullptr, *v_ptr = nullptr;
+  CUtensorMap tmQ, tmK, tmV, tmO;
+  const void *q_ptr = nullptr, *k_ptr = nullptr, *v_ptr = nullptr, *o_ptr = nullptr;
 };
 
 struct gc_compiled {
@@ -265,8 +265,9 @@ static gc_status_t make_tmap(CUtensorMap* m, const void* ptr, int dtype, uint64_
   cuuint64_t gstr[1] = {pitch_bytes};
   cuuint32_t box[2] = {box_inner, box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUtensorMapSwizzle sw = swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+  CUtensorMapSwizzle sw = swizzle_bytes == 128  ? CU_TENSOR_MAP_SWIZZLE_128B
                           : swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                          : swizzle_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B
                                                 : CU_TENSOR_MAP_SWIZZLE_NONE;
   CUresult r = enc(m, dt, 2, const_cast<void*>(ptr), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -807,7 +808,12 @@ static gc_status_t run_sdpa(gc_compiled& c, cudaStream_t st, const void* const* 
     if (r != GC_OK) return r;
     s.v_ptr = prm.V;
   }
-  CUDA_TRY(launch_sdpa_tc(s.tmQ, s.tmK, s.tmV, prm, c.num_sms, st));
+  if (s.o_ptr != prm.O) {
+    gc_status_t r = make_tmap(&s.tmO, prm.O, dt, prm.D, rows, static_cast<uint64_t>(prm.D) * esz, 32, 32, 32 * esz);
+    if (r != GC_OK) return r;
+    s.o_ptr = prm.O;
+  }
+  CUDA_TRY(launch_sdpa_tc(s.tmQ, s.tmK, s.tmV, s.tmO, prm, c.num_sms, st));
   return GC_OK;
 }
 

@@ -5,8 +5,9 @@
 //   warp 0      TMA producer: Q tile, all K rows and all V rows of the unit into one of two shared-memory
 //               slots (128B / 64B swizzle), one unit ahead of the math (no multicast)
 //   warp 1      MMA issuer (one thread): S = Q K^T in 128-key blocks into tensor memory, O = P V in 128-key
-//               blocks as soon as each P block is ready; the next unit's S blocks are issued as soon as the
-//               softmax warps release the corresponding TMEM columns
+//               blocks as soon as each P block is ready.  When two score buffers fit in tensor memory
+//               (S = 128) the next unit's S is issued a whole unit early; otherwise its blocks are issued as
+//               soon as the softmax warps release the corresponding TMEM columns
 //   warps 2-3   per-unit preparation: u8 -> s8 flip of Q (int8 path), mask row scaled by log2(e)
 //   warps 4-11  softmax: two threads per query row (TMEM lane), each owning 64 of every 128 key columns.
 //               Pass A: scale + mask, running row max, exp2 and running row sum (int8: the exponentials
@@ -22,6 +23,10 @@
 // K stays as stored: sum_d q'_d (k_d - z) = sum_d q'_d k_d - z sum_d q'_d differs from the wanted score
 // by a per-row constant, which softmax cancels.  V stays u8 and its zero point is removed from the
 // accumulator with the row sum of P:  sum_j P_j (V_j - z) = sum_j P_j V_j - z sum_j P_j.
+//
+// Integer <-> float conversions in the inner loops use the 1.5 * 2^23 bias trick on the FMA/ALU pipes
+// (exact for |x| < 2^22) because the conversion instructions share the special-function unit with exp2,
+// which is the busiest pipe of this kernel.
 #include <cuda_bf16.h>
 
 #include "epilogue.cuh"
@@ -35,34 +40,44 @@ constexpr int SDPA_BLOCK_Q = 128;
 constexpr int SDPA_THREADS = 384;
 constexpr int SDPA_SOFTMAX_WARPS = 8;
 constexpr float LOG2E = 1.4426950408889634f;
+constexpr float MAGIC_F = 12582912.0f;          // 1.5 * 2^23
+constexpr int MAGIC_I = 0x4B400000;             // its bit pattern
 
 template <bool INT8>
 struct SdpaSmem {
   static constexpr int ESZ = INT8 ? 1 : 2;
   static constexpr int ROW_BYTES = SDPA_D * ESZ;               // 64 (SW64) or 128 (SW128)
+  static constexpr int OUT_STAGING_BYTES = SDPA_SOFTMAX_WARPS * 2048;   // per softmax warp: 32 rows x <= 64 bytes
   __host__ __device__ static constexpr int q_bytes() { return SDPA_BLOCK_Q * ROW_BYTES; }
   __host__ __device__ static constexpr int kv_bytes(int S) { return S * ROW_BYTES; }
   // P: per 128-key block, 128 rows x (128 keys * ESZ) bytes = 16 KB (int8) or 32 KB (bf16)
   __host__ __device__ static constexpr int p_bytes(int S) { return (S / 128) * SDPA_BLOCK_Q * 128 * ESZ; }
   __host__ __device__ static constexpr int slot_bytes(int S) { return q_bytes() + 2 * kv_bytes(S); }
-  __host__ __device__ static constexpr int total(int S, int slots) {
-    return slots * slot_bytes(S) + p_bytes(S) + slots * S * 4 /*mask*/ + 4 * 128 * 4 /*row statistics*/ + 256;
+  __host__ __device__ static constexpr int total(int S, int slots, int nsb, int stage_out) {
+    return slots * slot_bytes(S) + nsb * p_bytes(S) + (stage_out ? OUT_STAGING_BYTES : 0) + slots * S * 4 /*mask*/ +
+           12 * 128 * 4 /*row statistics*/ + 256;
   }
 };
 
-static int sdpa_slots(int S, int is_int8, size_t smem_limit) {
-  for (int slots = 2; slots >= 1; --slots) {
-    const size_t need = 1024 + (is_int8 ? SdpaSmem<true>::total(S, slots) : SdpaSmem<false>::total(S, slots));
-    if (need <= smem_limit) return slots;
+struct SdpaCfg {
+  int slots;      // shared-memory slots for (Q, K, V): 2 = next unit prefetched
+  int nsb;        // score/output buffers in tensor memory and P buffers in shared memory
+  int stage_out;  // 1: outputs staged in shared memory and written with TMA stores; 0: plain vector stores
+  size_t smem;
+};
+
+static SdpaCfg sdpa_cfg(int S, int is_int8) {
+  const size_t limit = 227 * 1024;
+  const int tries[4][3] = {{2, 2, 1}, {2, 1, 1}, {1, 1, 1}, {1, 1, 0}};
+  for (auto& t : tries) {
+    if (t[1] == 2 && 2 * (S + SDPA_D) > 512) continue;
+    const size_t need = 1024 + (is_int8 ? SdpaSmem<true>::total(S, t[0], t[1], t[2]) : SdpaSmem<false>::total(S, t[0], t[1], t[2]));
+    if (need <= limit) return {t[0], t[1], t[2], need};
   }
-  return 0;
+  return {0, 0, 0, static_cast<size_t>(1) << 30};
 }
 
-size_t sdpa_tc_smem_bytes(int S, int is_int8) {
-  const int slots = sdpa_slots(S, is_int8, 227 * 1024);
-  if (!slots) return static_cast<size_t>(1) << 30;
-  return 1024 + (is_int8 ? SdpaSmem<true>::total(S, slots) : SdpaSmem<false>::total(S, slots));
-}
+size_t sdpa_tc_smem_bytes(int S, int is_int8) { return sdpa_cfg(S, is_int8).smem; }
 
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -70,10 +85,25 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+// exact (float)a for |a| < 2^22 without a conversion instruction
+__device__ __forceinline__ float int_to_float_magic(int a) { return __int_as_float(a + MAGIC_I) - MAGIC_F; }
+// exact (float)a for |a| < 2^24: high and low parts converted separately, recombined with one exact FMA
+__device__ __forceinline__ float int_to_float_magic24(int a) {
+  const float hi = int_to_float_magic(a >> 11), lo = int_to_float_magic(a & 0x7FF);
+  return fmaf(hi, 2048.0f, lo);
+}
+// saturate(rne(u) + zp) with the rounding done by the bias trick
+__device__ __forceinline__ int quantize_magic(float u, int zp, int lo, int hi) {
+  u = fminf(fmaxf(u, -1024.0f), 1024.0f);
+  const int r = __float_as_int(u + MAGIC_F) - MAGIC_I;
+  return min(max(r + zp, lo), hi);
+}
+
 template <bool INT8>
 __global__ void __launch_bounds__(SDPA_THREADS, 1)
 sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-               const __grid_constant__ CUtensorMap tmV, const SdpaParams p, const int slots) {
+               const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO, const SdpaParams p,
+               const int slots, const int nsb, const int stage_out) {
   using L = SdpaSmem<INT8>;
   constexpr int ROW_BYTES = L::ROW_BYTES;
   constexpr uint32_t SWZ = INT8 ? SWZ_64B : SWZ_128B;
@@ -83,19 +113,20 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 
   const int S = p.S;
   const int NB = S / 128;                                       // key blocks
-  const int O_COL = S;                                          // TMEM column of the output accumulator
+  const int BUF_COLS = S + SDPA_D;                              // TMEM columns per (S, O) buffer
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sSlots = smem;
-  uint8_t* sP = sSlots + slots * L::slot_bytes(S);
-  float* sMask = reinterpret_cast<float*>(sP + L::p_bytes(S));  // [slots][S]
-  float* sStat = sMask + slots * S;                             // [4][128]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sStat + 4 * 128);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
+  uint8_t* sPall = sSlots + slots * L::slot_bytes(S);
+  uint8_t* sOut = sPall + nsb * L::p_bytes(S);                            // output staging, 2 KB per softmax warp
+  float* sMask = reinterpret_cast<float*>(sOut + (stage_out ? L::OUT_STAGING_BYTES : 0));   // [slots][S]
+  float* sStat = sMask + slots * S;                                       // [3 kinds][2 parities][2 halves][128]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sStat + 12 * 128);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 24);
   const uint32_t b0 = smem_u32(bars);
   const uint32_t bar_kv_full = b0, bar_kv_empty = b0 + 16, bar_kv_ready = b0 + 32;   // [2] each
   const uint32_t bar_s_full = b0 + 48, bar_s_free = b0 + 72, bar_p_full = b0 + 96;   // [3] each
-  const uint32_t bar_o_full = b0 + 120, bar_o_free = b0 + 128, bar_xchg = b0 + 136;
+  const uint32_t bar_o_full = b0 + 120, bar_o_free = b0 + 136, bar_xchg = b0 + 152;  // [2], [2], [1]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int q_tiles = S / SDPA_BLOCK_Q;
@@ -106,19 +137,20 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       mbar_init(bar_kv_full + 8 * i, 1);
       mbar_init(bar_kv_empty + 8 * i, 1);
       mbar_init(bar_kv_ready + 8 * i, 2);
+      mbar_init(bar_o_full + 8 * i, 1);
+      mbar_init(bar_o_free + 8 * i, SDPA_SOFTMAX_WARPS);
     }
     for (int i = 0; i < 3; ++i) {
       mbar_init(bar_s_full + 8 * i, 1);
       mbar_init(bar_s_free + 8 * i, SDPA_SOFTMAX_WARPS);
       mbar_init(bar_p_full + 8 * i, SDPA_SOFTMAX_WARPS);
     }
-    mbar_init(bar_o_full, 1);
-    mbar_init(bar_o_free, SDPA_SOFTMAX_WARPS);
     mbar_init(bar_xchg, SDPA_SOFTMAX_WARPS);
     fence_mbar_init();
     tma_prefetch_desc(&tmQ);
     tma_prefetch_desc(&tmK);
     tma_prefetch_desc(&tmV);
+    tma_prefetch_desc(&tmO);
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
@@ -133,6 +165,11 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   auto slot_q = [&](int s) { return sSlots + s * L::slot_bytes(S); };
   auto slot_k = [&](int s) { return slot_q(s) + L::q_bytes(); };
   auto slot_v = [&](int s) { return slot_k(s) + L::kv_bytes(S); };
+  // Unit n of this CTA uses score/output buffer buf(n); it is that buffer's cnt(n)-th use.  With one
+  // buffer the per-key-block barriers are indexed by block, with two (one block per unit) by buffer.
+  auto buf_of = [&](int n) { return nsb == 2 ? (n & 1) : 0; };
+  auto cnt_of = [&](int n) { return nsb == 2 ? (n >> 1) : n; };
+  auto bx = [&](int buf, int b) { return nsb == 2 ? buf : b; };
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -164,66 +201,77 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                                    : make_idesc(ACC_F32, FMT_BF16, FMT_BF16, 128, SDPA_D, 0, 1);
       constexpr int K1_STEPS = ROW_BYTES / 32;                  // 32 bytes of the head dimension per MMA
       constexpr int K2_STEPS = 128 / (INT8 ? 32 : 16);          // MMAs per 128-key block of P.V
-      auto mma1 = [&](int s, int b) {                           // S[:, 128b .. 128b+127] = Q K_b^T
+      // S[:, 128b .. 128b+127] = Q K_b^T for unit n1 (waits until the softmax warps have released the columns)
+      auto mma1 = [&](int n1, int b) -> bool {
+        const int s = n1 % slots, buf = buf_of(n1);
+        if (!mbar_wait(bar_s_free + 8 * bx(buf, b), (cnt_of(n1) & 1) ^ 1)) return false;
+        tc_fence_after();
         const uint64_t a_desc = make_smem_desc(smem_u32(slot_q(s)), 16, SBO, SWZ);
         const uint64_t b_desc = make_smem_desc(smem_u32(slot_k(s)) + b * 128 * ROW_BYTES, 16, SBO, SWZ);
 #pragma unroll
         for (int k = 0; k < K1_STEPS; ++k)
-          umma_ss<INT8 ? KIND_I8 : KIND_BF16>(tmem_base + b * 128, a_desc + 2 * k, b_desc + 2 * k, idesc1, k != 0);
-        umma_commit(bar_s_full + 8 * b);
+          umma_ss<INT8 ? KIND_I8 : KIND_BF16>(tmem_base + buf * BUF_COLS + b * 128, a_desc + 2 * k, b_desc + 2 * k, idesc1,
+                                              k != 0);
+        umma_commit(bar_s_full + 8 * bx(buf, b));
+        return true;
       };
-      auto mma2 = [&](int s, int b) {                           // O += P_b V_b
+      auto mma2 = [&](int n0, int b) {                          // O += P_b V_b for unit n0
+        const int s = n0 % slots, buf = buf_of(n0);
+        const uint32_t sP = smem_u32(sPall) + buf * L::p_bytes(S);
 #pragma unroll
         for (int ks = 0; ks < K2_STEPS; ++ks) {
           // A: P block, K-major, 128B swizzle: 4 MMA steps of 32 bytes per 128-byte span, spans 16 KB apart
-          const uint64_t a_desc = make_smem_desc(smem_u32(sP) + b * P_BLOCK_BYTES + (ks >> 2) * (SDPA_BLOCK_Q * 128) +
-                                                     (ks & 3) * 32, 16, 1024, SWZ_128B);
+          const uint64_t a_desc =
+              make_smem_desc(sP + b * P_BLOCK_BYTES + (ks >> 2) * (SDPA_BLOCK_Q * 128) + (ks & 3) * 32, 16, 1024, SWZ_128B);
           // B: V as stored [key][d] = MN-major: one key per ROW_BYTES, 8-key groups SBO apart
           const int key0 = b * 128 + ks * (128 / K2_STEPS);
           const uint64_t b_desc = make_smem_desc(smem_u32(slot_v(s)) + key0 * ROW_BYTES, SBO, SBO, SWZ);
-          umma_ss<INT8 ? KIND_I8 : KIND_BF16>(tmem_base + O_COL, a_desc, b_desc, idesc2, (b | ks) != 0);
+          umma_ss<INT8 ? KIND_I8 : KIND_BF16>(tmem_base + buf * BUF_COLS + S, a_desc, b_desc, idesc2, (b | ks) != 0);
         }
       };
-      const bool interleave = slots == 2;
+      auto wait_inputs = [&](int n1) -> bool {
+        const int s = n1 % slots;
+        const uint32_t par = (n1 / slots) & 1;
+        return mbar_wait(bar_kv_ready + 8 * s, par) && mbar_wait(bar_kv_full + 8 * s, par);
+      };
       int n = 0;
       for (int unit = blockIdx.x; unit < num_units && !failed; unit += gridDim.x, ++n) {
-        const int s = n % slots;
+        const int s = n % slots, buf = buf_of(n);
+        const uint32_t fpar = cnt_of(n) & 1;
         const bool has_next = unit + static_cast<int>(gridDim.x) < num_units;
-        const int sn = (n + 1) % slots;
         if (n == 0) {
-          if (!mbar_wait(bar_kv_ready + 8 * s, 0) || !mbar_wait(bar_kv_full + 8 * s, 0)) { failed = true; break; }
-          tc_fence_after();
-          for (int b = 0; b < NB; ++b) mma1(s, b);
+          if (!wait_inputs(0)) { failed = true; break; }
+          for (int b = 0; b < NB && !failed; ++b) failed = !mma1(0, b);
+          if (failed) break;
+        }
+        bool next_issued = false;
+        if (has_next && nsb == 2) {                             // the other score buffer: a whole unit early
+          if (!wait_inputs(n + 1)) { failed = true; break; }
+          for (int b = 0; b < NB && !failed; ++b) failed = !mma1(n + 1, b);
+          if (failed) break;
+          next_issued = true;
         }
         bool next_ready = false;
         for (int b = 0; b < NB && !failed; ++b) {
-          if (!mbar_wait(bar_p_full + 8 * b, n & 1)) { failed = true; break; }
-          if (b == 0 && !mbar_wait(bar_o_free, (n & 1) ^ 1)) { failed = true; break; }
+          if (!mbar_wait(bar_p_full + 8 * bx(buf, b), fpar)) { failed = true; break; }
+          if (b == 0 && !mbar_wait(bar_o_free + 8 * buf, fpar ^ 1)) { failed = true; break; }
           tc_fence_after();
-          mma2(s, b);
+          mma2(n, b);
           if (b == NB - 1) {
-            umma_commit(bar_o_full);
+            umma_commit(bar_o_full + 8 * buf);
             umma_commit(bar_kv_empty + 8 * s);
           }
-          if (has_next && interleave) {
+          if (has_next && !next_issued && slots == 2) {         // same buffer: block by block as it frees up
             if (!next_ready) {
-              if (!mbar_wait(bar_kv_ready + 8 * sn, ((n + 1) / slots) & 1) ||
-                  !mbar_wait(bar_kv_full + 8 * sn, ((n + 1) / slots) & 1)) { failed = true; break; }
+              if (!wait_inputs(n + 1)) { failed = true; break; }
               next_ready = true;
             }
-            if (!mbar_wait(bar_s_free + 8 * b, n & 1)) { failed = true; break; }
-            tc_fence_after();
-            mma1(sn, b);
+            if (!mma1(n + 1, b)) { failed = true; break; }
           }
         }
-        if (!failed && has_next && !interleave) {
-          if (!mbar_wait(bar_kv_ready + 8 * sn, ((n + 1) / slots) & 1) ||
-              !mbar_wait(bar_kv_full + 8 * sn, ((n + 1) / slots) & 1)) { failed = true; break; }
-          for (int b = 0; b < NB && !failed; ++b) {
-            if (!mbar_wait(bar_s_free + 8 * b, n & 1)) { failed = true; break; }
-            tc_fence_after();
-            mma1(sn, b);
-          }
+        if (!failed && has_next && !next_issued && slots == 1) {
+          if (!wait_inputs(n + 1)) { failed = true; break; }
+          for (int b = 0; b < NB && !failed; ++b) failed = !mma1(n + 1, b);
         }
       }
       if (failed) report(p.status, DEV_TIMEOUT_MMA);
@@ -236,7 +284,7 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       const int s = n % slots;
       const int b = (unit / q_tiles) / p.H;
       float* mk = sMask + s * S;
-      // the mask slot is free once the unit that used it two steps ago has been fully consumed, which
+      // the mask slot is free once the unit that used this slot before has been fully consumed, which
       // the producer's own wait on kv_empty guarantees before kv_full can complete for this unit
       if (!mbar_wait(bar_kv_full + 8 * s, (n / slots) & 1)) {
         report(p.status, DEV_TIMEOUT_OTHER);
@@ -262,14 +310,16 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     const int q = warp & 3;                                     // TMEM lane quarter
     const int h = sw >> 2;                                      // which 64 of every 128 key columns
     const int r = q * 32 + lane;                                // query row within the tile = TMEM lane
-    const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+    const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
     const float c2 = (INT8 ? __fmul_rn(p.dq1, p.scalar) : p.scalar) * LOG2E;
     const uint32_t row_off = (r >> 3) * 1024 + (r & 7) * 128;
     uint32_t xphase = 0;
-    float* stA = sStat + h * 128;                               // my statistics
-    float* stB = sStat + (h ^ 1) * 128;                         // my partner's
-    float* stA2 = sStat + 256 + h * 128;
-    float* stB2 = sStat + 256 + (h ^ 1) * 128;
+    // statistics exchanged between the two threads of a row: [kind][unit parity][half][row]
+    auto stat = [&](int kind, int par, int half) { return sStat + ((kind * 2 + par) * 2 + half) * 128 + r; };
+    // this warp's staging buffer for the output tile: 32 rows x 32 columns, swizzled like its TMA store box
+    constexpr int OUT_ROW_BYTES = 32 * L::ESZ;                  // 32 (int8) or 64 (bf16)
+    uint8_t* my_out = sOut + sw * 2048;
+    const uint32_t out_swz = INT8 ? ((lane >> 2) & 1) : ((lane >> 1) & 3);   // 32B / 64B swizzle of 16-byte chunks
 
     auto xchg_sync = [&]() -> bool {
       __syncwarp();
@@ -278,17 +328,23 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       xphase ^= 1;
       return ok;
     };
-    // epilogue of unit (bh, qt): my 32 of the 64 output columns
-    auto epilogue = [&](int unit, uint32_t par, float stat_total) -> bool {
-      if (!mbar_wait(bar_o_full, par)) return false;
+    // epilogue of unit n0: my 32 of the 64 output columns
+    auto epilogue = [&](int unit, int n0, float stat_total) -> bool {
+      const int buf = buf_of(n0);
+      if (!mbar_wait(bar_o_full + 8 * buf, cnt_of(n0) & 1)) return false;
       tc_fence_after();
       uint32_t v[32];
-      tmem_ld32(t_row + O_COL + h * 32, v);
+      tmem_ld32(t_lane + buf * BUF_COLS + S + h * 32, v);
       tmem_wait_ld();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_o_free);
+      if (lane == 0) {
+        mbar_arrive(bar_o_free + 8 * buf);
+        if (stage_out) tma_store_wait_read<0>();                // the previous store has read the staging buffer
+      }
+      __syncwarp();
       const int bh = unit / q_tiles, qt = unit % q_tiles;
+      // without a staging buffer each thread stores its 32 columns of row `grow` directly
       const int64_t grow = static_cast<int64_t>(bh) * S + qt * SDPA_BLOCK_Q + r;
       if constexpr (INT8) {
         const int lo = p.out_dtype == GC_U8 ? 0 : -128, hi = p.out_dtype == GC_U8 ? 255 : 127;
@@ -300,14 +356,20 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
             const int acc = static_cast<int>(v[4 * i + k]) - corr;
-            const float t = __fmul_rn(__int2float_rn(acc), p.dq2);
-            word |= static_cast<uint32_t>(quantize_value(t, p.inv_o, p.zp_o, lo, hi) & 0xFF) << (8 * k);
+            const float t = __fmul_rn(int_to_float_magic24(acc), p.dq2);
+            word |= static_cast<uint32_t>(quantize_magic(__fmul_rn(t, p.inv_o), p.zp_o, lo, hi) & 0xFF) << (8 * k);
           }
           w[i] = word;
         }
-        uint4* dst = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.O) + grow * SDPA_D + h * 32);
-        dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-        dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+        if (stage_out) {
+          uint8_t* row = my_out + lane * OUT_ROW_BYTES;
+          *reinterpret_cast<uint4*>(row + ((0 ^ out_swz) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(row + ((1 ^ out_swz) * 16)) = make_uint4(w[4], w[5], w[6], w[7]);
+        } else {
+          uint4* dst = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.O) + grow * SDPA_D + h * 32);
+          dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+          dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+        }
       } else {
         const float rl = 1.0f / stat_total;                     // deferred normalisation by the row sum
         uint32_t w[16];
@@ -316,156 +378,215 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(v[2 * i]) * rl, __uint_as_float(v[2 * i + 1]) * rl);
           w[i] = *reinterpret_cast<uint32_t*>(&hh);
         }
-        uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.O) + grow * SDPA_D + h * 32);
+        if (stage_out) {
+          uint8_t* row = my_out + lane * OUT_ROW_BYTES;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) dst[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+          for (int i = 0; i < 4; ++i)
+            *reinterpret_cast<uint4*>(row + ((i ^ out_swz) * 16)) =
+                make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+        } else {
+          uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.O) + grow * SDPA_D + h * 32);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) dst[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+        }
+      }
+      if (stage_out) {
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_2d(&tmO, h * 32, bh * S + qt * SDPA_BLOCK_Q + q * 32, smem_u32(my_out));
+          tma_store_commit();
+        }
       }
       return true;
     };
 
     int n = 0;
     int prev_unit = -1;
-    float prev_stat = 0.f;                                      // row sum of P (int8: integer bits) of the previous unit
+    int prev_psum = 0;                                          // my half of the previous unit's row sum of P
+    float prev_lsum = 0.f;
     for (int unit = blockIdx.x; unit < num_units && !failed; unit += gridDim.x, ++n) {
-      const int s = n % slots;
+      const int s = n % slots, buf = buf_of(n);
       const float* mk = sMask + s * S;
-      const uint32_t par = n & 1;
+      const uint32_t fpar = cnt_of(n) & 1;
+      const int upar = n & 1;
+      const uint32_t t_row = t_lane + buf * BUF_COLS;
+      uint8_t* sP = sPall + buf * L::p_bytes(S);
       if (!mbar_wait(bar_kv_ready + 8 * s, (n / slots) & 1)) { failed = true; break; }
 
-      // ---------------- pass A
+      // ---------------- pass A: row maximum (both paths); int8 also exponentials and row sum
       float m = -INFINITY, l = 0.f;
       float mc[6];                                              // running max after each of my chunks (int8)
 #pragma unroll
       for (int i = 0; i < 6; ++i) mc[i] = 0.f;
-      for (int b = 0; b < NB && !failed; ++b) {
-        if (!mbar_wait(bar_s_full + 8 * b, par)) { failed = true; break; }
+      float x[32];
+      auto pass_a_chunk = [&](const uint32_t (&v)[32], int b, int cc) {
+        const int col = b * 128 + h * 64 + cc * 32;
+        const float4* mk4 = reinterpret_cast<const float4*>(mk + col);
+        float cmax = -INFINITY;
+        if constexpr (INT8) tmem_wait_st();                     // x[] may still be the source of a TMEM store
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const float4 mv = mk4[i];
+          const float mm[4] = {mv.x, mv.y, mv.z, mv.w};
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const float a = INT8 ? int_to_float_magic(static_cast<int>(v[4 * i + k])) : __uint_as_float(v[4 * i + k]);
+            x[4 * i + k] = fmaf(a, c2, mm[k]);
+            cmax = fmaxf(cmax, x[4 * i + k]);
+          }
+        }
+        if constexpr (INT8) {
+          const float m_new = fmaxf(m, cmax);
+          float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+          for (int i = 0; i < 32; i += 2) {
+            x[i] = ex2(x[i] - m_new);
+            x[i + 1] = ex2(x[i + 1] - m_new);
+            sum0 += x[i];
+            sum1 += x[i + 1];
+          }
+          l = l * ex2(m - m_new) + (sum0 + sum1);
+          m = m_new;
+          const int ci = b * 2 + cc;
+          if (ci == 0) mc[0] = m; else if (ci == 1) mc[1] = m; else if (ci == 2) mc[2] = m;
+          else if (ci == 3) mc[3] = m; else if (ci == 4) mc[4] = m; else mc[5] = m;
+          tmem_st32(t_row + col, reinterpret_cast<const uint32_t(&)[32]>(x));
+        } else {
+          m = fmaxf(m, cmax);
+        }
+      };
+      {
+        uint32_t va[32], vb[32];
+        if (!mbar_wait(bar_s_full + 8 * bx(buf, 0), fpar)) { failed = true; break; }
         tc_fence_after();
-#pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {
-          const int col = b * 128 + h * 64 + cc * 32;
-          uint32_t v[32];
-          tmem_ld32(t_row + col, v);
+        tmem_ld32(t_row + h * 64, va);
+        for (int b = 0; b < NB; ++b) {
           tmem_wait_ld();
-          float x[32];
-          float cmax = -INFINITY;
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float a = INT8 ? __int2float_rn(static_cast<int>(v[i])) : __uint_as_float(v[i]);
-            x[i] = fmaf(a, c2, mk[col + i]);
-            cmax = fmaxf(cmax, x[i]);
+          tmem_ld32(t_row + b * 128 + h * 64 + 32, vb);         // next chunk in flight while this one is processed
+          pass_a_chunk(va, b, 0);
+          tmem_wait_ld();
+          if (b + 1 < NB) {
+            if (!mbar_wait(bar_s_full + 8 * bx(buf, b + 1), fpar)) { failed = true; break; }
+            tc_fence_after();
+            tmem_ld32(t_row + (b + 1) * 128 + h * 64, va);
           }
-          if constexpr (INT8) {
-            const float m_new = fmaxf(m, cmax);
-            float sum = 0.f;
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const float e = ex2(x[i] - m_new);
-              sum += e;
-              v[i] = __float_as_uint(e);
-            }
-            l = l * ex2(m - m_new) + sum;
-            m = m_new;
-            if (b * 2 + cc == 0) mc[0] = m; else if (b * 2 + cc == 1) mc[1] = m; else if (b * 2 + cc == 2) mc[2] = m;
-            else if (b * 2 + cc == 3) mc[3] = m; else if (b * 2 + cc == 4) mc[4] = m; else mc[5] = m;
-            tmem_st32(t_row + col, v);
-          } else {
-            m = fmaxf(m, cmax);
-          }
+          pass_a_chunk(vb, b, 1);
         }
       }
       if (failed) break;
       if constexpr (INT8) tmem_wait_st();
-      stA[r] = m;
-      if constexpr (INT8) stA2[r] = l;
+      *stat(0, upar, h) = m;
+      if constexpr (INT8) *stat(1, upar, h) = l;
       if (!xchg_sync()) { failed = true; break; }
-      float scale;                                              // int8: inv_p / row sum
+      float scale = 1.f;                                        // int8: inv_p / row sum
       float M;
       {
-        const float m_p = stB[r];
+        const float m_p = *stat(0, upar, h ^ 1);
         M = fmaxf(m, m_p);
         if constexpr (INT8) {
-          const float l_p = stB2[r];
+          const float l_p = *stat(1, upar, h ^ 1);
           const float Lsum = l * ex2(m - M) + l_p * ex2(m_p - M);
           scale = p.inv_p / Lsum;
-        } else {
-          scale = 1.f;
         }
       }
-      // both threads of every row have read the statistics before they are overwritten below
-      if (!xchg_sync()) { failed = true; break; }
 
-      // ---------------- epilogue of the previous unit (its second MMA has had a whole pass to finish)
+      // ---------------- epilogue of the previous unit (its second MMA has had a whole pass to finish);
+      // the partner's half of that unit's row sum became visible with the exchange above
       if (prev_unit >= 0) {
-        if (!epilogue(prev_unit, (n - 1) & 1, prev_stat)) { failed = true; break; }
+        float total;
+        if constexpr (INT8) total = __int_as_float(prev_psum + __float_as_int(*stat(2, upar ^ 1, h ^ 1)));
+        else total = prev_lsum + *stat(2, upar ^ 1, h ^ 1);
+        if (!epilogue(prev_unit, n - 1, total)) { failed = true; break; }
       }
 
-      // ---------------- pass B
+      // ---------------- pass B: normalise, round, write P
       int psum = 0;
-      float lsum = 0.f;
-      for (int b = 0; b < NB; ++b) {
+      float lsum0 = 0.f, lsum1 = 0.f;
+      auto pass_b_chunk = [&](const uint32_t (&v)[32], int b, int cc) {
+        const int col = b * 128 + h * 64 + cc * 32;
+        if constexpr (INT8) {
+          const int ci = b * 2 + cc;
+          const float mcv = ci == 0 ? mc[0] : ci == 1 ? mc[1] : ci == 2 ? mc[2] : ci == 3 ? mc[3] : ci == 4 ? mc[4] : mc[5];
+          const float f = ex2(mcv - M) * scale;
+          uint32_t w[8];
 #pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {
-          const int col = b * 128 + h * 64 + cc * 32;
-          uint32_t v[32];
-          tmem_ld32(t_row + col, v);
+          for (int i = 0; i < 8; ++i) {
+            // rne(e * f) lands in the low mantissa bits of (e * f + 1.5 * 2^23); codes are within [0, 255]
+            // because p <= 1 and inv_p <= 255
+            const uint32_t y0 = __float_as_uint(fmaf(__uint_as_float(v[4 * i + 0]), f, MAGIC_F));
+            const uint32_t y1 = __float_as_uint(fmaf(__uint_as_float(v[4 * i + 1]), f, MAGIC_F));
+            const uint32_t y2 = __float_as_uint(fmaf(__uint_as_float(v[4 * i + 2]), f, MAGIC_F));
+            const uint32_t y3 = __float_as_uint(fmaf(__uint_as_float(v[4 * i + 3]), f, MAGIC_F));
+            w[i] = __byte_perm(__byte_perm(y0, y1, 0x0040), __byte_perm(y2, y3, 0x0040), 0x5410);
+            psum = static_cast<int>(__dp4a(w[i], 0x01010101u, static_cast<unsigned>(psum)));
+          }
+          uint8_t* blk = sP + b * P_BLOCK_BYTES + row_off;
+          const int c0 = h * 4 + cc * 2;                        // 16-byte chunk index inside the 128-byte row
+          *reinterpret_cast<uint4*>(blk + (((c0 + 0) ^ (r & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(blk + (((c0 + 1) ^ (r & 7)) * 16)) = make_uint4(w[4], w[5], w[6], w[7]);
+        } else {
+          const float4* mk4 = reinterpret_cast<const float4*>(mk + col);
+          uint32_t w[16];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const float4 mv = mk4[i];
+            const float e0 = ex2(fmaf(__uint_as_float(v[4 * i + 0]), c2, mv.x) - M);
+            const float e1 = ex2(fmaf(__uint_as_float(v[4 * i + 1]), c2, mv.y) - M);
+            const float e2 = ex2(fmaf(__uint_as_float(v[4 * i + 2]), c2, mv.z) - M);
+            const float e3 = ex2(fmaf(__uint_as_float(v[4 * i + 3]), c2, mv.w) - M);
+            lsum0 += e0 + e2;
+            lsum1 += e1 + e3;
+            __nv_bfloat162 h0 = __floats2bfloat162_rn(e0, e1), h1 = __floats2bfloat162_rn(e2, e3);
+            w[2 * i] = *reinterpret_cast<uint32_t*>(&h0);
+            w[2 * i + 1] = *reinterpret_cast<uint32_t*>(&h1);
+          }
+          // bf16: 64 keys = one 128-byte row of sub-tile (2b + h); this chunk covers 16-byte chunks 4cc..4cc+3
+          uint8_t* blk = sP + b * P_BLOCK_BYTES + h * (SDPA_BLOCK_Q * 128) + row_off;
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            *reinterpret_cast<uint4*>(blk + (((cc * 4 + i) ^ (r & 7)) * 16)) =
+                make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+        }
+      };
+      {
+        uint32_t va[32], vb[32];
+        tmem_ld32(t_row + h * 64, va);
+        for (int b = 0; b < NB; ++b) {
           tmem_wait_ld();
-          if constexpr (INT8) {
-            const int ci = b * 2 + cc;
-            const float mcv = ci == 0 ? mc[0] : ci == 1 ? mc[1] : ci == 2 ? mc[2] : ci == 3 ? mc[3] : ci == 4 ? mc[4] : mc[5];
-            const float f = ex2(mcv - M) * scale;
-            uint32_t w[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              const int q0 = __float2int_rn(__uint_as_float(v[4 * i + 0]) * f);
-              const int q1 = __float2int_rn(__uint_as_float(v[4 * i + 1]) * f);
-              const int q2 = __float2int_rn(__uint_as_float(v[4 * i + 2]) * f);
-              const int q3 = __float2int_rn(__uint_as_float(v[4 * i + 3]) * f);
-              // p <= 1 and inv_p <= 255, so the codes are already in [0, 255]; min() guards rounding noise
-              w[i] = min(q0, 255) | (min(q1, 255) << 8) | (min(q2, 255) << 16) | (min(q3, 255) << 24);
-              psum = static_cast<int>(__dp4a(w[i], 0x01010101u, static_cast<unsigned>(psum)));
-            }
-            uint8_t* blk = sP + b * P_BLOCK_BYTES + row_off;
-            const int c0 = h * 4 + cc * 2;                      // 16-byte chunk index inside the 128-byte row
-            *reinterpret_cast<uint4*>(blk + (((c0 + 0) ^ (r & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
-            *reinterpret_cast<uint4*>(blk + (((c0 + 1) ^ (r & 7)) * 16)) = make_uint4(w[4], w[5], w[6], w[7]);
-          } else {
-            uint32_t w[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const float e0 = ex2(fmaf(__uint_as_float(v[2 * i]), c2, mk[col + 2 * i]) - M);
-              const float e1 = ex2(fmaf(__uint_as_float(v[2 * i + 1]), c2, mk[col + 2 * i + 1]) - M);
-              __nv_bfloat162 hh = __floats2bfloat162_rn(e0, e1);
-              // the row sum is taken over the rounded values the second MMA will actually use
-              lsum += __low2float(hh) + __high2float(hh);
-              w[i] = *reinterpret_cast<uint32_t*>(&hh);
-            }
-            // bf16: 64 keys = one 128-byte row of sub-tile (2b + h); this chunk covers 16-byte chunks 4cc..4cc+3
-            uint8_t* blk = sP + b * P_BLOCK_BYTES + h * (SDPA_BLOCK_Q * 128) + row_off;
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-              *reinterpret_cast<uint4*>(blk + (((cc * 4 + i) ^ (r & 7)) * 16)) =
-                  make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+          tmem_ld32(t_row + b * 128 + h * 64 + 32, vb);
+          pass_b_chunk(va, b, 0);
+          tmem_wait_ld();
+          if (b + 1 < NB) tmem_ld32(t_row + (b + 1) * 128 + h * 64, va);
+          pass_b_chunk(vb, b, 1);
+          // this block of P is complete and its score columns have been read for the last time
+          fence_proxy_async_smem();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) {
+            mbar_arrive(bar_p_full + 8 * bx(buf, b));
+            mbar_arrive(bar_s_free + 8 * bx(buf, b));
           }
         }
-        fence_proxy_async_smem();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) {
-          mbar_arrive(bar_p_full + 8 * b);
-          mbar_arrive(bar_s_free + 8 * b);
-        }
       }
-      // combine the two halves' row sums
-      stA[r] = INT8 ? __int_as_float(psum) : lsum;
-      if (!xchg_sync()) { failed = true; break; }
-      if constexpr (INT8) prev_stat = __int_as_float(psum + __float_as_int(stB[r]));
-      else prev_stat = lsum + stB[r];
-      if (!xchg_sync()) { failed = true; break; }
+      // my half of the row sum; the partner reads it after the next exchange
+      *stat(2, upar, h) = INT8 ? __int_as_float(psum) : (lsum0 + lsum1);
+      prev_psum = psum;
+      prev_lsum = lsum0 + lsum1;
       prev_unit = unit;
     }
     if (!failed && prev_unit >= 0) {
-      if (!epilogue(prev_unit, (n - 1) & 1, prev_stat)) failed = true;
+      if (!xchg_sync()) {
+        failed = true;
+      } else {
+        const int upar = (n - 1) & 1;
+        float total;
+        if constexpr (INT8) total = __int_as_float(prev_psum + __float_as_int(*stat(2, upar, h ^ 1)));
+        else total = prev_lsum + *stat(2, upar, h ^ 1);
+        if (!epilogue(prev_unit, n - 1, total)) failed = true;
+      }
     }
+    if (lane == 0) tma_store_wait_all<0>();
     if (failed) report(p.status, DEV_TIMEOUT_EPILOGUE);
   }
 
@@ -482,22 +603,21 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   }
 }
 
-cudaError_t launch_sdpa_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const SdpaParams& p,
-                           int num_sms, cudaStream_t s) {
-  const int slots = sdpa_slots(p.S, p.is_int8, 227 * 1024);
-  if (!slots) return cudaErrorInvalidValue;
-  const size_t smem = sdpa_tc_smem_bytes(p.S, p.is_int8);
+cudaError_t launch_sdpa_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmO,
+                           const SdpaParams& p, int num_sms, cudaStream_t s) {
+  const SdpaCfg cfg = sdpa_cfg(p.S, p.is_int8);
+  if (!cfg.slots) return cudaErrorInvalidValue;
   const int units = p.B * p.H * (p.S / SDPA_BLOCK_Q);
   const int grid = units < num_sms ? units : num_sms;
   cudaError_t e;
   if (p.is_int8) {
-    e = cudaFuncSetAttribute(sdpa_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    e = cudaFuncSetAttribute(sdpa_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(cfg.smem));
     if (e != cudaSuccess) return e;
-    sdpa_tc_kernel<true><<<grid, SDPA_THREADS, smem, s>>>(tmQ, tmK, tmV, p, slots);
+    sdpa_tc_kernel<true><<<grid, SDPA_THREADS, cfg.smem, s>>>(tmQ, tmK, tmV, tmO, p, cfg.slots, cfg.nsb, cfg.stage_out);
   } else {
-    e = cudaFuncSetAttribute(sdpa_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    e = cudaFuncSetAttribute(sdpa_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(cfg.smem));
     if (e != cudaSuccess) return e;
-    sdpa_tc_kernel<false><<<grid, SDPA_THREADS, smem, s>>>(tmQ, tmK, tmV, p, slots);
+    sdpa_tc_kernel<false><<<grid, SDPA_THREADS, cfg.smem, s>>>(tmQ, tmK, tmV, tmO, p, cfg.slots, cfg.nsb, cfg.stage_out);
   }
   return cudaGetLastError();
 }
