@@ -93,7 +93,7 @@ cudaError_t launch_gemm_tc(int kind, int block_n, int a_signed, const CUtensorMa
                            const CUtensorMap& tmD, const GemmTcParams& p, int grid, bool pdl, cudaStream_t s);
 
 size_t sdpa_tc_smem_bytes(int S, int is_int8);
-// tmO: output [B*H*S, 64] with a [32 rows x 32 columns] box, swizzle = box row bytes (32 for 8-bit, 64 for bf16)
+// tmO: output [B*H*S, 64] with a [32 rows x 16 columns] box, no swizzle
 cudaError_t launch_sdpa_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmO,
                            const SdpaParams& p, int num_sms, cudaStream_t s);
 

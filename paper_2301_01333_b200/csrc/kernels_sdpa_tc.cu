@@ -1,7 +1,7 @@
 // Fused scaled-dot-product attention on tcgen05 (Section VII "MHA": two batch matmuls with the softmax and
 // the binary ops between them fused after the first one; the two matmul loop nests merged).
 //
-// Persistent CTAs (one per SM, 384 threads) walk over work units (batch, head, 128-query tile):
+// Persistent CTAs (one per SM, 640 threads) walk over work units (batch, head, 128-query tile):
 //   warp 0      TMA producer: Q tile, all K rows and all V rows of the unit into one of two shared-memory
 //               slots (128B / 64B swizzle), one unit ahead of the math (no multicast)
 //   warp 1      MMA issuer (one thread): S = Q K^T in 128-key blocks into tensor memory, O = P V in 128-key
@@ -9,9 +9,9 @@
 //               (S = 128) the next unit's S is issued a whole unit early; otherwise its blocks are issued as
 //               soon as the softmax warps release the corresponding TMEM columns
 //   warps 2-3   per-unit preparation: u8 -> s8 flip of Q (int8 path), mask row scaled by log2(e)
-//   warps 4-11  softmax: two threads per query row (TMEM lane), each owning 64 of every 128 key columns.
+//   warps 4-19  softmax: four threads per query row (TMEM lane), each owning 32 of every 128 key columns.
 //               Pass A: scale + mask, running row max, exp2 and running row sum (int8: the exponentials
-//               are written back to tensor memory); the two threads of a row combine their statistics;
+//               are written back to tensor memory); the four threads of a row combine their statistics;
 //               Pass B: normalise, quantise to u8 (int8) or cast to bf16, write P to shared memory as the
 //               K-major A operand of the second MMA.  V is consumed from its [key][d] layout as an
 //               MN-major B operand, so nothing is transposed in memory.
@@ -37,8 +37,8 @@ namespace gc {
 
 constexpr int SDPA_D = 64;
 constexpr int SDPA_BLOCK_Q = 128;
-constexpr int SDPA_THREADS = 384;
-constexpr int SDPA_SOFTMAX_WARPS = 8;
+constexpr int SDPA_THREADS = 640;
+constexpr int SDPA_SOFTMAX_WARPS = 16;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float MAGIC_F = 12582912.0f;          // 1.5 * 2^23
 constexpr int MAGIC_I = 0x4B400000;             // its bit pattern
@@ -47,7 +47,7 @@ template <bool INT8>
 struct SdpaSmem {
   static constexpr int ESZ = INT8 ? 1 : 2;
   static constexpr int ROW_BYTES = SDPA_D * ESZ;               // 64 (SW64) or 128 (SW128)
-  static constexpr int OUT_STAGING_BYTES = SDPA_SOFTMAX_WARPS * 2048;   // per softmax warp: 32 rows x <= 64 bytes
+  static constexpr int OUT_STAGING_BYTES = SDPA_SOFTMAX_WARPS * 1024;   // per softmax warp: 32 rows x <= 32 bytes
   __host__ __device__ static constexpr int q_bytes() { return SDPA_BLOCK_Q * ROW_BYTES; }
   __host__ __device__ static constexpr int kv_bytes(int S) { return S * ROW_BYTES; }
   // P: per 128-key block, 128 rows x (128 keys * ESZ) bytes = 16 KB (int8) or 32 KB (bf16)
@@ -55,7 +55,7 @@ struct SdpaSmem {
   __host__ __device__ static constexpr int slot_bytes(int S) { return q_bytes() + 2 * kv_bytes(S); }
   __host__ __device__ static constexpr int total(int S, int slots, int nsb, int stage_out) {
     return slots * slot_bytes(S) + nsb * p_bytes(S) + (stage_out ? OUT_STAGING_BYTES : 0) + slots * S * 4 /*mask*/ +
-           12 * 128 * 4 /*row statistics*/ + 256;
+           24 * 128 * 4 /*row statistics*/ + 256;
   }
 };
 
@@ -120,8 +120,8 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   uint8_t* sPall = sSlots + slots * L::slot_bytes(S);
   uint8_t* sOut = sPall + nsb * L::p_bytes(S);                            // output staging, 2 KB per softmax warp
   float* sMask = reinterpret_cast<float*>(sOut + (stage_out ? L::OUT_STAGING_BYTES : 0));   // [slots][S]
-  float* sStat = sMask + slots * S;                                       // [3 kinds][2 parities][2 halves][128]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sStat + 12 * 128);
+  float* sStat = sMask + slots * S;                                       // [3 kinds][2 parities][4 groups][128]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sStat + 24 * 128);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 24);
   const uint32_t b0 = smem_u32(bars);
   const uint32_t bar_kv_full = b0, bar_kv_empty = b0 + 16, bar_kv_ready = b0 + 32;   // [2] each
@@ -306,20 +306,22 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     }
   } else {
     // ------------------------------------------------------------------ softmax warps
-    const int sw = warp - 4;                                    // 0..7
+    // Four threads share a query row (TMEM lane): warp w covers lane quarter (w % 4) and, of every 128-key
+    // block, the 32 columns [32 g, 32 g + 32) with g = (w - 4) / 4.  Four warps per scheduler keep the
+    // TMEM / barrier / exp latencies of one warp hidden behind the others.
+    const int sw = warp - 4;                                    // 0..15
     const int q = warp & 3;                                     // TMEM lane quarter
-    const int h = sw >> 2;                                      // which 64 of every 128 key columns
+    const int g = sw >> 2;                                      // which 32 of every 128 key columns
     const int r = q * 32 + lane;                                // query row within the tile = TMEM lane
     const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
     const float c2 = (INT8 ? __fmul_rn(p.dq1, p.scalar) : p.scalar) * LOG2E;
     const uint32_t row_off = (r >> 3) * 1024 + (r & 7) * 128;
     uint32_t xphase = 0;
-    // statistics exchanged between the two threads of a row: [kind][unit parity][half][row]
-    auto stat = [&](int kind, int par, int half) { return sStat + ((kind * 2 + par) * 2 + half) * 128 + r; };
-    // this warp's staging buffer for the output tile: 32 rows x 32 columns, swizzled like its TMA store box
-    constexpr int OUT_ROW_BYTES = 32 * L::ESZ;                  // 32 (int8) or 64 (bf16)
-    uint8_t* my_out = sOut + sw * 2048;
-    const uint32_t out_swz = INT8 ? ((lane >> 2) & 1) : ((lane >> 1) & 3);   // 32B / 64B swizzle of 16-byte chunks
+    // statistics exchanged between the four threads of a row: [kind][unit parity][group][row]
+    auto stat = [&](int kind, int par, int grp) { return sStat + ((kind * 2 + par) * 4 + grp) * 128 + r; };
+    // this warp's staging buffer for the output tile: 32 rows x 16 columns, dense (no swizzle)
+    constexpr int OUT_ROW_BYTES = 16 * L::ESZ;                  // 16 (int8) or 32 (bf16)
+    uint8_t* my_out = sOut + sw * 1024;
 
     auto xchg_sync = [&]() -> bool {
       __syncwarp();
@@ -328,13 +330,13 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       xphase ^= 1;
       return ok;
     };
-    // epilogue of unit n0: my 32 of the 64 output columns
+    // epilogue of unit n0: my 16 of the 64 output columns
     auto epilogue = [&](int unit, int n0, float stat_total) -> bool {
       const int buf = buf_of(n0);
       if (!mbar_wait(bar_o_full + 8 * buf, cnt_of(n0) & 1)) return false;
       tc_fence_after();
-      uint32_t v[32];
-      tmem_ld32(t_lane + buf * BUF_COLS + S + h * 32, v);
+      uint32_t v[16];
+      tmem_ld16(t_lane + buf * BUF_COLS + S + g * 16, v);
       tmem_wait_ld();
       tc_fence_before();
       __syncwarp();
@@ -344,57 +346,48 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       }
       __syncwarp();
       const int bh = unit / q_tiles, qt = unit % q_tiles;
-      // without a staging buffer each thread stores its 32 columns of row `grow` directly
+      // without a staging buffer each thread stores its 16 columns of row `grow` directly
       const int64_t grow = static_cast<int64_t>(bh) * S + qt * SDPA_BLOCK_Q + r;
       if constexpr (INT8) {
         const int lo = p.out_dtype == GC_U8 ? 0 : -128, hi = p.out_dtype == GC_U8 ? 255 : 127;
         const int corr = p.zp_v * __float_as_int(stat_total);   // zero point of V times the row sum of P
-        uint32_t w[8];
+        // saturate(rne(u) + zp) = rne(clamp(u, lo - zp, hi - zp)) + zp: clamp in float, round with the bias
+        // trick, and fold "- bias bits + zp" into one integer add; the code is the low byte of the result
+        const float u_lo = static_cast<float>(lo - p.zp_o), u_hi = static_cast<float>(hi - p.zp_o);
+        const int kadd = p.zp_o - MAGIC_I;
+        uint32_t w[4];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          uint32_t word = 0;
+        for (int i = 0; i < 4; ++i) {
+          uint32_t y[4];
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
             const int acc = static_cast<int>(v[4 * i + k]) - corr;
-            const float t = __fmul_rn(int_to_float_magic24(acc), p.dq2);
-            word |= static_cast<uint32_t>(quantize_magic(__fmul_rn(t, p.inv_o), p.zp_o, lo, hi) & 0xFF) << (8 * k);
+            const float t = __fmul_rn(__int2float_rn(acc), p.dq2);
+            const float u = fminf(fmaxf(__fmul_rn(t, p.inv_o), u_lo), u_hi);
+            y[k] = static_cast<uint32_t>(__float_as_int(u + MAGIC_F) + kadd);
           }
-          w[i] = word;
+          w[i] = __byte_perm(__byte_perm(y[0], y[1], 0x0040), __byte_perm(y[2], y[3], 0x0040), 0x5410);
         }
-        if (stage_out) {
-          uint8_t* row = my_out + lane * OUT_ROW_BYTES;
-          *reinterpret_cast<uint4*>(row + ((0 ^ out_swz) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
-          *reinterpret_cast<uint4*>(row + ((1 ^ out_swz) * 16)) = make_uint4(w[4], w[5], w[6], w[7]);
-        } else {
-          uint4* dst = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.O) + grow * SDPA_D + h * 32);
-          dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-          dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
-        }
+        uint8_t* dst = stage_out ? my_out + lane * OUT_ROW_BYTES : static_cast<uint8_t*>(p.O) + grow * SDPA_D + g * 16;
+        *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
       } else {
         const float rl = 1.0f / stat_total;                     // deferred normalisation by the row sum
-        uint32_t w[16];
+        uint32_t w[8];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
+        for (int i = 0; i < 8; ++i) {
           __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(v[2 * i]) * rl, __uint_as_float(v[2 * i + 1]) * rl);
           w[i] = *reinterpret_cast<uint32_t*>(&hh);
         }
-        if (stage_out) {
-          uint8_t* row = my_out + lane * OUT_ROW_BYTES;
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-            *reinterpret_cast<uint4*>(row + ((i ^ out_swz) * 16)) =
-                make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
-        } else {
-          uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.O) + grow * SDPA_D + h * 32);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) dst[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
-        }
+        uint8_t* dst = stage_out ? my_out + lane * OUT_ROW_BYTES
+                                 : reinterpret_cast<uint8_t*>(static_cast<__nv_bfloat16*>(p.O) + grow * SDPA_D + g * 16);
+        reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+        reinterpret_cast<uint4*>(dst)[1] = make_uint4(w[4], w[5], w[6], w[7]);
       }
       if (stage_out) {
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
-          tma_store_2d(&tmO, h * 32, bh * S + qt * SDPA_BLOCK_Q + q * 32, smem_u32(my_out));
+          tma_store_2d(&tmO, g * 16, bh * S + qt * SDPA_BLOCK_Q + q * 32, smem_u32(my_out));
           tma_store_commit();
         }
       }
@@ -403,8 +396,6 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 
     int n = 0;
     int prev_unit = -1;
-    int prev_psum = 0;                                          // my half of the previous unit's row sum of P
-    float prev_lsum = 0.f;
     for (int unit = blockIdx.x; unit < num_units && !failed; unit += gridDim.x, ++n) {
       const int s = n % slots, buf = buf_of(n);
       const float* mk = sMask + s * S;
@@ -414,101 +405,96 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       uint8_t* sP = sPall + buf * L::p_bytes(S);
       if (!mbar_wait(bar_kv_ready + 8 * s, (n / slots) & 1)) { failed = true; break; }
 
-      // ---------------- pass A: row maximum (both paths); int8 also exponentials and row sum
+      // ---------------- pass A: one 32-column chunk per key block, transformed in place
+      // (accumulator -> scaled, masked score [-> exponential, stored back to tensor memory on the int8 path])
       float m = -INFINITY, l = 0.f;
-      float mc[6];                                              // running max after each of my chunks (int8)
-#pragma unroll
-      for (int i = 0; i < 6; ++i) mc[i] = 0.f;
-      float x[32];
-      auto pass_a_chunk = [&](const uint32_t (&v)[32], int b, int cc) {
-        const int col = b * 128 + h * 64 + cc * 32;
+      float mc[3] = {0.f, 0.f, 0.f};                            // running max after each block (int8)
+      uint32_t v[32];
+      for (int b = 0; b < NB; ++b) {
+        const int col = b * 128 + g * 32;
+        if (!mbar_wait(bar_s_full + 8 * bx(buf, b), fpar)) { failed = true; break; }
+        tc_fence_after();
+        if constexpr (INT8) tmem_wait_st();                     // v[] may still feed the previous block's store
+        tmem_ld32(t_row + col, v);
+        tmem_wait_ld();
         const float4* mk4 = reinterpret_cast<const float4*>(mk + col);
-        float cmax = -INFINITY;
-        if constexpr (INT8) tmem_wait_st();                     // x[] may still be the source of a TMEM store
+        float cm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const float4 mv = mk4[i];
           const float mm[4] = {mv.x, mv.y, mv.z, mv.w};
 #pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const float a = INT8 ? int_to_float_magic(static_cast<int>(v[4 * i + k])) : __uint_as_float(v[4 * i + k]);
-            x[4 * i + k] = fmaf(a, c2, mm[k]);
-            cmax = fmaxf(cmax, x[4 * i + k]);
+          for (int j = 0; j < 4; ++j) {
+            const float a = INT8 ? int_to_float_magic(static_cast<int>(v[4 * i + j])) : __uint_as_float(v[4 * i + j]);
+            const float xv = fmaf(a, c2, mm[j]);
+            v[4 * i + j] = __float_as_uint(xv);
+            cm[j] = fmaxf(cm[j], xv);
           }
         }
+        const float cmax = fmaxf(fmaxf(cm[0], cm[1]), fmaxf(cm[2], cm[3]));
         if constexpr (INT8) {
           const float m_new = fmaxf(m, cmax);
-          float sum0 = 0.f, sum1 = 0.f;
+          float sm[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-          for (int i = 0; i < 32; i += 2) {
-            x[i] = ex2(x[i] - m_new);
-            x[i + 1] = ex2(x[i + 1] - m_new);
-            sum0 += x[i];
-            sum1 += x[i + 1];
+          for (int i = 0; i < 32; i += 4) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const float e = ex2(__uint_as_float(v[i + j]) - m_new);
+              v[i + j] = __float_as_uint(e);
+              sm[j] += e;
+            }
           }
-          l = l * ex2(m - m_new) + (sum0 + sum1);
+          l = l * ex2(m - m_new) + ((sm[0] + sm[1]) + (sm[2] + sm[3]));
           m = m_new;
-          const int ci = b * 2 + cc;
-          if (ci == 0) mc[0] = m; else if (ci == 1) mc[1] = m; else if (ci == 2) mc[2] = m;
-          else if (ci == 3) mc[3] = m; else if (ci == 4) mc[4] = m; else mc[5] = m;
-          tmem_st32(t_row + col, reinterpret_cast<const uint32_t(&)[32]>(x));
+          if (b == 0) mc[0] = m; else if (b == 1) mc[1] = m; else mc[2] = m;
+          tmem_st32(t_row + col, v);
         } else {
           m = fmaxf(m, cmax);
-        }
-      };
-      {
-        uint32_t va[32], vb[32];
-        if (!mbar_wait(bar_s_full + 8 * bx(buf, 0), fpar)) { failed = true; break; }
-        tc_fence_after();
-        tmem_ld32(t_row + h * 64, va);
-        for (int b = 0; b < NB; ++b) {
-          tmem_wait_ld();
-          tmem_ld32(t_row + b * 128 + h * 64 + 32, vb);         // next chunk in flight while this one is processed
-          pass_a_chunk(va, b, 0);
-          tmem_wait_ld();
-          if (b + 1 < NB) {
-            if (!mbar_wait(bar_s_full + 8 * bx(buf, b + 1), fpar)) { failed = true; break; }
-            tc_fence_after();
-            tmem_ld32(t_row + (b + 1) * 128 + h * 64, va);
-          }
-          pass_a_chunk(vb, b, 1);
         }
       }
       if (failed) break;
       if constexpr (INT8) tmem_wait_st();
-      *stat(0, upar, h) = m;
-      if constexpr (INT8) *stat(1, upar, h) = l;
+      *stat(0, upar, g) = m;
+      if constexpr (INT8) *stat(1, upar, g) = l;
       if (!xchg_sync()) { failed = true; break; }
+      // every thread of a row combines the four parts in the same order, so all four get identical values
+      float M = -INFINITY;
+#pragma unroll
+      for (int o = 0; o < 4; ++o) M = fmaxf(M, *stat(0, upar, o));
       float scale = 1.f;                                        // int8: inv_p / row sum
-      float M;
-      {
-        const float m_p = *stat(0, upar, h ^ 1);
-        M = fmaxf(m, m_p);
-        if constexpr (INT8) {
-          const float l_p = *stat(1, upar, h ^ 1);
-          const float Lsum = l * ex2(m - M) + l_p * ex2(m_p - M);
-          scale = p.inv_p / Lsum;
-        }
+      if constexpr (INT8) {
+        float Lsum = 0.f;
+#pragma unroll
+        for (int o = 0; o < 4; ++o) Lsum += *stat(1, upar, o) * ex2(*stat(0, upar, o) - M);
+        scale = p.inv_p / Lsum;
       }
 
       // ---------------- epilogue of the previous unit (its second MMA has had a whole pass to finish);
-      // the partner's half of that unit's row sum became visible with the exchange above
+      // the other threads' parts of that unit's row sum became visible with the exchange above
       if (prev_unit >= 0) {
         float total;
-        if constexpr (INT8) total = __int_as_float(prev_psum + __float_as_int(*stat(2, upar ^ 1, h ^ 1)));
-        else total = prev_lsum + *stat(2, upar ^ 1, h ^ 1);
+        if constexpr (INT8) {
+          int t = 0;
+#pragma unroll
+          for (int o = 0; o < 4; ++o) t += __float_as_int(*stat(2, upar ^ 1, o));
+          total = __int_as_float(t);
+        } else {
+          total = 0.f;
+#pragma unroll
+          for (int o = 0; o < 4; ++o) total += *stat(2, upar ^ 1, o);
+        }
         if (!epilogue(prev_unit, n - 1, total)) { failed = true; break; }
       }
 
       // ---------------- pass B: normalise, round, write P
       int psum = 0;
-      float lsum0 = 0.f, lsum1 = 0.f;
-      auto pass_b_chunk = [&](const uint32_t (&v)[32], int b, int cc) {
-        const int col = b * 128 + h * 64 + cc * 32;
+      float lsum = 0.f;
+      for (int b = 0; b < NB; ++b) {
+        const int col = b * 128 + g * 32;
         if constexpr (INT8) {
-          const int ci = b * 2 + cc;
-          const float mcv = ci == 0 ? mc[0] : ci == 1 ? mc[1] : ci == 2 ? mc[2] : ci == 3 ? mc[3] : ci == 4 ? mc[4] : mc[5];
-          const float f = ex2(mcv - M) * scale;
+          tmem_ld32(t_row + col, v);
+          tmem_wait_ld();
+          const float f = ex2((b == 0 ? mc[0] : b == 1 ? mc[1] : mc[2]) - M) * scale;
           uint32_t w[8];
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
@@ -522,57 +508,56 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             psum = static_cast<int>(__dp4a(w[i], 0x01010101u, static_cast<unsigned>(psum)));
           }
           uint8_t* blk = sP + b * P_BLOCK_BYTES + row_off;
-          const int c0 = h * 4 + cc * 2;                        // 16-byte chunk index inside the 128-byte row
+          const int c0 = g * 2;                                 // 16-byte chunk index inside the 128-byte row
           *reinterpret_cast<uint4*>(blk + (((c0 + 0) ^ (r & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
           *reinterpret_cast<uint4*>(blk + (((c0 + 1) ^ (r & 7)) * 16)) = make_uint4(w[4], w[5], w[6], w[7]);
         } else {
-          const float4* mk4 = reinterpret_cast<const float4*>(mk + col);
+          if (NB > 1) {                                         // with one key block the scores are still in v[]
+            tmem_ld32(t_row + col, v);
+            tmem_wait_ld();
+            const float4* mk4 = reinterpret_cast<const float4*>(mk + col);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const float4 mv = mk4[i];
+              v[4 * i + 0] = __float_as_uint(fmaf(__uint_as_float(v[4 * i + 0]), c2, mv.x));
+              v[4 * i + 1] = __float_as_uint(fmaf(__uint_as_float(v[4 * i + 1]), c2, mv.y));
+              v[4 * i + 2] = __float_as_uint(fmaf(__uint_as_float(v[4 * i + 2]), c2, mv.z));
+              v[4 * i + 3] = __float_as_uint(fmaf(__uint_as_float(v[4 * i + 3]), c2, mv.w));
+            }
+          }
           uint32_t w[16];
+          float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            const float4 mv = mk4[i];
-            const float e0 = ex2(fmaf(__uint_as_float(v[4 * i + 0]), c2, mv.x) - M);
-            const float e1 = ex2(fmaf(__uint_as_float(v[4 * i + 1]), c2, mv.y) - M);
-            const float e2 = ex2(fmaf(__uint_as_float(v[4 * i + 2]), c2, mv.z) - M);
-            const float e3 = ex2(fmaf(__uint_as_float(v[4 * i + 3]), c2, mv.w) - M);
-            lsum0 += e0 + e2;
-            lsum1 += e1 + e3;
+            const float e0 = ex2(__uint_as_float(v[4 * i + 0]) - M);
+            const float e1 = ex2(__uint_as_float(v[4 * i + 1]) - M);
+            const float e2 = ex2(__uint_as_float(v[4 * i + 2]) - M);
+            const float e3 = ex2(__uint_as_float(v[4 * i + 3]) - M);
+            ls[0] += e0; ls[1] += e1; ls[2] += e2; ls[3] += e3;
             __nv_bfloat162 h0 = __floats2bfloat162_rn(e0, e1), h1 = __floats2bfloat162_rn(e2, e3);
             w[2 * i] = *reinterpret_cast<uint32_t*>(&h0);
             w[2 * i + 1] = *reinterpret_cast<uint32_t*>(&h1);
           }
-          // bf16: 64 keys = one 128-byte row of sub-tile (2b + h); this chunk covers 16-byte chunks 4cc..4cc+3
-          uint8_t* blk = sP + b * P_BLOCK_BYTES + h * (SDPA_BLOCK_Q * 128) + row_off;
+          lsum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+          // bf16: a 128-key block is two 64-key sub-tiles (128-byte rows); my 32 keys are 4 chunks of 16 bytes
+          uint8_t* blk = sP + b * P_BLOCK_BYTES + (g >> 1) * (SDPA_BLOCK_Q * 128) + row_off;
+          const int c0 = (g & 1) * 4;
 #pragma unroll
           for (int i = 0; i < 4; ++i)
-            *reinterpret_cast<uint4*>(blk + (((cc * 4 + i) ^ (r & 7)) * 16)) =
+            *reinterpret_cast<uint4*>(blk + (((c0 + i) ^ (r & 7)) * 16)) =
                 make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
         }
-      };
-      {
-        uint32_t va[32], vb[32];
-        tmem_ld32(t_row + h * 64, va);
-        for (int b = 0; b < NB; ++b) {
-          tmem_wait_ld();
-          tmem_ld32(t_row + b * 128 + h * 64 + 32, vb);
-          pass_b_chunk(va, b, 0);
-          tmem_wait_ld();
-          if (b + 1 < NB) tmem_ld32(t_row + (b + 1) * 128 + h * 64, va);
-          pass_b_chunk(vb, b, 1);
-          // this block of P is complete and its score columns have been read for the last time
-          fence_proxy_async_smem();
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) {
-            mbar_arrive(bar_p_full + 8 * bx(buf, b));
-            mbar_arrive(bar_s_free + 8 * bx(buf, b));
-          }
+        // this block of P is complete and its score columns have been read for the last time
+        fence_proxy_async_smem();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(bar_p_full + 8 * bx(buf, b));
+          mbar_arrive(bar_s_free + 8 * bx(buf, b));
         }
       }
-      // my half of the row sum; the partner reads it after the next exchange
-      *stat(2, upar, h) = INT8 ? __int_as_float(psum) : (lsum0 + lsum1);
-      prev_psum = psum;
-      prev_lsum = lsum0 + lsum1;
+      // my part of the row sum; the other threads of the row read it after the next exchange
+      *stat(2, upar, g) = INT8 ? __int_as_float(psum) : lsum;
       prev_unit = unit;
     }
     if (!failed && prev_unit >= 0) {
@@ -581,8 +566,16 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       } else {
         const int upar = (n - 1) & 1;
         float total;
-        if constexpr (INT8) total = __int_as_float(prev_psum + __float_as_int(*stat(2, upar, h ^ 1)));
-        else total = prev_lsum + *stat(2, upar, h ^ 1);
+        if constexpr (INT8) {
+          int t = 0;
+#pragma unroll
+          for (int o = 0; o < 4; ++o) t += __float_as_int(*stat(2, upar, o));
+          total = __int_as_float(t);
+        } else {
+          total = 0.f;
+#pragma unroll
+          for (int o = 0; o < 4; ++o) total += *stat(2, upar, o);
+        }
         if (!epilogue(prev_unit, n - 1, total)) failed = true;
       }
     }
