@@ -50,26 +50,28 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+// One try_wait with a suspend-time hint: the hardware parks the thread (it issues nothing and leaves the
+// schedulers to the working warps) until the phase completes or roughly `hint_ns` nanoseconds pass.
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred P;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2, %3;\n\t"
       "selp.b32 %0, 1, 0, P;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(hint_ns)
       : "memory");
   return ok != 0;
 }
 
-// Bounded wait: gives up after ~2 s of wall time (or 2^26 polls) and returns false.  The caller
-// then records an error code in the status word and leaves its loop; nothing spins forever.
+// Bounded wait: gives up after ~2 s of wall time and returns false.  The caller then records an error
+// code in the status word and leaves its loop; nothing spins forever.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
+  if (mbar_try_wait(bar, parity, 1000u)) return true;
   const uint64_t t0 = globaltimer_ns();
-  for (uint32_t i = 0; i < (1u << 26); ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 255u) == 255u && globaltimer_ns() - t0 > 2000000000ull) break;
+  for (uint32_t i = 0; i < (1u << 22); ++i) {
+    if (mbar_try_wait(bar, parity, 20000u)) return true;
+    if ((i & 15u) == 15u && globaltimer_ns() - t0 > 2000000000ull) break;
   }
   return false;
 }
