@@ -21,7 +21,7 @@ def _built():
 def test_library_exports_every_declared_symbol():
     text = open(os.path.join(ROOT, "include", "gc.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    declared = set(re.findall(r"\b(gc_[a-z_]+)\s*\(", text))
+    declared = set(re.findall(r"\b(gc_[a-z0-9_]+)\s*\(", text))
     assert declared == set(B.EXPORTS)
     lib = B.load_library()
     for name in declared:
