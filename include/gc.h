@@ -170,6 +170,31 @@ gc_status_t gc_query_status(gc_compiled_t* c, void* cuda_stream);
 gc_status_t gc_launches_per_execute(const gc_compiled_t* c, int32_t* n);
 const char* gc_plan_description(const gc_compiled_t* c);
 
+/* No counterpart in the paper: an entry point for callers that cannot allocate device memory.
+ *
+ * Some callers may not call cudaMalloc at all - a real-time loop with a fixed memory plan, a process
+ * whose allocator owns the whole device and gives nothing back at run time, a component that is only
+ * allowed to launch work on buffers it was handed.  The regular path asks such a caller for a
+ * workspace it cannot provide.  gc_matmul_s32_noalloc computes
+ *     out[m, n] (s32) = sum_k (a[m, k] - a_zero_point) * w[k, n]      a: u8 [m, k], w: s8 [k, n], row-major
+ * exactly, like a MatMul-only partition, but keeps its scratch (the transposed, zero-padded weight
+ * the kernel consumes) in a fixed array inside the library image.  It calls no allocating routine.
+ *
+ *   - Limit: n * round_up(k, 128) <= gc_noalloc_scratch_bytes() (1 MiB); larger problems are rejected
+ *     with GC_ERR_UNSUPPORTED and a message - use gc_compile / gc_execute with a workspace instead.
+ *   - The array costs every GPU that loads this library 1 MiB of device memory until the process exits.
+ *   - All calls share the array.  Calls that can overlap on the GPU (different streams, or host threads
+ *     racing on one stream) corrupt each other's scratch: keep them on one stream or serialise them.
+ *     The array keeps the previous call's contents; every byte that is read is rewritten first, so no
+ *     clearing is needed between calls.
+ *   - The first call on each device looks up the array's device address (with that device current) and
+ *     caches it; make that first call before any stream capture begins.
+ *   - All three pointers are device pointers on the current device; out must be 4-byte aligned.
+ *     Asynchronous on cuda_stream like gc_execute. */
+gc_status_t gc_matmul_s32_noalloc(void* cuda_stream, const void* a_dev, const void* w_dev, void* out_dev,
+                                  int32_t m, int32_t k, int32_t n, int32_t a_zero_point);
+size_t gc_noalloc_scratch_bytes(void);
+
 const char* gc_last_error(void);
 const char* gc_version(void);
 

@@ -33,6 +33,7 @@ EXPORTS = [
     "gc_partition_create", "gc_partition_destroy", "gc_compile", "gc_compiled_destroy", "gc_workspace_bytes",
     "gc_set_workspace", "gc_execute", "gc_host_staging_bytes", "gc_set_host_staging", "gc_execute_host",
     "gc_query_status", "gc_launches_per_execute", "gc_plan_description", "gc_last_error", "gc_version",
+    "gc_matmul_s32_noalloc", "gc_noalloc_scratch_bytes",
 ]
 
 
@@ -88,6 +89,9 @@ def load_library() -> C.CDLL:
     lib.gc_plan_description.restype = C.c_char_p
     lib.gc_last_error.restype = C.c_char_p
     lib.gc_version.restype = C.c_char_p
+    lib.gc_matmul_s32_noalloc.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32]
+    lib.gc_matmul_s32_noalloc.restype = i32
+    lib.gc_noalloc_scratch_bytes.restype = sz
     for name in ("gc_partition_create", "gc_compile", "gc_workspace_bytes", "gc_set_workspace", "gc_execute",
                  "gc_host_staging_bytes", "gc_set_host_staging", "gc_execute_host", "gc_query_status",
                  "gc_launches_per_execute"):
@@ -209,6 +213,18 @@ def gc_launches_per_execute(c) -> int:
 
 def gc_plan_description(c) -> str:
     return load_library().gc_plan_description(c).decode()
+
+
+def gc_noalloc_scratch_bytes() -> int:
+    return load_library().gc_noalloc_scratch_bytes()
+
+
+def gc_matmul_s32_noalloc(stream: int, a_ptr: int, w_ptr: int, out_ptr: int, m: int, k: int, n: int,
+                          a_zero_point: int = 0) -> None:
+    """out[m,n] (s32) = (a - zp) @ w for u8 a [m,k] and s8 w [k,n], all device pointers.  For callers
+    that cannot allocate: the scratch is a fixed 1 MiB array inside the library, shared by all calls."""
+    _check(load_library().gc_matmul_s32_noalloc(C.c_void_p(stream), C.c_void_p(a_ptr), C.c_void_p(w_ptr),
+                                                C.c_void_p(out_ptr), m, k, n, a_zero_point))
 
 
 class CompiledPartition:

@@ -36,6 +36,9 @@ static gc_status_t fail(gc_status_t st, const char* fmt, ...) {
     if (e__ != cudaSuccess) return fail(GC_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e__)); \
   } while (0)
 
+// for the other translation units of the library: record a message for gc_last_error() and pass the status on
+gc_status_t gc_set_error(gc_status_t st, const char* msg) { return fail(st, "%s", msg); }
+
 extern "C" const char* gc_last_error(void) { return g_err; }
 extern "C" const char* gc_version(void) { return "gc-b200 0.1 (sm_100a)"; }
 
