@@ -192,6 +192,7 @@ struct LayerPlan {
   size_t in_off = 0;         // workspace offset of the previous intermediate
   int64_t a_pitch = 0;       // elements
   bool use_tc = false;
+  bool cta2 = false;         // CTA-pair kernel (256 x 256 tiles per cluster of two)
   int kind = 0, block_n = 0, grid = 0, m_tiles = 0, n_tiles = 0, nkb = 0;
   bool need_pack = false;
   size_t pack_off = 0;
@@ -486,6 +487,14 @@ static void choose_tile(LayerPlan& L, int num_sms) {
   L.n_tiles = (L.N + pick - 1) / pick;
   const int tiles = L.m_tiles * L.n_tiles;
   L.grid = tiles < num_sms ? tiles : num_sms;
+  // Large problems: pair the CTAs.  A pair loads 32 KB per CTA and k-block instead of 48 KB, which lifts the
+  // operand-fetch bound of the one-CTA 128 x 256 tile.
+  L.cta2 = pick == 256 && L.m_tiles >= 2 && tiles >= num_sms;
+  if (L.cta2) {
+    const int pair_tiles = ((L.m_tiles + 1) / 2) * L.n_tiles;
+    const int clusters = pair_tiles < num_sms / 2 ? pair_tiles : num_sms / 2;
+    L.grid = 2 * clusters;
+  }
 }
 
 extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, const gc_compile_options_t* opt,
@@ -627,7 +636,7 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
       c->launches += 1;
       snprintf(line, sizeof(line), "  layer %zu: M=%d K=%d N=%d kernel=%s block_n=%d grid=%d%s act=%d out=%d\n", l, L.M, L.K,
                L.N, L.use_tc ? (L.kind == 0 ? "tcgen05.i8" : L.kind == 1 ? "tcgen05.bf16" : "tcgen05.tf32") : "cuda-core",
-               L.block_n, L.grid, L.need_pack ? " +pack" : "", L.epi.act, L.epi.out_dtype);
+               L.block_n, L.grid, L.cta2 ? " cta_pair" : (L.need_pack ? " +pack" : ""), L.epi.act, L.epi.out_dtype);
       c->desc += line;
     }
   }
@@ -731,7 +740,7 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
       }
       if (!L.tmB_valid) {
         gc_status_t s = make_tmap(&L.tmB, ws + L.wt_off, L.w_dtype, L.Kp, L.N, static_cast<uint64_t>(L.Kp) * esz, k_elems,
-                                  L.block_n, 128);
+                                  L.cta2 ? 128 : L.block_n, 128);
         if (s != GC_OK) return s;
         L.tmB_valid = true;
       }
@@ -754,8 +763,11 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
         L.tmD_ptr = O;
       }
       const bool pdl = !c.opt.no_chain_fusion && l > 0 && !L.need_pack;
-      CUDA_TRY(launch_gemm_tc(L.kind, L.block_n, L.a_dtype == GC_S8, L.tmA, L.tmB, box_cols ? L.tmD : L.tmA, g, L.grid,
-                              pdl, st));
+      if (L.cta2)
+        CUDA_TRY(launch_gemm_tc2(L.kind, L.a_dtype == GC_S8, L.tmA, L.tmB, L.tmD, g, L.grid, pdl, st));
+      else
+        CUDA_TRY(launch_gemm_tc(L.kind, L.block_n, L.a_dtype == GC_S8, L.tmA, L.tmB, box_cols ? L.tmD : L.tmA, g, L.grid,
+                                pdl, st));
     } else {
       GemmSimtParams g = {};
       g.A = A;

@@ -92,6 +92,12 @@ int gemm_tc_store_box_cols(int block_n, int out_elem_bytes);
 cudaError_t launch_gemm_tc(int kind, int block_n, int a_signed, const CUtensorMap& tmA, const CUtensorMap& tmB,
                            const CUtensorMap& tmD, const GemmTcParams& p, int grid, bool pdl, cudaStream_t s);
 
+// CTA-pair variant (cta_group::2): 256 x 256 tiles per cluster of two CTAs; tmB must have a 128-row box.
+// `grid` must be even.
+size_t gemm_tc2_smem_bytes();
+cudaError_t launch_gemm_tc2(int kind, int a_signed, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmD,
+                            const GemmTcParams& p, int grid, bool pdl, cudaStream_t s);
+
 size_t sdpa_tc_smem_bytes(int S, int is_int8);
 // tmO: output [B*H*S, 64] with a [32 rows x 16 columns] box, no swizzle
 cudaError_t launch_sdpa_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmO,

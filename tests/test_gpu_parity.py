@@ -97,6 +97,22 @@ def test_float_matmul(B, m, k, n, dtype, tol):
     assert np.abs(got - ref).max() <= tol * np.abs(ref).max()
 
 
+@pytest.mark.parametrize("m,k,n", [(2600, 512, 2048), (4096, 200, 1280)])
+def test_cta_pair_gemm_int8_exact(B, m, k, n):
+    # large enough for the CTA-pair kernel; 2600 rows = 21 row blocks, so the last pair has an empty partner
+    w = W.single_matmul("u8", "s8", m, k, n, seed=11)
+    got, plan = run_gpu(B, w)
+    assert "cta_pair" in plan
+    assert np.array_equal(got.astype(np.int64), oracle(w))
+
+
+def test_cta_pair_gemm_bf16_with_epilogue(B):
+    w = W.ffn_bf16(tokens=2600, d_model=256, d_ff=2048)
+    got, plan = run_gpu(B, w)
+    assert "cta_pair" in plan
+    assert np.abs(bf16_to_f64(got) - oracle(w)).max() <= 2e-2
+
+
 def test_batched_matmul_int8_exact(B):
     w = W.single_matmul("u8", "u8", 24, 16, 24, seed=3, transpose_b=True, a_zp=128, batch=(2, 3))
     w.graph.tensors[w.graph.inputs[1]].zero_point = 128
