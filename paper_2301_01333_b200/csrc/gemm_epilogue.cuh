@@ -21,8 +21,9 @@ __device__ __forceinline__ void epi_values32(const uint32_t (&raw)[32], float (&
     const float4* bp = reinterpret_cast<const float4*>(e.bias + n0);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      // columns at or beyond n_end belong to a clipped tile tail: never read the bias there
-      const float4 v = n0 + 4 * i < n_end ? __ldg(bp + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+      // columns at or beyond n_end belong to a clipped tile tail: never read the bias there.  The pointer
+      // may address global memory or a shared-memory copy of the tile's bias slice (generic load).
+      const float4 v = n0 + 4 * i < n_end ? bp[i] : make_float4(0.f, 0.f, 0.f, 0.f);
       b[4 * i] = v.x; b[4 * i + 1] = v.y; b[4 * i + 2] = v.z; b[4 * i + 3] = v.w;
     }
   } else {

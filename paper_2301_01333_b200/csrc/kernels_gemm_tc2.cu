@@ -21,14 +21,17 @@ namespace gc {
 constexpr int G2_BLOCK_M = 128;          // rows per CTA (256 per pair)
 constexpr int G2_BLOCK_N = 256;
 constexpr int G2_B_ROWS = 128;           // Wt rows each CTA loads
-constexpr int G2_STAGES = 6;
+constexpr int G2_STAGES = 5;
 constexpr int G2_STAGE_BYTES = (G2_BLOCK_M + G2_B_ROWS) * 128;
 constexpr int G2_EPI_WARPS = 8;
 constexpr int G2_THREADS = 64 + 32 * G2_EPI_WARPS;
-constexpr int G2_STAGING_BYTES = G2_EPI_WARPS * 4096;
+constexpr int G2_STAGING_BYTES = G2_EPI_WARPS * 4096;       // one [32 rows x 128 B] box per epilogue warp
+constexpr int G2_BIAS_BYTES = G2_EPI_WARPS * G2_BLOCK_N * 4;  // per epilogue warp: the tile's 256 bias values
 constexpr int G2_TMEM_COLS = 512;
 
-size_t gemm_tc2_smem_bytes() { return static_cast<size_t>(G2_STAGES) * G2_STAGE_BYTES + G2_STAGING_BYTES + 1024 + 256; }
+size_t gemm_tc2_smem_bytes() {
+  return static_cast<size_t>(G2_STAGES) * G2_STAGE_BYTES + G2_STAGING_BYTES + G2_BIAS_BYTES + 1024 + 256;
+}
 
 template <int KIND, int OUT>
 __global__ void __launch_bounds__(G2_THREADS, 1)
@@ -43,7 +46,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* staging = smem + G2_STAGES * G2_STAGE_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(staging + G2_STAGING_BYTES);
+  float* bias_smem = reinterpret_cast<float*>(staging + G2_STAGING_BYTES);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(staging + G2_STAGING_BYTES + G2_BIAS_BYTES);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * G2_STAGES + 4);
   const uint32_t smem_base = smem_u32(smem);
   const uint32_t bar_full = smem_u32(bars);                       // [STAGES]  (used in the leader)
@@ -160,10 +164,25 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     uint32_t acc_phase = 0;
     uint8_t* my_stage = staging + ew * 4096;
     const uint32_t my_stage_u32 = smem_u32(my_stage);
+    float* my_bias = bias_smem + ew * G2_BLOCK_N;
     const uint32_t row_off = (lane >> 3) * 1024 + (lane & 7) * 128;
     const uint32_t leader_tempty = leader ? bar_tempty : mapa_shared(bar_tempty, 0);
     for (int tile = cluster_id; tile < num_tiles; tile += num_clusters) {
       const int m_blk = (tile / p.n_tiles) * 2 + static_cast<int>(rank), n_blk = tile % p.n_tiles;
+      // Copy this tile's bias slice into shared memory while the accumulator is still being produced: a
+      // global load in the per-chunk loop would put its full latency on the critical path of every chunk.
+      Epilogue epi = p.epi;
+      if (p.epi.bias) {
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const int c = n_blk * G2_BLOCK_N + (lane + 32 * i) * 4;
+          const float4 v = c < p.N ? __ldg(reinterpret_cast<const float4*>(p.epi.bias + c)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          reinterpret_cast<float4*>(my_bias)[lane + 32 * i] = v;
+        }
+        __syncwarp();
+        epi.bias = my_bias - n_blk * G2_BLOCK_N;                   // indexed by absolute column below
+      }
       if (!mbar_wait(bar_tfull + 8 * acc, acc_phase)) {
         report(p.status, DEV_TIMEOUT_EPILOGUE);
         failed = true;
@@ -172,6 +191,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       tc_fence_after();
       const uint32_t t_row = tmem_base + acc * G2_BLOCK_N + (static_cast<uint32_t>(q * 32) << 16);
       for (int box = half; box < NUM_BOXES; box += 2) {
+        // the previous store out of this warp's staging buffer must have read it completely
         if (lane == 0) tma_store_wait_read<0>();
         __syncwarp();
 #pragma unroll 1
@@ -181,7 +201,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           tmem_wait_ld();
           constexpr int NW = 32 * OUT_BYTES / 4;
           uint32_t w[NW];
-          epi_chunk32<KIND, OUT>(r, w, n_blk * G2_BLOCK_N + box * BOX_COLS + sub * 32, p.N, p.epi);
+          epi_chunk32<KIND, OUT>(r, w, n_blk * G2_BLOCK_N + box * BOX_COLS + sub * 32, p.N, epi);
           const int c0 = sub * (NW / 4);
 #pragma unroll
           for (int i = 0; i < NW / 4; ++i)
