@@ -58,9 +58,37 @@ __device__ __forceinline__ void epi_store16(const uint32_t* raw, void* dst_row, 
     for (int i = 0; i < 4; ++i) d[i] = make_int4(raw[4 * i], raw[4 * i + 1], raw[4 * i + 2], raw[4 * i + 3]);
     return;
   }
+  // Fetch the 16 bias values with four vector loads up front: per-element loads behind per-element branches
+  // serialise into 16 dependent memory latencies.
+  float b[16];
+  if (e.bias) {
+    const float4* bp = reinterpret_cast<const float4*>(e.bias + n0);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float4 v = __ldg(bp + i);
+      b[4 * i] = v.x; b[4 * i + 1] = v.y; b[4 * i + 2] = v.z; b[4 * i + 3] = v.w;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) b[i] = 0.f;
+  }
+  const bool has_bias = e.bias != nullptr, acc_int = e.acc_is_int != 0;
+  const float dq = e.dq;
+  const int act = e.act;
   float t[16];
 #pragma unroll
-  for (int i = 0; i < 16; ++i) t[i] = epi_value(raw[i], n0 + i, e);
+  for (int i = 0; i < 16; ++i) {
+    float x = acc_int ? __fmul_rn(__int2float_rn(static_cast<int>(raw[i])), dq) : __uint_as_float(raw[i]);
+    x = has_bias ? __fadd_rn(x, b[i]) : x;      // separately rounded: exact on the integer path
+    t[i] = x;
+  }
+  if (act == ACT_RELU) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) t[i] = fmaxf(t[i], 0.0f);
+  } else if (act != ACT_NONE) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) t[i] = apply_act(t[i], act);
+  }
   if (e.out_dtype == GC_F32) {
     float4* d = reinterpret_cast<float4*>(static_cast<float*>(dst_row) + n0);
 #pragma unroll

@@ -231,6 +231,17 @@ struct gc_compiled {
   std::vector<const void*> const_ptrs;   // constant input pointers seen at the last prepack
   int launches = 0;
   std::string desc;
+  // fused small-batch chain (one persistent kernel for all layers)
+  bool chain_fused = false;
+  int chain_kind = 0, chain_grid = 0, chain_barriers = 0;
+  size_t chain_tmap_off = 0;                 // workspace offset of the tensor-map array
+  uint32_t chain_w_smem = 0;
+  int chain_a_stages = 0, chain_a_stage_bytes = 0, chain_a_rows = 0;
+  std::vector<uint32_t> chain_w_off;         // per layer: offset of its weight slice in shared memory
+  unsigned long long chain_arrivals = 0;     // value of the grid-barrier counter after the launches so far
+  std::vector<CUtensorMap> chain_tmaps;      // host copy of the tensor-map array
+  const void* chain_a0_ptr = nullptr;        // first-layer A pointer the array was built for
+  bool chain_tmaps_valid = false;
   // host staging
   size_t staging_bytes = 0;
   void* staging = nullptr;
@@ -640,6 +651,57 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
       c->desc += line;
     }
   }
+  if (c->pattern == PAT_MLP && !c->opt.no_chain_fusion && !c->opt.force_generic && c->layers.size() >= 2 &&
+      c->layers.size() <= static_cast<size_t>(CHAIN_MAX_LAYERS)) {
+    // Small-batch chains run as one persistent kernel when every layer fits one MMA row tile and all
+    // weight slices of a CTA fit in shared memory next to the activation ring.
+    bool ok = true;
+    int kind = -1, max_ctas = 0;
+    uint32_t w_smem = 0;
+    c->chain_w_off.assign(c->layers.size(), 0);
+    for (size_t l = 0; l < c->layers.size() && ok; ++l) {
+      LayerPlan& L = c->layers[l];
+      ok = L.M <= 128;
+      const int lk = is_int8(L.a_dtype) ? 0 : (L.a_dtype == GC_BF16 ? 1 : 2);
+      if (kind < 0) kind = lk;
+      ok = ok && lk == kind;
+      if (L.use_tc) {
+        const int ctas = (L.N + 31) / 32;
+        max_ctas = ctas > max_ctas ? ctas : max_ctas;
+        c->chain_w_off[l] = w_smem;
+        w_smem += static_cast<uint32_t>(L.nkb) * 32 * 128;
+      }
+    }
+    // A-operand ring: round_up(M, 8) rows per stage, as many stages as fit (all k-blocks of the deepest
+    // layer if possible, so every layer fetches its whole A operand in one burst)
+    int a_rows = 8, max_nkb = 1;
+    for (auto& L : c->layers) {
+      a_rows = ((L.M + 7) / 8 * 8) > a_rows ? ((L.M + 7) / 8 * 8) : a_rows;
+      if (L.use_tc && L.nkb > max_nkb) max_nkb = L.nkb;
+    }
+    const int a_stage_bytes = a_rows * 128;
+    int a_stages = max_nkb < 32 ? max_nkb : 32;
+    while (a_stages > 2 && mlp_chain_smem_bytes(w_smem, a_stages, a_stage_bytes) > static_cast<size_t>(prop.sharedMemPerBlockOptin))
+      --a_stages;
+    ok = ok && max_ctas > 0 && max_ctas <= c->num_sms && a_stages >= max_nkb &&
+         mlp_chain_smem_bytes(w_smem, a_stages, a_stage_bytes) <= static_cast<size_t>(prop.sharedMemPerBlockOptin);
+    if (ok) {
+      c->chain_a_stages = a_stages;
+      c->chain_a_stage_bytes = a_stage_bytes;
+      c->chain_a_rows = a_rows;
+      c->chain_fused = true;
+      c->chain_kind = kind;
+      c->chain_grid = max_ctas;
+      c->chain_w_smem = w_smem;
+      c->chain_barriers = (c->layers[0].need_pack ? 1 : 0) + static_cast<int>(c->layers.size()) - 1;
+      c->chain_tmap_off = ws;
+      ws = align_up(ws + 2 * CHAIN_MAX_LAYERS * sizeof(CUtensorMap), 1024);
+      c->launches = 1;
+      snprintf(line, sizeof(line), "  fused chain: one persistent kernel, %d CTAs, %u KB of resident weight slices per CTA, %d grid barriers\n",
+               max_ctas, w_smem / 1024, c->chain_barriers);
+      c->desc += line;
+    }
+  }
   c->ws_bytes = align_up(ws, 1024);
   // host staging layout
   size_t so = 0;
@@ -671,6 +733,8 @@ extern "C" gc_status_t gc_set_workspace(gc_compiled_t* c, void* ws, size_t bytes
   c->ws = ws;
   c->prepacked = false;
   c->status_cleared = false;
+  c->chain_arrivals = 0;                     // the header (status word + barrier counter) is cleared again
+  c->chain_tmaps_valid = false;
   for (auto& L : c->layers) {
     L.tmA_ptr = nullptr;
     L.tmD_ptr = nullptr;
@@ -717,6 +781,78 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
       c.const_ptrs[L.w_input] = in[L.w_input];
     }
     c.prepacked = true;
+  }
+  if (c.chain_fused) {
+    ChainParams cp = {};
+    cp.n_layers = static_cast<int>(c.layers.size());
+    cp.w_smem_bytes = c.chain_w_smem;
+    cp.a_stages = c.chain_a_stages;
+    cp.a_stage_bytes = c.chain_a_stage_bytes;
+    cp.status = status;
+    cp.barrier = reinterpret_cast<unsigned long long*>(ws + 64);
+    cp.barrier_base = c.chain_arrivals;
+    const LayerPlan& L0 = c.layers[0];
+    const void* a0 = in[L0.a_input];
+    if (L0.need_pack) {
+      const int esz0 = dtype_bytes(L0.a_dtype);
+      cp.pack_src = a0;
+      cp.pack_dst = ws + L0.pack_off;
+      cp.pack_rows = L0.M;
+      cp.pack_src_pitch = L0.a_pitch * esz0;
+      cp.pack_dst_pitch = L0.pack_pitch * esz0;
+    }
+    const bool rebuild = !c.chain_tmaps_valid || (!L0.need_pack && c.chain_a0_ptr != a0);
+    if (rebuild) c.chain_tmaps.assign(2 * CHAIN_MAX_LAYERS, CUtensorMap());
+    for (size_t l = 0; l < c.layers.size(); ++l) {
+      const LayerPlan& L = c.layers[l];
+      const int esz = dtype_bytes(L.a_dtype);
+      ChainLayer& cl = cp.L[l];
+      const void* A = l == 0 ? (L.need_pack ? static_cast<const void*>(ws + L.pack_off) : a0)
+                             : static_cast<const void*>(ws + L.in_off);
+      const int64_t a_pitch = (l == 0 && L.need_pack) ? L.pack_pitch : L.a_pitch;
+      cl.M = L.M;
+      cl.N = L.N;
+      cl.K = L.K;
+      cl.nkb = L.nkb;
+      cl.active_ctas = L.use_tc ? (L.N + 31) / 32 : 0;
+      cl.a_tm = static_cast<int>(2 * l);
+      cl.b_tm = static_cast<int>(2 * l + 1);
+      cl.w_smem_off = c.chain_w_off[l];
+      cl.a_ptr = A;
+      cl.wt_ptr = ws + L.wt_off;
+      cl.a_pitch = a_pitch;
+      cl.w_pitch = L.Kp;
+      cl.a_dtype = L.a_dtype;
+      cl.w_dtype = L.w_dtype;
+      cl.a_zp = L.a_zp;
+      cl.out = L.out_pos >= 0 ? out[L.out_pos] : static_cast<void*>(ws + L.out_off);
+      cl.out_pitch = L.out_pitch;
+      cl.out_elem = L.out_elem;
+      cl.epi = L.epi;
+      cl.epi.bias = L.bias_input >= 0 ? static_cast<const float*>(in[L.bias_input]) : nullptr;
+      if (L.use_tc) {
+        const uint32_t afmt = L.a_dtype == GC_S8 ? 1u : 0u;
+        cl.idesc = L.kind == 0   ? ((2u << 4) | (afmt << 7) | (1u << 10) | ((32u >> 3) << 17) | ((128u >> 4) << 24))
+                   : L.kind == 1 ? ((1u << 4) | (1u << 7) | (1u << 10) | ((32u >> 3) << 17) | ((128u >> 4) << 24))
+                                 : ((1u << 4) | (2u << 7) | (2u << 10) | ((32u >> 3) << 17) | ((128u >> 4) << 24));
+        if (rebuild) {
+          const int k_elems = 128 / esz;
+          gc_status_t s = make_tmap(&c.chain_tmaps[2 * l], A, L.a_dtype, L.K, L.M, a_pitch * esz, k_elems, c.chain_a_rows, 128);
+          if (s != GC_OK) return s;
+          s = make_tmap(&c.chain_tmaps[2 * l + 1], ws + L.wt_off, L.w_dtype, L.Kp, L.N, static_cast<uint64_t>(L.Kp) * esz,
+                        k_elems, 32, 128);
+          if (s != GC_OK) return s;
+        }
+      }
+    }
+    if (rebuild) {
+      c.chain_tmaps_valid = true;
+      c.chain_a0_ptr = a0;
+    }
+    memcpy(cp.tmaps, c.chain_tmaps.data(), sizeof(cp.tmaps));
+    CUDA_TRY(launch_mlp_chain(c.chain_kind, cp, c.chain_grid, st));
+    c.chain_arrivals += static_cast<unsigned long long>(c.chain_barriers) * c.chain_grid;
+    return GC_OK;
   }
   for (size_t l = 0; l < c.layers.size(); ++l) {
     LayerPlan& L = c.layers[l];

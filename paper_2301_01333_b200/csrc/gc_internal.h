@@ -73,6 +73,43 @@ struct SdpaParams {
   uint32_t* status;
 };
 
+// One layer of the fused small-batch chain kernel (kernels_chain.cu).
+constexpr int CHAIN_MAX_LAYERS = 8;
+struct ChainLayer {
+  int M, N, K, nkb;        // nkb: 128-byte blocks along the reduction axis
+  int active_ctas;         // CTAs that own 32 output columns each; 0 = this layer runs on CUDA cores
+  int a_tm, b_tm;          // indices into ChainParams::tmaps (A operand, prepacked weight)
+  uint32_t idesc;          // tcgen05 instruction descriptor
+  uint32_t w_smem_off;     // where this layer's weight slice lives in shared memory
+  const void* a_ptr;       // CUDA-core layers: activation and prepacked weight in global memory
+  const void* wt_ptr;
+  int64_t a_pitch, w_pitch;
+  int a_dtype, w_dtype, a_zp;
+  void* out;
+  int64_t out_pitch;       // elements
+  int out_elem;            // bytes per stored element
+  Epilogue epi;
+};
+struct ChainParams {
+  int n_layers;
+  ChainLayer L[CHAIN_MAX_LAYERS];
+  uint32_t w_smem_bytes;   // shared memory taken by the resident weight slices
+  int a_stages;            // A-operand ring: stages and bytes per stage (round_up(M, 8) rows of 128 bytes)
+  int a_stage_bytes;
+  const void* pack_src;    // graph-entry reorder (pack_rows == 0: none)
+  void* pack_dst;
+  int pack_rows;
+  int64_t pack_src_pitch, pack_dst_pitch;   // bytes
+  unsigned long long* barrier;              // grid-barrier counter (only grows)
+  unsigned long long barrier_base;          // its value before this launch
+  uint32_t* status;
+  // TMA descriptors travel in the kernel parameter space (fetched once, cached by the TMA unit); descriptors
+  // kept in global memory cost a fetch of several hundred clocks on every load instruction.
+  alignas(64) CUtensorMap tmaps[2 * CHAIN_MAX_LAYERS];
+};
+size_t mlp_chain_smem_bytes(size_t w_smem_bytes, int a_stages, int a_stage_bytes);
+cudaError_t launch_mlp_chain(int kind, const ChainParams& p, int grid, cudaStream_t s);
+
 // ---- launchers (each enqueues exactly one kernel on the stream and returns cudaGetLastError) ----
 cudaError_t launch_pack_rows(const void* src, void* dst, int rows, int64_t src_pitch_bytes, int64_t dst_pitch_bytes,
                              cudaStream_t s);

@@ -1,0 +1,306 @@
+// One persistent kernel for a whole small-batch MLP chain (the analogue of the paper's coarse-grain fusion,
+// Section V: the outer loops of consecutive fused ops merged so that activations stay in the fastest cache
+// and the per-op synchronisation overhead disappears; Section VII: 2.0x on the int8 MLP-1).
+//
+// Shape of the problem: M <= 128 rows (one MMA row tile), L layers with N_l output columns.  CTA c owns
+// output columns [32 c, 32 c + 32) of every tensor-core layer that has that many columns:
+//   * at kernel start it TMA-loads its 32-row slice of EVERY layer's prepacked weight into shared memory
+//     (HBM latency is paid once, not once per layer);
+//   * per layer it fetches the layer's A operand (the previous activation, L2-resident) with as many
+//     k-blocks in flight as shared memory allows - normally all of them, so the L2 latency is paid once per
+//     layer -, issues tcgen05.mma into a 32-column TMEM accumulator, applies the post-ops and stores its
+//     32 columns of the next activation.  A stage holds only round_up(M, 8) rows; the MMA still reads 128
+//     rows, the surplus rows come from whatever follows in shared memory and only feed accumulator rows
+//     that are never stored (rows of a matmul are independent);
+//   * a grid-wide barrier (epoch-counted atomic in global memory, bounded spin) separates the layers;
+//   * layers the tensor-core path does not take (N not a multiple of 16, e.g. the 256 -> 1 tail) run on
+//     CUDA cores inside the same kernel, one warp per output;
+//   * an input whose row pitch TMA cannot address is first copied to a padded buffer by all threads.
+// At most one CTA per SM (<= 148 CTAs of 192 threads), so all CTAs of the grid are resident together.
+#include <cuda_bf16.h>
+
+#include "epilogue.cuh"
+#include "gc_internal.h"
+#include "ptx.cuh"
+
+namespace gc {
+
+constexpr int CH_THREADS = 192;          // warp 0 producer, warp 1 MMA, warps 2-5 epilogue
+constexpr int CH_MAX_STAGES = 32;
+constexpr int CH_BLOCK_N = 32;
+// Consecutive MMAs into one accumulator form a dependent chain of roughly 130 clocks per instruction however
+// narrow the tile is, so the four 32-byte k-steps of a k-block go to four independent 32-column accumulators
+// that the epilogue adds up (exact for s32; a fixed summation order for fp32).
+constexpr int CH_NACC = 4;
+
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// Grid-wide barrier: every CTA adds one to a counter that only grows; the caller passes the value the
+// counter reaches when all CTAs of this launch have arrived at this barrier.  Bounded: gives up after 2 s.
+__device__ __forceinline__ bool grid_barrier(unsigned long long* ctr, unsigned long long target) {
+  __syncthreads();
+  int ok = 1;
+  if (threadIdx.x == 0) {
+    asm volatile("fence.proxy.async;" ::: "memory");   // async-proxy (TMA) accesses vs. generic stores
+    __threadfence();
+    atomicAdd(ctr, 1ULL);
+    const uint64_t t0 = globaltimer_ns();
+    uint32_t i = 0;
+    while (ld_acquire_u64(ctr) < target) {
+      if ((++i & 1023u) == 0 && globaltimer_ns() - t0 > 2000000000ull) {
+        ok = 0;
+        break;
+      }
+    }
+    asm volatile("fence.proxy.async;" ::: "memory");
+  }
+  return __syncthreads_and(ok) != 0;
+}
+
+__device__ __forceinline__ float ch_load_f(const void* p, int64_t i, int dtype) {
+  if (dtype == GC_F32) return static_cast<const float*>(p)[i];
+  return __bfloat162float(static_cast<const __nv_bfloat16*>(p)[i]);
+}
+__device__ __forceinline__ int ch_load_i(const void* p, int64_t i, int dtype) {
+  if (dtype == GC_U8) return static_cast<const uint8_t*>(p)[i];
+  return static_cast<const int8_t*>(p)[i];
+}
+
+template <int KIND>
+__global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_constant__ ChainParams p) {
+  constexpr int K_ELEMS = KIND == KIND_I8 ? 128 : (KIND == KIND_BF16 ? 64 : 32);
+  constexpr int ESZ = KIND == KIND_I8 ? 1 : (KIND == KIND_BF16 ? 2 : 4);
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int CH_STAGES = p.a_stages;
+  const int CH_A_STAGE_BYTES = p.a_stage_bytes;
+  uint8_t* sA = smem;                                             // a_stages x a_stage_bytes
+  // the weight slices (padded to at least 16 KB) follow the ring, so the 128-row MMA reads of the last stages
+  // stay inside this CTA's shared memory
+  uint8_t* sW = sA + ((CH_STAGES * CH_A_STAGE_BYTES + 1023) & ~1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sW + (p.w_smem_bytes < 16384u ? 16384u : p.w_smem_bytes));
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * CH_MAX_STAGES + 1 + CHAIN_MAX_LAYERS);
+  const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * CH_MAX_STAGES;
+  const uint32_t bar_tfull = bar_empty + 8 * CH_MAX_STAGES;       // [1]
+  const uint32_t bar_wfull = bar_tfull + 8;                       // [CHAIN_MAX_LAYERS]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int cta = blockIdx.x;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < CH_STAGES; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    mbar_init(bar_tfull, 1);
+    for (int l = 0; l < CHAIN_MAX_LAYERS; ++l) mbar_init(bar_wfull + 8 * l, 1);
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_slot), CH_NACC * CH_BLOCK_N);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  // every layer's weight slice starts moving now (constants: they do not depend on earlier layers)
+  if (warp == 0 && lane == 0) {
+    for (int l = 0; l < p.n_layers; ++l) {
+      const ChainLayer& L = p.L[l];
+      if (L.active_ctas == 0 || cta >= L.active_ctas) continue;
+      mbar_arrive_expect_tx(bar_wfull + 8 * l, static_cast<uint32_t>(L.nkb) * (CH_BLOCK_N * 128));
+      for (int kb = 0; kb < L.nkb; ++kb)
+        tma_load_2d(smem_u32(sW) + L.w_smem_off + kb * (CH_BLOCK_N * 128), p.tmaps + L.b_tm, kb * K_ELEMS,
+                    cta * CH_BLOCK_N, bar_wfull + 8 * l);
+    }
+  }
+
+  bool failed = false;
+  unsigned long long bar_count = p.barrier_base;                  // counter value before this launch
+  auto next_barrier = [&]() {
+    bar_count += gridDim.x;
+    if (!grid_barrier(p.barrier, bar_count)) {
+      failed = true;
+      report(p.status, DEV_TIMEOUT_OTHER);
+    }
+  };
+
+  // graph-entry reorder: copy the input into a buffer whose row pitch TMA can address
+  if (p.pack_rows > 0) {
+    const int64_t words_per_row = p.pack_dst_pitch / 4;
+    const int64_t total = static_cast<int64_t>(p.pack_rows) * words_per_row;
+    const uint8_t* src = static_cast<const uint8_t*>(p.pack_src);
+    uint8_t* dst = static_cast<uint8_t*>(p.pack_dst);
+    for (int64_t i = static_cast<int64_t>(cta) * CH_THREADS + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * CH_THREADS) {
+      const int64_t r = i / words_per_row, c = (i % words_per_row) * 4;
+      uint32_t w = 0;
+#pragma unroll
+      for (int b = 0; b < 4; ++b)
+        if (c + b < p.pack_src_pitch) w |= static_cast<uint32_t>(src[r * p.pack_src_pitch + c + b]) << (8 * b);
+      *reinterpret_cast<uint32_t*>(dst + r * p.pack_dst_pitch + c) = w;
+    }
+    next_barrier();
+  }
+
+  int stage = 0;                 // ring position, shared by construction between producer and MMA thread
+  uint32_t phase = 0;
+  uint32_t tphase = 0;           // parity of the accumulator-ready barrier (one completion per active layer)
+  for (int l = 0; l < p.n_layers && !failed; ++l) {
+    // A by-value copy: fields read through a reference into the parameter space are re-fetched around every
+    // store (possible aliasing) at a few hundred clocks each, which made a 16-element epilogue cost thousands.
+    const ChainLayer L = p.L[l];
+    if (L.active_ctas > 0) {
+      if (cta < L.active_ctas) {
+        if (warp == 0) {
+          if (lane == 0) {
+            asm volatile("fence.proxy.async;" ::: "memory");     // activations were written with generic stores
+            // a_stages >= nkb (planner): a stage is never reused within a layer, and between layers the
+            // accumulator-ready commit plus the grid barrier guarantee that every MMA has read its stage
+            for (int kb = 0; kb < L.nkb; ++kb) {
+              mbar_arrive_expect_tx(bar_full + 8 * stage, CH_A_STAGE_BYTES);
+              tma_load_2d(smem_u32(sA) + stage * CH_A_STAGE_BYTES, p.tmaps + L.a_tm, kb * K_ELEMS, 0, bar_full + 8 * stage);
+              if (++stage == CH_STAGES) {
+                stage = 0;
+                phase ^= 1;
+              }
+            }
+          }
+        } else if (warp == 1) {
+          if (lane == 0) {
+            bool ok = mbar_wait(bar_wfull + 8 * l, 0);
+            const uint32_t idesc = L.idesc;
+            const int nkb = L.nkb;
+            const uint64_t a_desc0 = make_smem_desc(smem_u32(sA), 16, 1024, SWZ_128B);
+            uint64_t b_desc = make_smem_desc(smem_u32(sW) + L.w_smem_off, 16, 1024, SWZ_128B);
+            const uint32_t a_step = static_cast<uint32_t>(CH_A_STAGE_BYTES) >> 4;   // descriptor address units of 16 bytes
+            for (int kb = 0; kb < nkb && ok; ++kb, b_desc += (CH_BLOCK_N * 128) >> 4) {
+              ok = mbar_wait(bar_full + 8 * stage, phase);
+              if (!ok) break;
+              tc_fence_after();
+              const uint64_t a_desc = a_desc0 + static_cast<uint64_t>(stage) * a_step;
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                umma_ss<KIND>(tmem_base + k * CH_BLOCK_N, a_desc + 2 * k, b_desc + 2 * k, idesc, kb != 0);
+              if (++stage == CH_STAGES) {
+                stage = 0;
+                phase ^= 1;
+              }
+            }
+            if (ok) umma_commit(bar_tfull);
+            else report(p.status, DEV_TIMEOUT_MMA);
+          }
+        } else {
+          const int q = warp & 3;
+          if (mbar_wait(bar_tfull, tphase)) {
+            tc_fence_after();
+            uint32_t r[32];
+            {
+              uint32_t r1[32], r2[32], r3[32];
+              const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+              tmem_ld32(t_row, r);
+              tmem_ld32(t_row + CH_BLOCK_N, r1);
+              tmem_ld32(t_row + 2 * CH_BLOCK_N, r2);
+              tmem_ld32(t_row + 3 * CH_BLOCK_N, r3);
+              tmem_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) {
+                if constexpr (KIND == KIND_I8)
+                  r[i] = (r[i] + r1[i]) + (r2[i] + r3[i]);
+                else
+                  r[i] = __float_as_uint((__uint_as_float(r[i]) + __uint_as_float(r1[i])) +
+                                         (__uint_as_float(r2[i]) + __uint_as_float(r3[i])));
+              }
+            }
+            tc_fence_before();
+            const int row = q * 32 + lane;
+            const int n0 = cta * CH_BLOCK_N;
+            if (row < L.M) {
+              char* dst_row = static_cast<char*>(L.out) + static_cast<int64_t>(row) * L.out_pitch * L.out_elem;
+              if (n0 < L.N) epi_store16(r, dst_row, n0, L.epi);
+              if (n0 + 16 < L.N) epi_store16(r + 16, dst_row, n0 + 16, L.epi);
+            }
+          } else {
+            report(p.status, DEV_TIMEOUT_EPILOGUE);
+          }
+        }
+        // the ring position advances identically in the threads that did not walk it
+        if (!(warp <= 1 && lane == 0)) {
+          const int adv = L.nkb;
+          const int pos = stage + adv;
+          phase ^= (pos / CH_STAGES) & 1;
+          stage = pos % CH_STAGES;
+        }
+        tphase ^= 1;
+      }
+    } else {
+      // CUDA-core layer: one warp per output element, lanes stride the reduction axis
+      const int64_t outputs = static_cast<int64_t>(L.M) * L.N;
+      for (int64_t o = static_cast<int64_t>(cta) * (CH_THREADS / 32) + warp; o < outputs;
+           o += static_cast<int64_t>(gridDim.x) * (CH_THREADS / 32)) {
+        const int m = static_cast<int>(o / L.N), n = static_cast<int>(o % L.N);
+        const char* A = static_cast<const char*>(L.a_ptr) + static_cast<int64_t>(m) * L.a_pitch * ESZ;
+        const char* Wt = static_cast<const char*>(L.wt_ptr) + static_cast<int64_t>(n) * L.w_pitch * ESZ;
+        uint32_t raw;
+        if (L.epi.acc_is_int) {
+          int acc = 0;
+          for (int k = lane; k < L.K; k += 32) acc += (ch_load_i(A, k, L.a_dtype) - L.a_zp) * ch_load_i(Wt, k, L.w_dtype);
+#pragma unroll
+          for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+          raw = static_cast<uint32_t>(acc);
+        } else {
+          float acc = 0.f;
+          for (int k = lane; k < L.K; k += 32) acc = fmaf(ch_load_f(A, k, L.a_dtype), ch_load_f(Wt, k, L.w_dtype), acc);
+#pragma unroll
+          for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+          raw = __float_as_uint(acc);
+        }
+        if (lane == 0) {
+          char* row = static_cast<char*>(L.out) + static_cast<int64_t>(m) * L.out_pitch * L.out_elem;
+          epi_store1(raw, row, n, L.epi);
+        }
+      }
+    }
+    if (l + 1 < p.n_layers) next_barrier();
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, CH_NACC * CH_BLOCK_N);
+  }
+}
+
+size_t mlp_chain_smem_bytes(size_t w_smem_bytes, int a_stages, int a_stage_bytes) {
+  return ((static_cast<size_t>(a_stages) * a_stage_bytes + 1023) & ~size_t(1023)) +
+         (w_smem_bytes < 16384 ? size_t(16384) : w_smem_bytes) + 1024 + 1024;
+}
+
+cudaError_t launch_mlp_chain(int kind, const ChainParams& p, int grid, cudaStream_t s) {
+  const size_t smem = mlp_chain_smem_bytes(p.w_smem_bytes, p.a_stages, p.a_stage_bytes);
+  void* kern = kind == KIND_I8 ? reinterpret_cast<void*>(mlp_chain_kernel<KIND_I8>)
+               : kind == KIND_BF16 ? reinterpret_cast<void*>(mlp_chain_kernel<KIND_BF16>)
+                                   : reinterpret_cast<void*>(mlp_chain_kernel<KIND_TF32>);
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(CH_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  // No cooperative-launch attribute: it costs tens of microseconds per launch, more than the whole chain.
+  // The grid is at most one CTA per SM, so its CTAs become resident together whenever the SMs are free; if
+  // they are not, the waiting CTAs only wait for unrelated work to finish, and every spin is bounded anyway.
+  cfg.attrs = nullptr;
+  cfg.numAttrs = 0;
+  void* args[] = {const_cast<ChainParams*>(&p)};
+  return cudaLaunchKernelExC(&cfg, kern, args);
+}
+
+}  // namespace gc
