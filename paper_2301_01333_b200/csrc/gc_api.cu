@@ -960,7 +960,7 @@ static gc_status_t run_sdpa(gc_compiled& c, cudaStream_t st, const void* const* 
     s.v_ptr = prm.V;
   }
   if (s.o_ptr != prm.O) {
-    gc_status_t r = make_tmap(&s.tmO, prm.O, dt, prm.D, rows, static_cast<uint64_t>(prm.D) * esz, 16, 32, 0);
+    gc_status_t r = make_tmap(&s.tmO, prm.O, dt, prm.D, rows, static_cast<uint64_t>(prm.D) * esz, prm.D, 32, prm.D * esz);
     if (r != GC_OK) return r;
     s.o_ptr = prm.O;
   }

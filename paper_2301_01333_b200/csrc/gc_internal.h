@@ -136,7 +136,7 @@ cudaError_t launch_gemm_tc2(int kind, int a_signed, const CUtensorMap& tmA, cons
                             const GemmTcParams& p, int grid, bool pdl, cudaStream_t s);
 
 size_t sdpa_tc_smem_bytes(int S, int is_int8);
-// tmO: output [B*H*S, 64] with a [32 rows x 16 columns] box, no swizzle
+// tmO: output [B*H*S, 64] with a [32 rows x 64 columns] box, swizzle = row bytes (64 for 8-bit, 128 for bf16)
 cudaError_t launch_sdpa_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmO,
                            const SdpaParams& p, int num_sms, cudaStream_t s);
 

@@ -1,15 +1,17 @@
 // Fused scaled-dot-product attention on tcgen05 (Section VII "MHA": two batch matmuls with the softmax and
 // the binary ops between them fused after the first one; the two matmul loop nests merged).
 //
-// Persistent CTAs (one per SM, 640 threads) walk over work units (batch, head, 128-query tile):
+// Persistent CTAs (one per SM, 704 threads) walk over work units (batch, head, 128-query tile):
 //   warp 0      TMA producer: Q tile, all K rows and all V rows of the unit into one of two shared-memory
 //               slots (128B / 64B swizzle), one unit ahead of the math (no multicast)
 //   warp 1      MMA issuer (one thread): S = Q K^T in 128-key blocks into tensor memory, O = P V in 128-key
 //               blocks as soon as each P block is ready.  When two score buffers fit in tensor memory
 //               (S = 128) the next unit's S is issued a whole unit early; otherwise its blocks are issued as
 //               soon as the softmax warps release the corresponding TMEM columns
-//   warps 2-3   per-unit preparation: u8 -> s8 flip of Q (int8 path), mask row scaled by log2(e)
-//   warps 4-19  softmax: four threads per query row (TMEM lane), each owning 32 of every 128 key columns.
+//   warps 2-5   per-unit preparation (u8 -> s8 flip of Q on the int8 path, mask row scaled by log2(e)) and the
+//               epilogue of the previous unit: O out of tensor memory, deferred normalisation (bf16) or
+//               dequantize/requantize (int8), swizzled staging, one TMA store per 32 rows
+//   warps 6-21  softmax: four threads per query row (TMEM lane), each owning 32 of every 128 key columns.
 //               Pass A: scale + mask, running row max, exp2 and running row sum (int8: the exponentials
 //               are written back to tensor memory); the four threads of a row combine their statistics;
 //               Pass B: normalise, quantise to u8 (int8) or cast to bf16, write P to shared memory as the
@@ -37,7 +39,7 @@ namespace gc {
 
 constexpr int SDPA_D = 64;
 constexpr int SDPA_BLOCK_Q = 128;
-constexpr int SDPA_THREADS = 640;
+constexpr int SDPA_THREADS = 704;
 constexpr int SDPA_SOFTMAX_WARPS = 16;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float MAGIC_F = 12582912.0f;          // 1.5 * 2^23
@@ -47,7 +49,7 @@ template <bool INT8>
 struct SdpaSmem {
   static constexpr int ESZ = INT8 ? 1 : 2;
   static constexpr int ROW_BYTES = SDPA_D * ESZ;               // 64 (SW64) or 128 (SW128)
-  static constexpr int OUT_STAGING_BYTES = SDPA_SOFTMAX_WARPS * 1024;   // per softmax warp: 32 rows x <= 32 bytes
+  static constexpr int OUT_STAGING_BYTES = 4 * 4096;           // per auxiliary warp: 32 rows x <= 128 bytes
   __host__ __device__ static constexpr int q_bytes() { return SDPA_BLOCK_Q * ROW_BYTES; }
   __host__ __device__ static constexpr int kv_bytes(int S) { return S * ROW_BYTES; }
   // P: per 128-key block, 128 rows x (128 keys * ESZ) bytes = 16 KB (int8) or 32 KB (bf16)
@@ -118,15 +120,16 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sSlots = smem;
   uint8_t* sPall = sSlots + slots * L::slot_bytes(S);
-  uint8_t* sOut = sPall + nsb * L::p_bytes(S);                            // output staging, 2 KB per softmax warp
+  uint8_t* sOut = sPall + nsb * L::p_bytes(S);                            // output staging, 4 KB per auxiliary warp
   float* sMask = reinterpret_cast<float*>(sOut + (stage_out ? L::OUT_STAGING_BYTES : 0));   // [slots][S]
   float* sStat = sMask + slots * S;                                       // [3 kinds][2 parities][4 groups][128]
   uint64_t* bars = reinterpret_cast<uint64_t*>(sStat + 24 * 128);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 24);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 26);
   const uint32_t b0 = smem_u32(bars);
   const uint32_t bar_kv_full = b0, bar_kv_empty = b0 + 16, bar_kv_ready = b0 + 32;   // [2] each
   const uint32_t bar_s_full = b0 + 48, bar_s_free = b0 + 72, bar_p_full = b0 + 96;   // [3] each
   const uint32_t bar_o_full = b0 + 120, bar_o_free = b0 + 136, bar_xchg = b0 + 152;  // [2], [2], [1]
+  const uint32_t bar_st_ready = b0 + 160, bar_st_free = b0 + 176;                    // [2], [2]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int q_tiles = S / SDPA_BLOCK_Q;
@@ -136,9 +139,11 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_kv_full + 8 * i, 1);
       mbar_init(bar_kv_empty + 8 * i, 1);
-      mbar_init(bar_kv_ready + 8 * i, 2);
+      mbar_init(bar_kv_ready + 8 * i, 4);
       mbar_init(bar_o_full + 8 * i, 1);
-      mbar_init(bar_o_free + 8 * i, SDPA_SOFTMAX_WARPS);
+      mbar_init(bar_o_free + 8 * i, 4);
+      mbar_init(bar_st_ready + 8 * i, SDPA_SOFTMAX_WARPS);
+      mbar_init(bar_st_free + 8 * i, 4);
     }
     for (int i = 0; i < 3; ++i) {
       mbar_init(bar_s_full + 8 * i, 1);
@@ -276,11 +281,111 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       }
       if (failed) report(p.status, DEV_TIMEOUT_MMA);
     }
-  } else if (warp < 4) {
-    // ------------------------------------------------------------------ per-unit preparation
-    const int t = tid - 64;                                     // 0..63
+  } else if (warp < 6) {
+    // ------------------------------------------------------------------ auxiliary warps
+    // Per unit: (1) preparation of the inputs that have just landed - mask row scaled by log2(e), u8 -> s8
+    // flip of Q on the int8 path; (2) epilogue of the previous unit - read O from tensor memory once its
+    // second MMA has completed, finish it with the row statistics the softmax warps left in shared memory,
+    // stage it and hand it to a TMA store.  This keeps the whole epilogue off the softmax warps' critical path.
+    const int t = tid - 64;                                     // 0..127
+    const int aw = warp - 2;                                    // staging buffer index
+    const int q = warp & 3;                                     // TMEM lane quarter this warp may access
+    const int r = q * 32 + lane;                                // query row within the tile
+    const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+    constexpr int OUT_ROW_BYTES = SDPA_D * L::ESZ;              // 64 (int8) or 128 (bf16)
+    uint8_t* my_out = sOut + aw * 4096;
+    auto stat2 = [&](int par, int grp) { return sStat + ((2 * 2 + par) * 4 + grp) * 128 + r; };
+
+    auto epilogue = [&](int unit, int n0) -> bool {
+      const int buf = buf_of(n0), par = n0 & 1;
+      if (!mbar_wait(bar_st_ready + 8 * par, (n0 >> 1) & 1)) return false;
+      float total;
+      if constexpr (INT8) {
+        int ti = 0;
+#pragma unroll
+        for (int o = 0; o < 4; ++o) ti += __float_as_int(*stat2(par, o));
+        total = __int_as_float(ti);
+      } else {
+        total = 0.f;
+#pragma unroll
+        for (int o = 0; o < 4; ++o) total += *stat2(par, o);
+      }
+      if (!mbar_wait(bar_o_full + 8 * buf, cnt_of(n0) & 1)) return false;
+      tc_fence_after();
+      uint32_t v[64];
+      {
+        uint32_t (&v0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&v[0]);
+        uint32_t (&v1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&v[32]);
+        tmem_ld32(t_lane + buf * BUF_COLS + S, v0);
+        tmem_ld32(t_lane + buf * BUF_COLS + S + 32, v1);
+      }
+      tmem_wait_ld();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(bar_o_free + 8 * buf);
+        mbar_arrive(bar_st_free + 8 * par);
+        if (stage_out) tma_store_wait_read<0>();                // the previous store has read the staging buffer
+      }
+      __syncwarp();
+      const int bh = unit / q_tiles, qt = unit % q_tiles;
+      const int64_t grow = static_cast<int64_t>(bh) * S + qt * SDPA_BLOCK_Q + r;
+      uint8_t* dst_direct = static_cast<uint8_t*>(p.O) + grow * OUT_ROW_BYTES;
+      if constexpr (INT8) {
+        const int lo = p.out_dtype == GC_U8 ? 0 : -128, hi = p.out_dtype == GC_U8 ? 255 : 127;
+        const int corr = p.zp_v * __float_as_int(total);       // zero point of V times the row sum of P
+        // saturate(rne(u) + zp) = rne(clamp(u, lo - zp, hi - zp)) + zp: clamp in float, round with the bias
+        // trick, and fold "- bias bits + zp" into one integer add; the code is the low byte of the result
+        const float u_lo = static_cast<float>(lo - p.zp_o), u_hi = static_cast<float>(hi - p.zp_o);
+        const int kadd = p.zp_o - MAGIC_I;
+        uint32_t w[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          uint32_t y[4];
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const int acc = static_cast<int>(v[4 * i + k]) - corr;
+            const float tt = __fmul_rn(__int2float_rn(acc), p.dq2);
+            const float u = fminf(fmaxf(__fmul_rn(tt, p.inv_o), u_lo), u_hi);
+            y[k] = static_cast<uint32_t>(__float_as_int(u + MAGIC_F) + kadd);
+          }
+          w[i] = __byte_perm(__byte_perm(y[0], y[1], 0x0040), __byte_perm(y[2], y[3], 0x0040), 0x5410);
+        }
+        // 64-byte rows, 64B swizzle: 16-byte chunk c of row r goes to chunk c ^ ((r >> 1) & 3)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint8_t* dst = stage_out ? my_out + lane * OUT_ROW_BYTES + ((c ^ ((lane >> 1) & 3)) * 16) : dst_direct + c * 16;
+          *reinterpret_cast<uint4*>(dst) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+        }
+      } else {
+        const float rl = 1.0f / total;                         // deferred normalisation by the row sum
+        uint32_t w[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(v[2 * i]) * rl, __uint_as_float(v[2 * i + 1]) * rl);
+          w[i] = *reinterpret_cast<uint32_t*>(&hh);
+        }
+        // 128-byte rows, 128B swizzle: chunk c of row r goes to chunk c ^ (r & 7)
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          uint8_t* dst = stage_out ? my_out + lane * OUT_ROW_BYTES + ((c ^ (lane & 7)) * 16) : dst_direct + c * 16;
+          *reinterpret_cast<uint4*>(dst) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+        }
+      }
+      if (stage_out) {
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_2d(&tmO, 0, bh * S + qt * SDPA_BLOCK_Q + q * 32, smem_u32(my_out));
+          tma_store_commit();
+        }
+      }
+      return true;
+    };
+
     int n = 0;
-    for (int unit = blockIdx.x; unit < num_units; unit += gridDim.x, ++n) {
+    int prev_unit = -1;
+    for (int unit = blockIdx.x; unit < num_units && !failed; unit += gridDim.x, ++n) {
       const int s = n % slots;
       const int b = (unit / q_tiles) / p.H;
       float* mk = sMask + s * S;
@@ -291,10 +396,10 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         failed = true;
         break;
       }
-      for (int j = t; j < S; j += 64) mk[j] = p.mask ? __ldg(p.mask + static_cast<int64_t>(b) * S + j) * LOG2E : 0.0f;
+      for (int j = t; j < S; j += 128) mk[j] = p.mask ? __ldg(p.mask + static_cast<int64_t>(b) * S + j) * LOG2E : 0.0f;
       if (INT8 && !p.q_signed) {
         uint4* q4 = reinterpret_cast<uint4*>(slot_q(s));
-        for (int i = t; i < L::q_bytes() / 16; i += 64) {
+        for (int i = t; i < L::q_bytes() / 16; i += 128) {
           uint4 v = q4[i];
           v.x ^= 0x80808080u; v.y ^= 0x80808080u; v.z ^= 0x80808080u; v.w ^= 0x80808080u;
           q4[i] = v;
@@ -303,13 +408,24 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_kv_ready + 8 * s);
+      if (prev_unit >= 0 && !epilogue(prev_unit, n - 1)) {
+        report(p.status, DEV_TIMEOUT_OTHER);
+        failed = true;
+        break;
+      }
+      prev_unit = unit;
     }
+    if (!failed && prev_unit >= 0 && !epilogue(prev_unit, n - 1)) {
+      report(p.status, DEV_TIMEOUT_OTHER);
+      failed = true;
+    }
+    if (lane == 0) tma_store_wait_all<0>();
   } else {
     // ------------------------------------------------------------------ softmax warps
     // Four threads share a query row (TMEM lane): warp w covers lane quarter (w % 4) and, of every 128-key
-    // block, the 32 columns [32 g, 32 g + 32) with g = (w - 4) / 4.  Four warps per scheduler keep the
+    // block, the 32 columns [32 g, 32 g + 32) with g = (w - 6) / 4.  Four warps per scheduler keep the
     // TMEM / barrier / exp latencies of one warp hidden behind the others.
-    const int sw = warp - 4;                                    // 0..15
+    const int sw = warp - 6;                                    // 0..15
     const int q = warp & 3;                                     // TMEM lane quarter
     const int g = sw >> 2;                                      // which 32 of every 128 key columns
     const int r = q * 32 + lane;                                // query row within the tile = TMEM lane
@@ -317,11 +433,8 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     const float c2 = (INT8 ? __fmul_rn(p.dq1, p.scalar) : p.scalar) * LOG2E;
     const uint32_t row_off = (r >> 3) * 1024 + (r & 7) * 128;
     uint32_t xphase = 0;
-    // statistics exchanged between the four threads of a row: [kind][unit parity][group][row]
+    // statistics shared between the four threads of a row and the auxiliary warps: [kind][unit parity][group][row]
     auto stat = [&](int kind, int par, int grp) { return sStat + ((kind * 2 + par) * 4 + grp) * 128 + r; };
-    // this warp's staging buffer for the output tile: 32 rows x 16 columns, dense (no swizzle)
-    constexpr int OUT_ROW_BYTES = 16 * L::ESZ;                  // 16 (int8) or 32 (bf16)
-    uint8_t* my_out = sOut + sw * 1024;
 
     auto xchg_sync = [&]() -> bool {
       __syncwarp();
@@ -330,72 +443,8 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       xphase ^= 1;
       return ok;
     };
-    // epilogue of unit n0: my 16 of the 64 output columns
-    auto epilogue = [&](int unit, int n0, float stat_total) -> bool {
-      const int buf = buf_of(n0);
-      if (!mbar_wait(bar_o_full + 8 * buf, cnt_of(n0) & 1)) return false;
-      tc_fence_after();
-      uint32_t v[16];
-      tmem_ld16(t_lane + buf * BUF_COLS + S + g * 16, v);
-      tmem_wait_ld();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) {
-        mbar_arrive(bar_o_free + 8 * buf);
-        if (stage_out) tma_store_wait_read<0>();                // the previous store has read the staging buffer
-      }
-      __syncwarp();
-      const int bh = unit / q_tiles, qt = unit % q_tiles;
-      // without a staging buffer each thread stores its 16 columns of row `grow` directly
-      const int64_t grow = static_cast<int64_t>(bh) * S + qt * SDPA_BLOCK_Q + r;
-      if constexpr (INT8) {
-        const int lo = p.out_dtype == GC_U8 ? 0 : -128, hi = p.out_dtype == GC_U8 ? 255 : 127;
-        const int corr = p.zp_v * __float_as_int(stat_total);   // zero point of V times the row sum of P
-        // saturate(rne(u) + zp) = rne(clamp(u, lo - zp, hi - zp)) + zp: clamp in float, round with the bias
-        // trick, and fold "- bias bits + zp" into one integer add; the code is the low byte of the result
-        const float u_lo = static_cast<float>(lo - p.zp_o), u_hi = static_cast<float>(hi - p.zp_o);
-        const int kadd = p.zp_o - MAGIC_I;
-        uint32_t w[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          uint32_t y[4];
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const int acc = static_cast<int>(v[4 * i + k]) - corr;
-            const float t = __fmul_rn(__int2float_rn(acc), p.dq2);
-            const float u = fminf(fmaxf(__fmul_rn(t, p.inv_o), u_lo), u_hi);
-            y[k] = static_cast<uint32_t>(__float_as_int(u + MAGIC_F) + kadd);
-          }
-          w[i] = __byte_perm(__byte_perm(y[0], y[1], 0x0040), __byte_perm(y[2], y[3], 0x0040), 0x5410);
-        }
-        uint8_t* dst = stage_out ? my_out + lane * OUT_ROW_BYTES : static_cast<uint8_t*>(p.O) + grow * SDPA_D + g * 16;
-        *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
-      } else {
-        const float rl = 1.0f / stat_total;                     // deferred normalisation by the row sum
-        uint32_t w[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(v[2 * i]) * rl, __uint_as_float(v[2 * i + 1]) * rl);
-          w[i] = *reinterpret_cast<uint32_t*>(&hh);
-        }
-        uint8_t* dst = stage_out ? my_out + lane * OUT_ROW_BYTES
-                                 : reinterpret_cast<uint8_t*>(static_cast<__nv_bfloat16*>(p.O) + grow * SDPA_D + g * 16);
-        reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
-        reinterpret_cast<uint4*>(dst)[1] = make_uint4(w[4], w[5], w[6], w[7]);
-      }
-      if (stage_out) {
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) {
-          tma_store_2d(&tmO, g * 16, bh * S + qt * SDPA_BLOCK_Q + q * 32, smem_u32(my_out));
-          tma_store_commit();
-        }
-      }
-      return true;
-    };
 
     int n = 0;
-    int prev_unit = -1;
     for (int unit = blockIdx.x; unit < num_units && !failed; unit += gridDim.x, ++n) {
       const int s = n % slots, buf = buf_of(n);
       const float* mk = sMask + s * S;
@@ -469,23 +518,6 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         scale = p.inv_p / Lsum;
       }
 
-      // ---------------- epilogue of the previous unit (its second MMA has had a whole pass to finish);
-      // the other threads' parts of that unit's row sum became visible with the exchange above
-      if (prev_unit >= 0) {
-        float total;
-        if constexpr (INT8) {
-          int t = 0;
-#pragma unroll
-          for (int o = 0; o < 4; ++o) t += __float_as_int(*stat(2, upar ^ 1, o));
-          total = __int_as_float(t);
-        } else {
-          total = 0.f;
-#pragma unroll
-          for (int o = 0; o < 4; ++o) total += *stat(2, upar ^ 1, o);
-        }
-        if (!epilogue(prev_unit, n - 1, total)) { failed = true; break; }
-      }
-
       // ---------------- pass B: normalise, round, write P
       int psum = 0;
       float lsum = 0.f;
@@ -556,30 +588,13 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           mbar_arrive(bar_s_free + 8 * bx(buf, b));
         }
       }
-      // my part of the row sum; the other threads of the row read it after the next exchange
+      // my part of the row sum goes to the auxiliary warps, which finish and store the output; the slot is
+      // free once they have read the sums of the unit that used it two units ago
+      if (!mbar_wait(bar_st_free + 8 * upar, ((n >> 1) & 1) ^ 1)) { failed = true; break; }
       *stat(2, upar, g) = INT8 ? __int_as_float(psum) : lsum;
-      prev_unit = unit;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_st_ready + 8 * upar);
     }
-    if (!failed && prev_unit >= 0) {
-      if (!xchg_sync()) {
-        failed = true;
-      } else {
-        const int upar = (n - 1) & 1;
-        float total;
-        if constexpr (INT8) {
-          int t = 0;
-#pragma unroll
-          for (int o = 0; o < 4; ++o) t += __float_as_int(*stat(2, upar, o));
-          total = __int_as_float(t);
-        } else {
-          total = 0.f;
-#pragma unroll
-          for (int o = 0; o < 4; ++o) total += *stat(2, upar, o);
-        }
-        if (!epilogue(prev_unit, n - 1, total)) failed = true;
-      }
-    }
-    if (lane == 0) tma_store_wait_all<0>();
     if (failed) report(p.status, DEV_TIMEOUT_EPILOGUE);
   }
 
