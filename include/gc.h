@@ -20,7 +20,9 @@
  *   Attention   (Section VII "MHA": two batch matmuls, a softmax and the binary ops between):
  *       MatMul(Q, K, transpose_b) [-> Dequantize] [-> Mul(scalar)] [-> Add(mask)] -> SoftMax
  *           [-> Quantize | TypeCast] -> MatMul(P, V) [-> Dequantize -> Quantize | -> TypeCast]
- *     Q, K, V, O are [B,H,S,D] contiguous; mask is fp32 [B,1,1,S].
+ *     Q, K, V, O are [B,H,S,D] contiguous; mask is fp32 [B,1,1,S].  The tensor P that the second
+ *     MatMul consumes (u8 codes or bf16, [B,H,S,S]) may be listed as a second graph output; it is
+ *     then written out as well, which lets a caller verify the integer stage after the softmax exactly.
  *
  * Semantics of the ops (what an unfused, op-by-op evaluation gives, which the fused kernels must
  * reproduce):

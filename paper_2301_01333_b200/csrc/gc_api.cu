@@ -209,6 +209,7 @@ struct LayerPlan {
 struct SdpaPlan {
   SdpaParams prm = {};
   int q_input = -1, k_input = -1, v_input = -1, mask_input = -1, out_pos = 0;
+  int p_out_pos = -1;        // graph output position of the probabilities tensor, if it is an output too
   bool use_tc = false;
   CUtensorMap tmQ, tmK, tmV, tmO;
   const void *q_ptr = nullptr, *k_ptr = nullptr, *v_ptr = nullptr, *o_ptr = nullptr;
@@ -449,6 +450,7 @@ static gc_status_t match_sdpa(const gc_partition& p, gc_compiled& c) {
   if (!(i < p.ops.size() && p.ops[i].kind == GC_OP_MATMUL && p.ops[i].in[0] == t && !p.ops[i].transpose_b))
     return fail(GC_ERR_UNSUPPORTED, "attention: expected the P.V matmul");
   const auto* pt = p.lt(t);
+  const int64_t p_tensor = t;
   const auto* v = p.lt(p.ops[i].in[1]);
   s.v_input = p.input_pos(p.ops[i].in[1]);
   if (s.v_input < 0 || !same_dims(*v, *q) || (i8 ? !is_int8(v->dtype) : v->dtype != GC_BF16))
@@ -473,8 +475,12 @@ static gc_status_t match_sdpa(const gc_partition& p, gc_compiled& c) {
     prm.out_dtype = GC_BF16;
     t = p.ops[i++].out;
   }
-  if (i != p.ops.size() || p.out_ids.size() != 1 || p.output_pos(t) != 0)
+  // outputs: the attention result, optionally followed by the probabilities tensor (for inspection: it lets
+  // a caller check the integer stage after the softmax exactly, given the probabilities the kernel used)
+  if (i != p.ops.size() || p.output_pos(t) != 0 || p.out_ids.size() > 2 ||
+      (p.out_ids.size() == 2 && p.output_pos(p_tensor) != 1))
     return fail(GC_ERR_UNSUPPORTED, "attention: trailing ops or wrong outputs");
+  s.p_out_pos = p.out_ids.size() == 2 ? 1 : -1;
   return GC_OK;
 }
 
@@ -583,6 +589,7 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
     SdpaParams& s = c->sdpa.prm;
     bool tc = !c->opt.force_generic && s.D == 64 && s.S % 128 == 0 && s.S <= 384 &&
               sdpa_tc_smem_bytes(s.S, s.is_int8) <= static_cast<size_t>(prop.sharedMemPerBlockOptin);
+    if (!s.is_int8 && c->sdpa.p_out_pos >= 0) tc = false;   // the bf16 tcgen05 kernel never forms normalised P
     if (s.is_int8)
       // Q must be exactly centred (s8 / zero point 0, or u8 / zero point 128); a zero point on K only
       // shifts every score of a row by the same amount, which softmax cancels
@@ -935,6 +942,7 @@ static gc_status_t run_sdpa(gc_compiled& c, cudaStream_t st, const void* const* 
   prm.V = in[s.v_input];
   prm.mask = s.mask_input >= 0 ? static_cast<const float*>(in[s.mask_input]) : nullptr;
   prm.O = out[0];
+  prm.P_out = s.p_out_pos >= 0 ? out[s.p_out_pos] : nullptr;
   prm.status = reinterpret_cast<uint32_t*>(c.ws);
   if (!s.use_tc) {
     CUDA_TRY(launch_sdpa_simt(prm, st));

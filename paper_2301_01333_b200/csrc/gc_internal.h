@@ -57,6 +57,8 @@ struct SdpaParams {
   const void* V;
   const float* mask;   // [B, S_kv] or nullptr
   void* O;
+  void* P_out;         // optional second graph output: the probabilities as the second MatMul consumes them
+                       // (u8 codes or bf16), [B,H,S,S]; nullptr when not requested
   int B, H, S, D;
   int is_int8;         // u8/s8 operands (else bf16)
   int zp_q, zp_k, zp_v;

@@ -204,10 +204,15 @@ __global__ void sdpa_simt_kernel(const SdpaParams p) {
   const float rl = 1.0f / sum;
   for (int j = lane; j < S; j += 32) {
     const float pj = x[j] * rl;
-    if (p.p_is_quant)
-      x[j] = static_cast<float>(quantize_value(pj, p.inv_p, p.zp_p, 0, 255) - p.zp_p);
-    else
-      x[j] = __bfloat162float(__float2bfloat16_rn(pj));
+    if (p.p_is_quant) {
+      const int code = quantize_value(pj, p.inv_p, p.zp_p, 0, 255);
+      if (p.P_out) static_cast<uint8_t*>(p.P_out)[row * S + j] = static_cast<uint8_t>(code);
+      x[j] = static_cast<float>(code - p.zp_p);
+    } else {
+      const __nv_bfloat16 pb = __float2bfloat16_rn(pj);
+      if (p.P_out) static_cast<__nv_bfloat16*>(p.P_out)[row * S + j] = pb;
+      x[j] = __bfloat162float(pb);
+    }
   }
   __syncwarp();
   for (int d = lane; d < D; d += 32) {

@@ -543,6 +543,12 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           const int c0 = g * 2;                                 // 16-byte chunk index inside the 128-byte row
           *reinterpret_cast<uint4*>(blk + (((c0 + 0) ^ (r & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
           *reinterpret_cast<uint4*>(blk + (((c0 + 1) ^ (r & 7)) * 16)) = make_uint4(w[4], w[5], w[6], w[7]);
+          if (p.P_out) {                                          // optional output: the codes the second MMA consumes
+            const int64_t grow = static_cast<int64_t>(unit / q_tiles) * S + (unit % q_tiles) * SDPA_BLOCK_Q + r;
+            uint4* po = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.P_out) + grow * S + col);
+            po[0] = make_uint4(w[0], w[1], w[2], w[3]);
+            po[1] = make_uint4(w[4], w[5], w[6], w[7]);
+          }
         } else {
           if (NB > 1) {                                         // with one key block the scores are still in v[]
             tmem_ld32(t_row + col, v);

@@ -214,6 +214,61 @@ def test_mha_int8_reduced(B, b, h, s, d, generic):
     check_int8_attention(got, oracle(w))
 
 
+@pytest.mark.parametrize("generic", [False, True])
+def test_mha_int8_stages_around_the_softmax(B, generic):
+    """The fp32 softmax sits between two exact integer stages.  With the probabilities as a second output:
+    (a) the codes differ from the oracle's by at most one, rarely; (b) given the codes the kernel itself used,
+    the integer stage after the softmax (P.V, dequantize, requantize) is reproduced by the oracle bit for bit."""
+    import torch
+    from paper_2301_01333_b200.graph import Graph
+    w = W.mha_int8(batch=1, heads=3, seq=384, head_dim=64, seed=5)
+    g = w.graph
+    g.mark_output(w.info["p_quant"])
+    c = B.CompiledPartition(g, 0, force_generic=generic)
+    assert ("tcgen05" in c.plan) == (not generic)
+    ins = B.device_inputs(w)
+    outs = B.device_outputs(g)
+    c.execute(ins, outs)
+    c.query_status()
+    torch.cuda.synchronize()
+    o_gpu = B.output_to_numpy(g, g.outputs[0], outs[0]).copy()
+    p_gpu = B.output_to_numpy(g, g.outputs[1], outs[1]).copy()
+    c.close()
+    ref = interp.run(g, w.feeds)
+    dp = np.abs(p_gpu.astype(np.int64) - ref[g.outputs[1]])
+    assert dp.max() <= 1 and (dp != 0).mean() <= 1e-3
+    check_int8_attention(o_gpu, ref[g.outputs[0]])
+    # stage after the softmax alone, fed with the kernel's own codes
+    v_id = g.inputs[2]
+    g3 = Graph()
+    pin = g3.input("u8", g.tensors[g.outputs[1]].dims, scale=g.tensors[g.outputs[1]].scale, zero_point=0)
+    vin = g3.input("u8", g.tensors[v_id].dims, scale=g.tensors[v_id].scale, zero_point=g.tensors[v_id].zero_point)
+    a2 = g3.op("matmul", (pin, vin), g3.tensor("s32", g.tensors[g.outputs[0]].dims))
+    d2 = g3.op("dequantize", (a2,), g3.tensor("f32", g.tensors[g.outputs[0]].dims))
+    ot = g.tensors[g.outputs[0]]
+    g3.mark_output(g3.op("quantize", (d2,), g3.tensor("u8", ot.dims, scale=ot.scale, zero_point=ot.zero_point)))
+    exact = interp.run(g3, {pin: p_gpu, vin: w.feeds[v_id]})[g3.outputs[0]]
+    assert np.array_equal(o_gpu.astype(np.int64), exact)
+
+
+def test_mha_bf16_probabilities_output(B):
+    w = W.mha_bf16(batch=1, heads=2, seq=128, head_dim=64, seed=8)
+    g = w.graph
+    p_id = [op.output for op in g.ops if op.kind == "typecast"][0]
+    g.mark_output(p_id)
+    c = B.CompiledPartition(g, 0)
+    ins = B.device_inputs(w)
+    outs = B.device_outputs(g)
+    c.execute(ins, outs)
+    c.query_status()
+    p_gpu = bf16_to_f64(B.output_to_numpy(g, p_id, outs[1]))
+    o_gpu = bf16_to_f64(B.output_to_numpy(g, g.outputs[0], outs[0]))
+    c.close()
+    ref = interp.run(g, w.feeds)
+    assert np.abs(p_gpu - ref[p_id]).max() <= 4e-3 and np.abs(p_gpu.sum(-1) - 1.0).max() <= 2e-2
+    assert np.abs(o_gpu - ref[g.outputs[0]]).max() <= 2e-2
+
+
 def test_mha_int8_all_128_inputs_give_zero_point(B):
     w = W.mha_int8(batch=1, heads=2, seq=128, head_dim=64, all_value=128)
     got, _ = run_gpu(B, w)
