@@ -104,9 +104,9 @@ class ClockSampler:
 
 
 class Replica:
-    def __init__(self, B, w, seed_shift, device):
+    def __init__(self, B, w, seed_shift, device, **opts):
         import torch
-        self.c = B.CompiledPartition(w.graph, device)
+        self.c = B.CompiledPartition(w.graph, device, **opts)
         self.ins = B.device_inputs(w, device)
         if seed_shift:   # distinct activations per replica (weights may repeat: only addresses matter)
             for t, tid in zip(self.ins, w.graph.inputs):
@@ -120,14 +120,14 @@ class Replica:
         self.c.execute(self.ins, self.outs, stream)
 
 
-def time_config(B, name, steps, warmup, device, want_e2e=True):
-    """Returns dict with device-timed and end-to-end results for one config on this rank."""
+def time_config(B, name, steps, warmup, device, **opts):
+    """Builds the rotating replicas of one config (total footprint above the L2 size) and warms them up."""
     import torch
     w = W.CONFIGS[name]()
     stream = torch.cuda.current_stream(device).cuda_stream
-    first = Replica(B, w, 0, device)
+    first = Replica(B, w, 0, device, **opts)
     n_rep = int(min(64, max(2, -(-int(1.25 * L2_BYTES) // first.bytes))))
-    reps = [first] + [Replica(B, w, i + 1, device) for i in range(n_rep - 1)]
+    reps = [first] + [Replica(B, w, i + 1, device, **opts) for i in range(n_rep - 1)]
     for r in reps:                      # first call prepacks the constant weights: outside the timing
         r.step(stream)
     torch.cuda.synchronize(device)
@@ -150,6 +150,40 @@ def run_timed(reps, n_rep, steps, device, barrier):
     torch.cuda.synchronize(device)
     barrier()
     return e0.elapsed_time(e1)          # ms
+
+
+def launch_floor_us(B, device, steps=2000):
+    """Back-to-back launches of the smallest partition (a 16x16x16 matmul on one CTA): the per-launch cost that
+    bounds the small-batch configs from below however fast their kernels are."""
+    import torch
+    w = W.single_matmul("u8", "s8", 16, 16, 16)
+    r = Replica(B, w, 0, device)
+    stream = torch.cuda.current_stream(device).cuda_stream
+    for _ in range(20):
+        r.step(stream)
+    torch.cuda.synchronize(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        r.step(stream)
+    e1.record()
+    torch.cuda.synchronize(device)
+    n = r.c.launches
+    r.c.close()
+    return e0.elapsed_time(e1) * 1e3 / steps / max(n, 1)
+
+
+# exp2 evaluations per second of the special-function units: 16 per clock per SM (4 per sub-partition) x 148 SMs
+def exp_peak_per_s(sm_mhz):
+    return 148 * 16 * sm_mhz * 1e6
+
+
+def softmax_scores(w):
+    """Number of attention scores (one exponential each) of an attention workload, else 0."""
+    for op in w.graph.ops:
+        if op.kind == "softmax":
+            return int(np.prod(w.graph.tensors[op.inputs[0]].dims))
+    return 0
 
 
 def run_e2e(w, rep, steps, warmup, device):
@@ -280,6 +314,8 @@ def main():
     head = args.workload
     names = [head] if args.only else [head] + [n for n in W.CONFIGS if n != head]
     results = {}
+    floor_us = launch_floor_us(B, local) if rank == 0 else 0.0
+    sm_max_mhz = 1965.0
     clocks = None
     launches_total = 0
     e2e = None
@@ -314,6 +350,30 @@ def main():
             "roofline_frac_measured_peak": max(t_tensor_meas, t_hbm_meas) / (us * 1e-6),
             "roofline_frac_nominal_peak": max(t_tensor, w.bytes / (NOMINAL["hbm_gbs"] * 1e9)) / (us * 1e-6),
         }
+        res["launch_floor_us"] = floor_us * reps[0].c.launches
+        # warm: the same buffers every call, so weights and small activations stay in L2
+        warm_steps = max(20, steps // 4)
+        res["us_per_subgraph_warm"] = max_over_ranks(run_timed(reps[:1], 1, warm_steps, local, barrier)) * 1e3 / warm_steps
+        if name in ("c1", "c2") and not args.only:
+            # coarse-grain fusion ablation (Section VII, Fig. 8): the whole chain in one persistent launch, one
+            # launch per layer (fine-grain fusion only), and the CUDA-core kernels
+            abl = {"fused_chain": {"us_cold": us, "us_warm": res["us_per_subgraph_warm"], "launches": reps[0].c.launches}}
+            for label, opts in (("per_layer", {"no_chain_fusion": True}), ("cuda_core_per_layer", {"force_generic": True})):
+                _, areps, an = time_config(B, name, steps, args.warmup, local, **opts)
+                cold = max_over_ranks(run_timed(areps, an, steps, local, barrier)) * 1e3 / steps
+                warm = max_over_ranks(run_timed(areps[:1], 1, warm_steps, local, barrier)) * 1e3 / warm_steps
+                abl[label] = {"us_cold": cold, "us_warm": warm, "launches": areps[0].c.launches}
+                for r in areps:
+                    r.c.close()
+                del areps
+            res["ablation"] = abl
+        n_exp = softmax_scores(w)
+        if n_exp:
+            # attention: one exponential per score on the special-function units bounds the softmax from below
+            t_exp = n_exp / exp_peak_per_s(sm_max_mhz)
+            res["exp_bound_us"] = t_exp * 1e6
+            res["exp_bound_frac"] = t_exp / (us * 1e-6)
+            res["scores"] = n_exp
         if name == head:
             launches_total = steps * reps[0].c.launches
             e2e_s, h2d, d2h = run_e2e(w, reps[0], max(3, min(steps, 50)), args.warmup, local)
@@ -334,7 +394,16 @@ def main():
     hr = results[head]
     us = hr["us_per_subgraph"]
     n_launch = hr["launches_per_step"]
-    if hr["roofline_bound"] == "tensor":
+    if "exp_bound_us" in hr and hr["exp_bound_us"] > us * hr["roofline_frac_measured_peak"]:
+        # attention: neither DRAM nor the tensor pipe but the exponentials bound it
+        peak = exp_peak_per_s(sm_max_mhz) / 1e12
+        achieved = hr["scores"] / (us * 1e-6) / 1e12
+        roof = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "Texp/s", "frac": achieved / peak,
+                "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(head),
+                "peak_source": "derived: 148 SMs x 16 ex2 per clock x 1965 MHz (one exponential per attention score)",
+                "kernel": DOMINANT_KERNEL[head], "launches_per_step": n_launch, "avg_launch_us": us / n_launch,
+                "hbm_frac_measured_peak": hr["roofline_frac_measured_peak"]}
+    elif hr["roofline_bound"] == "tensor":
         peak = peaks.get(head_peak_key, 1590.0) * KIND_RATIO[head]
         achieved = head_w.ops / (us * 1e-6) / 1e12
         roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s" if "FLOP" in UNIT[head] else "TOP/s",
