@@ -23,7 +23,8 @@ Arithmetic domains
     its declared dtype).
 
 Constants derived from logical-tensor attributes are formed in fp32 exactly like this:
-    dq  = float32(scale_a) * float32(scale_b)         (scale of an s32 MatMul result)
+    dq  = float32(scale_a) * float32(scale_b)         (scale of an s32 MatMul result; with per-channel
+                                                       weight scales one such product per output column)
     inv = float32(1) / float32(scale_out)              (Quantize multiplies by the reciprocal)
 
 Parity pins: tests/test_oracle_pins.py (brute force with Python integers, closed forms, rounding
@@ -44,8 +45,11 @@ _INT_RANGE = {"u8": (0, 255), "s8": (-128, 127), "s32": (-(2 ** 31), 2 ** 31 - 1
 class Value:
     data: np.ndarray          # int64 | float32 | float64
     kind: str                 # "int" | "f32x" | "wide"
-    qscale: Optional[np.float32] = None   # for "int": scale that Dequantize applies
+    qscale: Optional[np.float32] = None   # for "int": scale that Dequantize applies; a per-channel weight
+                                          # carries a float32 vector and `qaxis`, a MatMul result of one a
+                                          # vector over its last axis
     zero_point: int = 0                   # for "int": offset that MatMul / Dequantize subtract
+    qaxis: int = -1                       # axis a vector-valued qscale runs along
 
 
 def _bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
@@ -72,8 +76,12 @@ def _round_to_bf16(x: np.ndarray) -> np.ndarray:
 def load_input(lt, arr) -> Value:
     """Wrap a host array as an oracle value according to its logical tensor."""
     if lt.dtype in ("u8", "s8", "s32"):
-        return Value(np.asarray(arr).astype(np.int64).reshape(lt.dims), "int",
-                     np.float32(lt.scale), int(lt.zero_point))
+        data = np.asarray(arr).astype(np.int64).reshape(lt.dims)
+        if getattr(lt, "channel_scales", None) is not None:
+            # per-channel weight scales (Section VII, the int8 scheme of the evaluation)
+            return Value(data, "int", np.asarray(lt.channel_scales, dtype=np.float32), int(lt.zero_point),
+                         int(lt.channel_axis) % len(lt.dims))
+        return Value(data, "int", np.float32(lt.scale), int(lt.zero_point))
     if lt.dtype == "bf16":
         return Value(_bf16_bits_to_f32(arr).reshape(lt.dims), "f32x")
     if lt.dtype == "f32":
@@ -100,6 +108,15 @@ def op_matmul(a: Value, b: Value, transpose_b: bool) -> Value:
         C = np.matmul(A, B)                       # int64, exact
         if C.size and (C.max() > 2 ** 31 - 1 or C.min() < -(2 ** 31)):
             raise OverflowError("int8 matmul result does not fit the s32 accumulator")
+        if np.ndim(a.qscale) != 0:
+            raise TypeError("per-channel scales are defined for the weight operand only")
+        if np.ndim(b.qscale) != 0:
+            # the scales must run along the weight's output-channel axis (n): the last axis of [.., k, n],
+            # the one before it when the weight is stored transposed
+            n_axis = b.data.ndim - (2 if transpose_b else 1)
+            if b.qaxis != n_axis:
+                raise TypeError("per-channel scales must follow the output-channel axis of the weight")
+            return Value(C, "int", np.float32(a.qscale) * b.qscale.astype(np.float32), 0, C.ndim - 1)
         return Value(C, "int", np.float32(a.qscale) * np.float32(b.qscale), 0)
     if a.kind == "int" or b.kind == "int":
         raise TypeError("mixed integer/float MatMul")
@@ -114,6 +131,10 @@ def op_dequantize(x: Value) -> Value:
     if x.kind != "int":
         raise TypeError("Dequantize needs an integer tensor")
     t = (x.data - x.zero_point).astype(np.float32)      # round-to-nearest-even for |.| > 2^24
+    if np.ndim(x.qscale) != 0:                          # one scale per index of axis `qaxis`
+        shape = [1] * t.ndim
+        shape[x.qaxis] = -1
+        return Value((t * x.qscale.astype(np.float32).reshape(shape)).astype(np.float32), "f32x")
     return Value(t * np.float32(x.qscale), "f32x")
 
 

@@ -40,6 +40,11 @@ class LogicalTensor:
     zero_point: int = 0
     is_constant: bool = False  # same pointer and contents on every execution (weights, biases)
     name: str = ""
+    # per-channel quantisation of a constant s8 weight (Section VII: "per channel s8 symmetric quantization
+    # for weight"): one scale per index of `channel_axis`, which must be the output-channel axis of the
+    # MatMul that consumes the tensor.  None = the per-tensor `scale` applies.
+    channel_scales: Optional[Tuple[float, ...]] = None
+    channel_axis: int = -1
 
     @property
     def numel(self) -> int:
@@ -73,11 +78,18 @@ class Graph:
 
     # -- small builder helpers (bookkeeping only) ---------------------------------------------
     def tensor(self, dtype: str, dims: Sequence[int], *, scale: float = 1.0, zero_point: int = 0,
-               is_constant: bool = False, name: str = "") -> int:
+               is_constant: bool = False, name: str = "", channel_scales: Optional[Sequence[float]] = None,
+               channel_axis: int = -1) -> int:
         assert dtype in DTYPES, dtype
         tid = len(self.tensors)
-        self.tensors[tid] = LogicalTensor(tid, dtype, tuple(int(d) for d in dims), float(scale),
-                                          int(zero_point), bool(is_constant), name)
+        dims = tuple(int(d) for d in dims)
+        cs = None
+        if channel_scales is not None:
+            channel_axis = channel_axis % len(dims)
+            cs = tuple(float(s) for s in channel_scales)
+            assert len(cs) == dims[channel_axis], "one scale per channel"
+        self.tensors[tid] = LogicalTensor(tid, dtype, dims, float(scale), int(zero_point), bool(is_constant), name,
+                                          cs, int(channel_axis))
         return tid
 
     def input(self, *a, **k) -> int:

@@ -90,20 +90,28 @@ def mlp_f32(batch: int = 32, dims: Sequence[int] = (13, 512, 256, 128), seed: in
 
 def mlp_int8(batch: int = 128, dims: Sequence[int] = (479, 1024, 1024, 512, 256, 1), seed: int = 0,
              s_x: float = 0.02, s_w: float = 0.005, s_act: float = 0.05,
-             final: str = "sigmoid") -> Workload:
+             final: str = "sigmoid", per_channel: bool = False, x_zp: int = 0, act_zp: int = 0) -> Workload:
     """int8 MLP (config 2 at the defaults): u8 activations, s8 weights, s32 accumulation;
     hidden layers dequantize + bias + ReLU + requantize to u8; the last layer dequantizes,
-    adds its bias and applies ``final`` ("sigmoid", or "none" to expose the fp32 logits)."""
+    adds its bias and applies ``final`` ("sigmoid", or "none" to expose the fp32 logits).
+    ``per_channel`` gives every weight one scale per output column (drawn in [0.5, 1.5] x s_w), ``x_zp`` /
+    ``act_zp`` are the zero points of the input and of the requantised hidden activations: together the
+    evaluation's scheme of asymmetric u8 activations and per-channel symmetric s8 weights."""
     rng = np.random.default_rng(seed)
-    g = Graph(name=f"mlp_int8_b{batch}_" + "x".join(map(str, dims)))
+    g = Graph(name=f"mlp_int8_b{batch}_" + "x".join(map(str, dims)) + ("_pc" if per_channel else "") +
+              (f"_zp{x_zp}_{act_zp}" if (x_zp or act_zp) else ""))
     feeds = {}
-    x = g.input("u8", (batch, dims[0]), scale=s_x, zero_point=0, name="x")
+    x = g.input("u8", (batch, dims[0]), scale=s_x, zero_point=x_zp, name="x")
     feeds[x] = rng.integers(0, 256, size=(batch, dims[0]), dtype=np.int64).astype(np.uint8)
     nl = len(dims) - 1
     ws, bs = [], []
     for l in range(nl):
         k, n = dims[l], dims[l + 1]
-        w = g.input("s8", (k, n), scale=s_w, is_constant=True, name=f"w{l}")
+        if per_channel:
+            cs = (s_w * np.random.default_rng(seed + 1000 + l).uniform(0.5, 1.5, size=n)).astype(np.float32)
+            w = g.input("s8", (k, n), scale=s_w, is_constant=True, name=f"w{l}", channel_scales=cs, channel_axis=1)
+        else:
+            w = g.input("s8", (k, n), scale=s_w, is_constant=True, name=f"w{l}")
         feeds[w] = rng.integers(-127, 128, size=(k, n), dtype=np.int64).astype(np.int8)
         ws.append(w)
     for l in range(nl):
@@ -119,7 +127,7 @@ def mlp_int8(batch: int = 128, dims: Sequence[int] = (479, 1024, 1024, 512, 256,
         z = g.op("add", (z, bs[l]), g.tensor("f32", (batch, n)))
         if l < nl - 1:
             z = g.op("relu", (z,), g.tensor("f32", (batch, n)))
-            h = g.op("quantize", (z,), g.tensor("u8", (batch, n), scale=s_act, zero_point=0))
+            h = g.op("quantize", (z,), g.tensor("u8", (batch, n), scale=s_act, zero_point=act_zp))
         else:
             h = z if final == "none" else g.op(final, (z,), g.tensor("f32", (batch, n)))
     g.mark_output(h)

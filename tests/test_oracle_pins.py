@@ -294,6 +294,78 @@ def test_mlp_int8_against_straight_line_restatement():
         assert abs(sg[m, 0] - 1.0 / (1.0 + math.exp(-float(got[m, 0])))) < 1e-15
 
 
+def test_mlp_int8_per_channel_asymmetric_against_straight_line_restatement():
+    # the evaluation's scheme (Section VII): asymmetric u8 activations, per-channel symmetric s8 weights.
+    # Python integers for the sums, struct-rounded fp32 for every float step.
+    import struct
+
+    def r32(v):
+        return struct.unpack("f", struct.pack("f", v))[0]
+
+    w = W.mlp_int8(batch=3, dims=(9, 8, 5), seed=5, final="none", per_channel=True, x_zp=7, act_zp=3)
+    got = run1(w)
+    g = w.graph
+    x = w.feeds[g.inputs[0]].tolist()
+    ws = [w.feeds[g.inputs[1 + l]].tolist() for l in range(2)]
+    bs = [[float(v) for v in w.feeds[g.inputs[3 + l]]] for l in range(2)]
+    cs = [[r32(v) for v in g.tensors[g.inputs[1 + l]].channel_scales] for l in range(2)]
+    assert len(set(cs[0])) > 1                       # the scales really differ per column
+    a_scale, a_zp = [r32(0.02), r32(0.05)], [7, 3]
+    inv = r32(1.0 / r32(0.05))
+    for m in range(3):
+        act = x[m]
+        for l in range(2):
+            K, N = len(ws[l]), len(ws[l][0])
+            nxt = []
+            for n in range(N):
+                acc = sum((act[k] - a_zp[l]) * ws[l][k][n] for k in range(K))
+                # the identity the low-precision conversion relies on: the zero point leaves the sum as a
+                # per-column constant, a_z * colsum(W)
+                assert acc == sum(act[k] * ws[l][k][n] for k in range(K)) - a_zp[l] * sum(ws[l][k][n] for k in range(K))
+                dq = r32(a_scale[l] * cs[l][n])      # product of two fp32 values is exact in fp64: one rounding
+                t = r32(r32(float(acc)) * dq)
+                t = r32(t + bs[l][n])
+                if l == 0:
+                    t = max(t, 0.0)
+                    u = r32(t * inv)
+                    r = int(np.rint(np.float64(u)))
+                    nxt.append(min(max(r + 3, 0), 255))
+                else:
+                    nxt.append(t)
+            act = nxt
+        assert got.dtype == np.float32
+        assert got[m].tolist() == act
+
+
+def test_per_channel_scales_reduce_to_per_tensor_and_follow_the_n_axis():
+    # equal channel scales are the per-tensor case; a transposed weight carries them on axis 0
+    base = W.mlp_int8(batch=4, dims=(12, 6), seed=2, final="none")
+    ref = run1(base)
+    for transposed in (False, True):
+        g = Graph()
+        feeds = {}
+        x = g.input("u8", (4, 12), scale=0.02, name="x")
+        wshape = (6, 12) if transposed else (12, 6)
+        wt = g.input("s8", wshape, scale=123.0, is_constant=True, channel_scales=[0.005] * 6,
+                     channel_axis=0 if transposed else 1)
+        b = g.input("f32", (6,), is_constant=True)
+        wv = base.feeds[base.graph.inputs[1]]
+        feeds[x], feeds[wt], feeds[b] = base.feeds[base.graph.inputs[0]], (wv.T.copy() if transposed else wv), \
+            base.feeds[base.graph.inputs[2]]
+        acc = g.op("matmul", (x, wt), g.tensor("s32", (4, 6)), transpose_b=transposed)
+        z = g.op("dequantize", (acc,), g.tensor("f32", (4, 6)))
+        g.mark_output(g.op("add", (z, b), g.tensor("f32", (4, 6))))
+        got = interp.run(g, feeds)[g.outputs[0]]
+        assert np.array_equal(got, ref)
+    # scales on the reduction axis are meaningless and refused
+    g = Graph()
+    x = g.input("u8", (2, 4), scale=0.02)
+    wt = g.input("s8", (4, 3), is_constant=True, channel_scales=[0.1] * 4, channel_axis=0)
+    g.mark_output(g.op("matmul", (x, wt), g.tensor("s32", (2, 3))))
+    with pytest.raises(TypeError):
+        interp.run(g, {x: np.zeros((2, 4), np.uint8), wt: np.zeros((4, 3), np.int8)})
+
+
 def test_mlp_f32_against_straight_line_restatement():
     w = W.mlp_f32(batch=2, dims=(5, 6, 3), seed=12)
     got = run1(w)
