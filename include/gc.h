@@ -95,6 +95,13 @@ typedef struct {
   float scale;            /* per-tensor quantisation scale; ignored for float dtypes */
   int32_t zero_point;
   int32_t is_constant;    /* 1: same pointer and contents on every execution (weights, biases) */
+  /* Per-channel quantisation (Section VII: "per channel s8 symmetric quantization for weight"): a HOST array
+   * of dims[channel_axis] scales, copied by gc_partition_create; NULL = the per-tensor `scale` applies.
+   * Accepted only on the constant s8 weight of a 2-D MatMul, along its output-channel axis (1 for a [k,n]
+   * weight, 0 for a transposed [n,k] one); anything else is GC_ERR_UNSUPPORTED. */
+  const float* channel_scales;
+  int32_t channel_axis;
+  int32_t reserved_;
 } gc_logical_tensor_t;
 
 /* Op (Section II: kind, attributes, input and output logical tensors). */

@@ -39,7 +39,8 @@ EXPORTS = [
 
 class gc_logical_tensor_t(C.Structure):
     _fields_ = [("id", C.c_int64), ("dtype", C.c_int32), ("ndims", C.c_int32), ("dims", C.c_int64 * 6),
-                ("scale", C.c_float), ("zero_point", C.c_int32), ("is_constant", C.c_int32)]
+                ("scale", C.c_float), ("zero_point", C.c_int32), ("is_constant", C.c_int32),
+                ("channel_scales", C.POINTER(C.c_float)), ("channel_axis", C.c_int32), ("reserved_", C.c_int32)]
 
 
 class gc_op_t(C.Structure):
@@ -116,6 +117,7 @@ def gc_version() -> str:
 def marshal_graph(g: Graph):
     """Graph -> (ops array, tensors array, input ids, output ids) in the C layout."""
     tensors = (gc_logical_tensor_t * len(g.tensors))()
+    keep = []
     for i, t in enumerate(g.tensors.values()):
         tensors[i].id = t.id
         tensors[i].dtype = DTYPE_CODE[t.dtype]
@@ -125,6 +127,12 @@ def marshal_graph(g: Graph):
         tensors[i].scale = t.scale
         tensors[i].zero_point = t.zero_point
         tensors[i].is_constant = int(t.is_constant)
+        if t.channel_scales is not None:
+            cs = (C.c_float * len(t.channel_scales))(*t.channel_scales)
+            keep.append(cs)                      # alive until gc_partition_create has copied it
+            tensors[i].channel_scales = C.cast(cs, C.POINTER(C.c_float))
+            tensors[i].channel_axis = t.channel_axis
+    tensors._channel_scale_arrays = keep
     ops = (gc_op_t * len(g.ops))()
     for i, op in enumerate(g.ops):
         ops[i].kind = OP_CODE[op.kind]

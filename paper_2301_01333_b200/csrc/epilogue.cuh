@@ -32,8 +32,8 @@ __device__ __forceinline__ float apply_act(float t, int act) {
 __device__ __forceinline__ float epi_value(uint32_t raw, int n, const Epilogue& e) {
   float t;
   if (e.acc_is_int) {
-    t = __int2float_rn(static_cast<int>(raw));
-    t = __fmul_rn(t, e.dq);
+    t = __int2float_rn(static_cast<int>(raw) - (e.comp ? __ldg(e.comp + n) : 0));
+    t = __fmul_rn(t, e.dqv ? __ldg(e.dqv + n) : e.dq);
   } else {
     t = __uint_as_float(raw);
   }
@@ -52,10 +52,25 @@ __device__ __forceinline__ int quantize_value(float t, float inv, int zp, int lo
 // `dst_row` points at column 0 of the row; n0 is a multiple of 16 and the row pitch keeps 16-byte
 // alignment of (dst_row + n0) for every supported dtype.
 __device__ __forceinline__ void epi_store16(const uint32_t* raw, void* dst_row, int n0, const Epilogue& e) {
+  // zero-point compensation of the integer accumulator (exact in s32)
+  int c[16];
+  if (e.comp) {
+    const int4* cp = reinterpret_cast<const int4*>(e.comp + n0);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int4 v = __ldg(cp + i);
+      c[4 * i] = v.x; c[4 * i + 1] = v.y; c[4 * i + 2] = v.z; c[4 * i + 3] = v.w;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) c[i] = 0;
+  }
   if (e.acc_is_int && !e.has_dq) {   // raw s32 accumulators
     int4* d = reinterpret_cast<int4*>(static_cast<int*>(dst_row) + n0);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) d[i] = make_int4(raw[4 * i], raw[4 * i + 1], raw[4 * i + 2], raw[4 * i + 3]);
+    for (int i = 0; i < 4; ++i)
+      d[i] = make_int4(static_cast<int>(raw[4 * i]) - c[4 * i], static_cast<int>(raw[4 * i + 1]) - c[4 * i + 1],
+                       static_cast<int>(raw[4 * i + 2]) - c[4 * i + 2], static_cast<int>(raw[4 * i + 3]) - c[4 * i + 3]);
     return;
   }
   // Fetch the 16 bias values with four vector loads up front: per-element loads behind per-element branches
@@ -73,12 +88,23 @@ __device__ __forceinline__ void epi_store16(const uint32_t* raw, void* dst_row, 
     for (int i = 0; i < 16; ++i) b[i] = 0.f;
   }
   const bool has_bias = e.bias != nullptr, acc_int = e.acc_is_int != 0;
-  const float dq = e.dq;
+  float dq[16];
+  if (e.dqv) {
+    const float4* dp = reinterpret_cast<const float4*>(e.dqv + n0);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float4 v = __ldg(dp + i);
+      dq[4 * i] = v.x; dq[4 * i + 1] = v.y; dq[4 * i + 2] = v.z; dq[4 * i + 3] = v.w;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) dq[i] = e.dq;
+  }
   const int act = e.act;
   float t[16];
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
-    float x = acc_int ? __fmul_rn(__int2float_rn(static_cast<int>(raw[i])), dq) : __uint_as_float(raw[i]);
+    float x = acc_int ? __fmul_rn(__int2float_rn(static_cast<int>(raw[i]) - c[i]), dq[i]) : __uint_as_float(raw[i]);
     x = has_bias ? __fadd_rn(x, b[i]) : x;      // separately rounded: exact on the integer path
     t[i] = x;
   }

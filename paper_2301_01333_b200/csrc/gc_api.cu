@@ -49,6 +49,11 @@ struct gc_partition {
   std::vector<gc_op_t> ops;
   std::vector<gc_logical_tensor_t> tensors;
   std::map<int64_t, int> index;   // tensor id -> position in `tensors`
+  std::map<int64_t, std::vector<float>> channel_scales;   // copies of the callers' per-channel scale arrays
+  const std::vector<float>* ch_scales(int64_t id) const {
+    auto it = channel_scales.find(id);
+    return it == channel_scales.end() ? nullptr : &it->second;
+  }
   std::vector<int64_t> in_ids, out_ids;
   const gc_logical_tensor_t* lt(int64_t id) const {
     auto it = index.find(id);
@@ -107,6 +112,16 @@ extern "C" gc_status_t gc_partition_create(gc_partition_t** out, const gc_op_t* 
     if (is_int8(t.dtype) && !(t.scale > 0.f) ) return bail(fail(GC_ERR_INVALID_ARG, "tensor %lld: scale must be positive", (long long)t.id));
     p->index[t.id] = static_cast<int>(p->tensors.size());
     p->tensors.push_back(t);
+    p->tensors.back().channel_scales = nullptr;       // the caller's array is not kept; see p->channel_scales
+    if (t.channel_scales) {
+      if (t.dtype != GC_S8 || !t.is_constant || t.ndims != 2 || t.channel_axis < 0 || t.channel_axis > 1)
+        return bail(fail(GC_ERR_UNSUPPORTED, "tensor %lld: per-channel scales need a constant 2-D s8 weight and axis 0 or 1",
+                         (long long)t.id));
+      std::vector<float> cs(t.channel_scales, t.channel_scales + t.dims[t.channel_axis]);
+      for (float s : cs)
+        if (!(s > 0.f)) return bail(fail(GC_ERR_INVALID_ARG, "tensor %lld: channel scales must be positive", (long long)t.id));
+      p->channel_scales[t.id] = std::move(cs);
+    }
   }
   std::map<int64_t, bool> defined;
   for (int i = 0; i < n_in; ++i) {
@@ -199,6 +214,10 @@ struct LayerPlan {
   int64_t pack_pitch = 0;    // elements
   size_t wt_off = 0;
   int Kp = 0;
+  std::vector<float> dqv_host;   // per-channel weights: float32(a_scale) * float32(w_scale[n]) per output column
+  size_t dqv_off = 0;            // workspace offset of their device copy
+  bool need_comp = false;        // tcgen05 path with a non-zero activation zero point
+  size_t comp_off = 0;           // workspace offset of a_zp * colsum(W), s32 per output column
   // cached tensor maps
   CUtensorMap tmA, tmB, tmD;
   const void* tmA_ptr = nullptr;
@@ -338,6 +357,12 @@ static gc_status_t match_mlp(const gc_partition& p, gc_compiled& c) {
       if (!int_path) return fail(GC_ERR_UNSUPPORTED, "dequantize after a float matmul");
       L.epi.has_dq = 1;
       L.epi.dq = a->scale * w->scale;   // fp32 product, the scale of the s32 result
+      if (const std::vector<float>* cs = p.ch_scales(mm.in[1])) {
+        if (w->channel_axis != (mm.transpose_b ? 0 : 1))
+          return fail(GC_ERR_UNSUPPORTED, "op %zu: per-channel scales must run along the weight's output-channel axis", i);
+        L.dqv_host.resize(cs->size());
+        for (size_t n = 0; n < cs->size(); ++n) L.dqv_host[n] = a->scale * (*cs)[n];
+      }
       L.epi.out_dtype = GC_F32;
       t = p.ops[i++].out;
     }
@@ -611,6 +636,15 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
       L.Kp = static_cast<int>(align_up(static_cast<size_t>(L.K) * esz, 128) / esz);
       L.wt_off = ws;
       ws = align_up(ws + static_cast<size_t>(L.N) * L.Kp * esz, 1024);
+      // constants derived from the quantisation parameters and the weight: per-column scales, compensation
+      if (!L.dqv_host.empty()) {
+        L.dqv_off = ws;
+        ws = align_up(ws + align_up(static_cast<size_t>(L.N), 16) * sizeof(float), 256);
+      }
+      if (L.epi.acc_is_int && L.a_zp != 0) {
+        L.comp_off = ws;
+        ws = align_up(ws + align_up(static_cast<size_t>(L.N), 16) * sizeof(int), 256);
+      }
     }
     // temporaries between fused ops: two buffers reused alternately (life spans never overlap by
     // more than one layer), each sized for the largest tensor it ever holds
@@ -637,9 +671,12 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
       } else {
         L.a_pitch = L.K;
       }
-      const bool dt_ok = (is_int8(L.a_dtype) && L.w_dtype == GC_S8 && L.a_zp == 0) || L.a_dtype == GC_BF16 ||
-                         L.a_dtype == GC_F32;
+      // 8-bit operands go to the tensor cores as stored; a non-zero activation zero point is removed afterwards
+      // with the compensation term, which needs |sum_k a_k w_kn| and |a_z colsum(W)_n| to stay inside s32
+      const bool dt_ok = (is_int8(L.a_dtype) && L.w_dtype == GC_S8 && (L.a_zp == 0 || L.K <= 65536)) ||
+                         L.a_dtype == GC_BF16 || L.a_dtype == GC_F32;
       L.use_tc = !c->opt.force_generic && dt_ok && L.N >= 16 && L.N % 16 == 0;
+      L.need_comp = L.use_tc && is_int8(L.a_dtype) && L.a_zp != 0;
       if (L.use_tc) {
         L.kind = is_int8(L.a_dtype) ? 0 : (L.a_dtype == GC_BF16 ? 1 : 2);
         choose_tile(L, c->num_sms);
@@ -785,6 +822,10 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
   if (need) {
     for (auto& L : c.layers) {
       CUDA_TRY(launch_prepack_weight(in[L.w_input], ws + L.wt_off, L.K, L.N, L.Kp, L.transposed_w, L.w_dtype, st));
+      if (!L.dqv_host.empty())
+        CUDA_TRY(cudaMemcpyAsync(ws + L.dqv_off, L.dqv_host.data(), L.dqv_host.size() * sizeof(float), cudaMemcpyHostToDevice, st));
+      if (L.need_comp)
+        CUDA_TRY(launch_weight_compensation(ws + L.wt_off, L.N, L.Kp, L.a_zp, reinterpret_cast<int*>(ws + L.comp_off), st));
       c.const_ptrs[L.w_input] = in[L.w_input];
     }
     c.prepacked = true;
@@ -837,6 +878,8 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
       cl.out_elem = L.out_elem;
       cl.epi = L.epi;
       cl.epi.bias = L.bias_input >= 0 ? static_cast<const float*>(in[L.bias_input]) : nullptr;
+      cl.epi.dqv = L.dqv_host.empty() ? nullptr : reinterpret_cast<const float*>(ws + L.dqv_off);
+      cl.epi.comp = L.need_comp ? reinterpret_cast<const int*>(ws + L.comp_off) : nullptr;
       if (L.use_tc) {
         const uint32_t afmt = L.a_dtype == GC_S8 ? 1u : 0u;
         cl.idesc = L.kind == 0   ? ((2u << 4) | (afmt << 7) | (1u << 10) | ((32u >> 3) << 17) | ((128u >> 4) << 24))
@@ -869,6 +912,8 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
     void* O = L.out_pos >= 0 ? out[L.out_pos] : ws + L.out_off;
     Epilogue e = L.epi;
     e.bias = L.bias_input >= 0 ? static_cast<const float*>(in[L.bias_input]) : nullptr;
+    e.dqv = L.dqv_host.empty() ? nullptr : reinterpret_cast<const float*>(ws + L.dqv_off);
+    e.comp = L.need_comp ? reinterpret_cast<const int*>(ws + L.comp_off) : nullptr;
     if (L.use_tc) {
       if (L.need_pack) {
         CUDA_TRY(launch_pack_rows(A, ws + L.pack_off, L.M, L.a_pitch * esz, L.pack_pitch * esz, st));

@@ -22,6 +22,9 @@ struct Epilogue {
   int acc_is_int;
   int has_dq;
   float dq;
+  const float* dqv;  // per-output-column dequantisation scales (per-channel weight scales), or null: `dq` applies
+  const int* comp;   // per-output-column s32 compensation a_z * colsum(W), subtracted from the raw accumulator
+                     // of a kernel that multiplies the stored (not zero-point-shifted) activation codes; or null
   const float* bias;
   int act;
   int out_dtype;   // gc_dtype_t
@@ -119,6 +122,8 @@ cudaError_t launch_pack_rows(const void* src, void* dst, int rows, int64_t src_p
 // reduction axis contiguous and zero padded.  f32 weights are rounded to tf32 (nearest, ties away).
 cudaError_t launch_prepack_weight(const void* W, void* Wt, int K, int N, int Kp, int transposed, int dtype,
                                   cudaStream_t s);
+// comp[n] = a_zp * sum_k Wt[n][k] for a prepacked s8 weight (zero padded to Kp)
+cudaError_t launch_weight_compensation(const void* Wt, int N, int Kp, int a_zp, int* comp, cudaStream_t s);
 cudaError_t launch_gemm_simt(const GemmSimtParams& p, cudaStream_t s);
 cudaError_t launch_sdpa_simt(const SdpaParams& p, cudaStream_t s);
 

@@ -30,11 +30,39 @@ __device__ __forceinline__ void epi_values32(const uint32_t (&raw)[32], float (&
 #pragma unroll
     for (int i = 0; i < 32; ++i) b[i] = 0.f;
   }
+  // integer path: optional per-column compensation and per-column scales (global memory, a multiple of 16
+  // columns is always allocated so whole vectors inside [n0, n_end rounded up to 16) are readable)
+  int c[32];
+  float dq[32];
+  if constexpr (KIND == KIND_I8) {
+    if (e.comp) {
+      const int4* cp = reinterpret_cast<const int4*>(e.comp + n0);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int4 v = n0 + 4 * i < n_end ? __ldg(cp + i) : make_int4(0, 0, 0, 0);
+        c[4 * i] = v.x; c[4 * i + 1] = v.y; c[4 * i + 2] = v.z; c[4 * i + 3] = v.w;
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) c[i] = 0;
+    }
+    if (e.dqv) {
+      const float4* dp = reinterpret_cast<const float4*>(e.dqv + n0);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float4 v = n0 + 4 * i < n_end ? __ldg(dp + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        dq[4 * i] = v.x; dq[4 * i + 1] = v.y; dq[4 * i + 2] = v.z; dq[4 * i + 3] = v.w;
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) dq[i] = e.dq;
+    }
+  }
 #pragma unroll
   for (int i = 0; i < 32; ++i) {
     float x;
     if constexpr (KIND == KIND_I8) {
-      x = __fmul_rn(__int2float_rn(static_cast<int>(raw[i])), e.dq);
+      x = __fmul_rn(__int2float_rn(static_cast<int>(raw[i]) - c[i]), dq[i]);
       x = e.bias ? __fadd_rn(x, b[i]) : x;                      // separately rounded on the integer path
     } else {
       x = __uint_as_float(raw[i]) + b[i];
@@ -83,8 +111,13 @@ template <int KIND, int OUT>
 __device__ __forceinline__ void epi_chunk32(const uint32_t (&raw)[32], uint32_t* w, int n0, int n_end,
                                             const Epilogue& e) {
   if constexpr (OUT == OUT_RAW32) {
+    if (KIND == KIND_I8 && e.comp) {
 #pragma unroll
-    for (int i = 0; i < 32; ++i) w[i] = raw[i];
+      for (int i = 0; i < 32; ++i) w[i] = raw[i] - static_cast<uint32_t>(n0 + i < n_end ? __ldg(e.comp + n0 + i) : 0);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) w[i] = raw[i];
+    }
   } else {
     float t[32];
     switch (e.act) {

@@ -94,6 +94,29 @@ cudaError_t launch_prepack_weight(const void* W, void* Wt, int K, int N, int Kp,
 }
 
 // ------------------------------------------------------------------------------------------------
+// Compensated weight (Section V, constant weight preprocessing; Section VII "compensated weight"):
+// sum_k (a_k - a_z) w_kn = sum_k a_k w_kn - a_z colsum(W)_n.  The second term depends on constants only and is
+// formed once from the prepacked s8 weight Wt[N][Kp]; one warp per output column.
+// ------------------------------------------------------------------------------------------------
+__global__ void weight_compensation_kernel(const int8_t* __restrict__ Wt, int N, int Kp, int a_zp, int* __restrict__ comp) {
+  const int lane = threadIdx.x & 31;
+  const int n = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (n >= N) return;
+  const int8_t* row = Wt + static_cast<int64_t>(n) * Kp;
+  int acc = 0;
+  for (int k = lane; k < Kp; k += 32) acc += row[k];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) comp[n] = a_zp * acc;
+}
+
+cudaError_t launch_weight_compensation(const void* Wt, int N, int Kp, int a_zp, int* comp, cudaStream_t s) {
+  const int threads = 256, blocks = (N * 32 + threads - 1) / threads;
+  weight_compensation_kernel<<<blocks, threads, 0, s>>>(static_cast<const int8_t*>(Wt), N, Kp, a_zp, comp);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
 // gemm_simt: one warp per output element, lanes stride the reduction axis, fixed-order shuffle tree.
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ float load_as_float(const void* p, int64_t i, int dtype) {

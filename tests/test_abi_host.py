@@ -115,3 +115,28 @@ def test_compile_rejects_unsupported_patterns():
     with pytest.raises(B.GcError):
         B.gc_compile(p, 99)
     B.gc_partition_destroy(p)
+
+
+def test_per_channel_scales_and_zero_points_plan_on_tensor_cores_and_bad_uses_are_refused():
+    c = plan(W.mlp_int8(per_channel=True, x_zp=12, act_zp=5).graph)
+    assert c.plan.count("tcgen05.i8") == 4          # a non-zero activation zero point no longer leaves the tcgen05 path
+    # scales along the reduction axis
+    w = W.mlp_int8(batch=4, dims=(16, 16), per_channel=True)
+    w.graph.tensors[w.graph.inputs[1]].channel_axis = 0
+    with pytest.raises(B.GcError) as e:
+        plan(w.graph)
+    assert e.value.status == B.GC_ERR_UNSUPPORTED
+    # scales on an activation
+    w = W.mlp_int8(batch=4, dims=(16, 16))
+    x = w.graph.tensors[w.graph.inputs[0]]
+    x.channel_scales, x.channel_axis = (0.1,) * 16, 1
+    with pytest.raises(B.GcError) as e:
+        B.gc_partition_create(w.graph)
+    assert e.value.status == B.GC_ERR_UNSUPPORTED
+    # a non-positive scale
+    w = W.mlp_int8(batch=4, dims=(16, 16), per_channel=True)
+    t = w.graph.tensors[w.graph.inputs[1]]
+    t.channel_scales = (0.0,) + t.channel_scales[1:]
+    with pytest.raises(B.GcError) as e:
+        B.gc_partition_create(w.graph)
+    assert e.value.status == B.GC_ERR_INVALID_ARG

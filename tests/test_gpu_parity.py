@@ -144,6 +144,29 @@ def test_mlp_int8_logits_bit_exact_and_sigmoid(B, batch, dims, opts):
     assert np.abs(gs.astype(np.float64) - oracle(ws)).max() <= 2e-6
 
 
+@pytest.mark.parametrize("batch,dims", [(128, (479, 1024, 1024, 512, 256, 1)), (37, (100, 80, 48, 16)),
+                                        (2600, (512, 2048, 256))])
+@pytest.mark.parametrize("opts", [{}, {"force_generic": True}, {"no_chain_fusion": True}])
+def test_mlp_int8_per_channel_scales_and_zero_points_bit_exact(B, batch, dims, opts):
+    # the evaluation's scheme (Section VII): asymmetric u8 activations, per-channel s8 weight scales; the tensor
+    # cores multiply the stored codes and the zero point leaves through the compensated-weight term
+    w = W.mlp_int8(batch=batch, dims=dims, final="none", per_channel=True, x_zp=12, act_zp=5)
+    got, plan = run_gpu(B, w, **opts)
+    if not opts.get("force_generic"):
+        assert "tcgen05.i8" in plan
+    ref = oracle(w)
+    assert ref.dtype == np.float32
+    assert np.array_equal(got, ref)
+
+
+@pytest.mark.parametrize("m,k,n,zp", [(128, 1024, 256, 128), (77, 130, 48, 3), (2600, 512, 2048, 200)])
+def test_int8_matmul_nonzero_zero_point_on_tensor_cores_exact(B, m, k, n, zp):
+    w = W.single_matmul("u8", "s8", m, k, n, seed=zp, a_zp=zp)
+    got, plan = run_gpu(B, w)
+    assert "tcgen05.i8" in plan
+    assert np.array_equal(got.astype(np.int64), oracle(w))
+
+
 def test_mlp_int8_hidden_layer_codes_bit_exact(B):
     # a chain that ends on a requantised u8 tensor: compares the codes themselves
     w = W.mlp_int8(batch=128, dims=(479, 1024, 512), final="none")
