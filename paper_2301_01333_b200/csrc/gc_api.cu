@@ -465,6 +465,14 @@ static gc_status_t match_sdpa(const gc_partition& p, gc_compiled& c) {
     if (pq->dtype != GC_U8) return fail(GC_ERR_UNSUPPORTED, "attention: quantized probabilities must be u8");
     prm.p_is_quant = 1;
     prm.inv_p = 1.0f / pq->scale;
+    {
+      // Largest |score| in log2 units: |q - 128| <= 128, |k code| <= 255 over D terms, times the folded scale.
+      // A key whose mask term is below -(2 bound + 1 + 150) sits more than 150 binades under any row maximum
+      // that an unmasked key (mask term >= -1) sets, so its fp32 exponential is exactly zero.
+      const double bound = 128.0 * 255.0 * static_cast<double>(prm.D) *
+                           std::fabs(static_cast<double>(prm.dq1) * prm.scalar) * 1.4426950408889634;
+      prm.skip_thr = static_cast<float>(2.0 * bound + 151.0);
+    }
     prm.zp_p = pq->zero_point;
     t = p.ops[i++].out;
   } else {

@@ -75,6 +75,9 @@ struct SdpaParams {
   int zp_o;
   int out_dtype;       // GC_BF16 or GC_U8 / GC_S8
   int q_signed, k_signed, v_signed;   // s8 instead of u8 storage
+  float skip_thr;      // int8: a 32-key chunk whose mask values times log2(e) are all <= -skip_thr contributes exactly
+                       // zero to the softmax of any row that has an unmasked key (bound derived from the largest
+                       // possible integer score); 0 disables the skipping of such chunks
   uint32_t* status;
 };
 

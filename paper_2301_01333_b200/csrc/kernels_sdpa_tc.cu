@@ -57,7 +57,7 @@ struct SdpaSmem {
   __host__ __device__ static constexpr int slot_bytes(int S) { return q_bytes() + 2 * kv_bytes(S); }
   __host__ __device__ static constexpr int total(int S, int slots, int nsb, int stage_out) {
     return slots * slot_bytes(S) + nsb * p_bytes(S) + (stage_out ? OUT_STAGING_BYTES : 0) + slots * S * 4 /*mask*/ +
-           24 * 128 * 4 /*row statistics*/ + 256;
+           24 * 128 * 4 /*row statistics*/ + 384 /*barriers, TMEM address, chunk flags*/;
   }
 };
 
@@ -125,6 +125,8 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   float* sStat = sMask + slots * S;                                       // [3 kinds][2 parities][4 groups][128]
   uint64_t* bars = reinterpret_cast<uint64_t*>(sStat + 24 * 128);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 26);
+  // per slot and 32-key chunk: 1 = every key of the chunk is masked out, 2 = the chunk has an unmasked key, 0 = neither
+  uint32_t* sChunk = tmem_slot + 4;                                       // [2 slots][16]
   const uint32_t b0 = smem_u32(bars);
   const uint32_t bar_kv_full = b0, bar_kv_empty = b0 + 16, bar_kv_ready = b0 + 32;   // [2] each
   const uint32_t bar_s_full = b0 + 48, bar_s_free = b0 + 72, bar_p_full = b0 + 96;   // [3] each
@@ -396,7 +398,15 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         failed = true;
         break;
       }
-      for (int j = t; j < S; j += 128) mk[j] = p.mask ? __ldg(p.mask + static_cast<int64_t>(b) * S + j) * LOG2E : 0.0f;
+      for (int j = t; j < S; j += 128) {                        // a warp covers one aligned 32-key chunk per step
+        const float mv = p.mask ? __ldg(p.mask + static_cast<int64_t>(b) * S + j) * LOG2E : 0.0f;
+        mk[j] = mv;
+        if constexpr (INT8) {
+          const bool all_masked = __all_sync(0xffffffffu, p.skip_thr > 0.f && mv <= -p.skip_thr);
+          const bool any_valid = __any_sync(0xffffffffu, mv >= -1.0f);
+          if (lane == 0) sChunk[s * 16 + (j >> 5)] = all_masked ? 1u : (any_valid ? 2u : 0u);
+        }
+      }
       if (INT8 && !p.q_signed) {
         uint4* q4 = reinterpret_cast<uint4*>(slot_q(s));
         for (int i = t; i < L::q_bytes() / 16; i += 128) {
@@ -453,6 +463,16 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       const uint32_t t_row = t_lane + buf * BUF_COLS;
       uint8_t* sP = sPall + buf * L::p_bytes(S);
       if (!mbar_wait(bar_kv_ready + 8 * s, (n / slots) & 1)) { failed = true; break; }
+      // Mask-aware skipping (int8): with at least one unmasked key in the row, a chunk whose keys are all
+      // masked has exponentials that underflow to exactly zero, so neither pass touches it: its codes are zero.
+      uint32_t skip = 0;                                        // bit b: my chunk of key block b is skipped
+      if constexpr (INT8) {
+        const uint32_t* fl = sChunk + s * 16;
+        bool any_valid = false;
+        for (int i = 0; i < NB * 4; ++i) any_valid = any_valid || fl[i] == 2u;
+        if (any_valid)
+          for (int b = 0; b < NB; ++b) skip |= (fl[b * 4 + g] == 1u ? 1u : 0u) << b;
+      }
 
       // ---------------- pass A: one 32-column chunk per key block, transformed in place
       // (accumulator -> scaled, masked score [-> exponential, stored back to tensor memory on the int8 path])
@@ -461,6 +481,10 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       uint32_t v[32];
       for (int b = 0; b < NB; ++b) {
         const int col = b * 128 + g * 32;
+        if (INT8 && ((skip >> b) & 1u)) {
+          if (b == 0) mc[0] = m; else if (b == 1) mc[1] = m; else mc[2] = m;
+          continue;
+        }
         if (!mbar_wait(bar_s_full + 8 * bx(buf, b), fpar)) { failed = true; break; }
         tc_fence_after();
         if constexpr (INT8) tmem_wait_st();                     // v[] may still feed the previous block's store
@@ -524,10 +548,14 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       for (int b = 0; b < NB; ++b) {
         const int col = b * 128 + g * 32;
         if constexpr (INT8) {
+          uint32_t w[8];
+          if ((skip >> b) & 1u) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) w[i] = 0u;
+          } else {
           tmem_ld32(t_row + col, v);
           tmem_wait_ld();
           const float f = ex2((b == 0 ? mc[0] : b == 1 ? mc[1] : mc[2]) - M) * scale;
-          uint32_t w[8];
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             // rne(e * f) lands in the low mantissa bits of (e * f + 1.5 * 2^23); codes are within [0, 255]
@@ -538,6 +566,7 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             const uint32_t y3 = __float_as_uint(fmaf(__uint_as_float(v[4 * i + 3]), f, MAGIC_F));
             w[i] = __byte_perm(__byte_perm(y0, y1, 0x0040), __byte_perm(y2, y3, 0x0040), 0x5410);
             psum = static_cast<int>(__dp4a(w[i], 0x01010101u, static_cast<unsigned>(psum)));
+          }
           }
           uint8_t* blk = sP + b * P_BLOCK_BYTES + row_off;
           const int c0 = g * 2;                                 // 16-byte chunk index inside the 128-byte row

@@ -237,6 +237,47 @@ def test_mha_int8_reduced(B, b, h, s, d, generic):
     check_int8_attention(got, oracle(w))
 
 
+def test_mha_int8_masked_chunk_skipping_edge_cases(B):
+    # the tcgen05 kernel leaves out 32-key chunks whose keys are all masked; rows must not notice.  Batches:
+    # everything masked (no skipping allowed: the mask then cancels in the softmax), one valid key, a valid
+    # length inside a chunk, a whole masked 128-key block, nothing masked, a mild mask value that is not
+    # skippable, masked keys in the middle of the row, and -inf.
+    w = W.mha_int8(batch=8, heads=2, seq=384, head_dim=64, seed=3)
+    g = w.graph
+    mid = [t for t in g.inputs if g.tensors[t].name == "mask"][0]
+    mask = np.zeros((8, 1, 1, 384), dtype=np.float32)
+    mask[0] = -10000.0
+    mask[1, ..., 1:] = -10000.0
+    mask[2, ..., 211:] = -10000.0
+    mask[3, ..., 256:] = -10000.0
+    mask[5, ..., 100:] = -3.0
+    mask[6, ..., 64:160] = -10000.0
+    mask[7, ..., 130:] = -np.inf
+    w.feeds[mid] = mask
+    g.mark_output(w.info["p_quant"])
+    import torch
+    c = B.CompiledPartition(g, 0)
+    assert "tcgen05" in c.plan
+    ins = B.device_inputs(w)
+    outs = B.device_outputs(g)
+    c.execute(ins, outs)
+    c.query_status()
+    torch.cuda.synchronize()
+    got_o = B.output_to_numpy(g, g.outputs[0], outs[0])
+    got_p = B.output_to_numpy(g, g.outputs[1], outs[1]).astype(np.int64)
+    c.close()
+    ref = interp.run(g, w.feeds)
+    # the rows of this test sit on many more rounding boundaries than random data (a handful of equal large
+    # probabilities per row): the codes may differ by one more often, the output by one code at most
+    dp = np.abs(got_p - ref[g.outputs[1]])
+    assert dp.max() <= 1 and (dp != 0).mean() <= 1e-3
+    assert np.abs(got_o.astype(np.int64) - ref[g.outputs[0]]).max() <= 1
+    assert_stage_after_softmax_exact(w, got_o, got_p.astype(np.uint8))
+    assert not got_p[2, :, :, 211:].any() and not got_p[3, :, :, 256:].any() and not got_p[6, :, :, 64:160].any()
+    assert not got_p[7, :, :, 130:].any()
+    assert got_p[0].any(axis=-2).all()               # fully masked batch: every key still receives weight
+
+
 @pytest.mark.parametrize("generic", [False, True])
 def test_mha_int8_stages_around_the_softmax(B, generic):
     """The fp32 softmax sits between two exact integer stages.  With the probabilities as a second output:
@@ -261,7 +302,13 @@ def test_mha_int8_stages_around_the_softmax(B, generic):
     dp = np.abs(p_gpu.astype(np.int64) - ref[g.outputs[1]])
     assert dp.max() <= 1 and (dp != 0).mean() <= 1e-3
     check_int8_attention(o_gpu, ref[g.outputs[0]])
-    # stage after the softmax alone, fed with the kernel's own codes
+    assert_stage_after_softmax_exact(w, o_gpu, p_gpu)
+
+
+def assert_stage_after_softmax_exact(w, o_gpu, p_gpu):
+    """P.V, dequantize, requantize recomputed by the oracle from the kernel's own probability codes."""
+    from paper_2301_01333_b200.graph import Graph
+    g = w.graph
     v_id = g.inputs[2]
     g3 = Graph()
     pin = g3.input("u8", g.tensors[g.outputs[1]].dims, scale=g.tensors[g.outputs[1]].scale, zero_point=0)
