@@ -186,6 +186,51 @@ def softmax_scores(w):
     return 0
 
 
+def sweep_cases():
+    """The shapes of the evaluation's workload table (Section VII, Table I): MLP-1 / MLP-2 at batch 32..512 and
+    MHA-1..4 at batch 32..128, in the 8-bit scheme and in this build's float types (tf32 MLP, bf16 attention)."""
+    cases = []
+    for b in (32, 64, 128, 256, 512):
+        cases.append((f"MLP-1 int8 b{b}", lambda b=b: W.mlp_int8(batch=b, dims=(13, 512, 256, 128), final="none")))
+        cases.append((f"MLP-1 f32 b{b}", lambda b=b: W.mlp_f32(batch=b)))
+        cases.append((f"MLP-2 int8 b{b}", lambda b=b: W.mlp_int8(batch=b)))
+        cases.append((f"MLP-2 f32 b{b}", lambda b=b: W.mlp_f32(batch=b, dims=(479, 1024, 1024, 512, 256, 1))))
+    for tag, seq, heads, hd in (("MHA-1", 128, 8, 96), ("MHA-2", 128, 12, 64), ("MHA-3", 384, 8, 128), ("MHA-4", 512, 16, 64)):
+        for b in (32, 64, 128):
+            cases.append((f"{tag} int8 b{b}", lambda b=b, s=seq, h=heads, d=hd: W.mha_int8(batch=b, heads=h, seq=s, head_dim=d)))
+            cases.append((f"{tag} bf16 b{b}", lambda b=b, s=seq, h=heads, d=hd: W.mha_bf16(batch=b, heads=h, seq=s, head_dim=d)))
+    return cases
+
+
+def run_sweep(B, device, peaks):
+    """One line per shape: cold time (rotating replicas above the L2 size), kernels chosen, HBM-roofline time."""
+    import torch
+    out = []
+    stream = torch.cuda.current_stream(device).cuda_stream
+    for label, make in sweep_cases():
+        w = make()
+        first = Replica(B, w, 0, device)
+        n_rep = int(min(32, max(2, -(-int(1.25 * L2_BYTES) // first.bytes))))
+        reps = [first] + [Replica(B, w, i + 1, device) for i in range(n_rep - 1)]
+        for r in reps:
+            r.step(stream)
+        torch.cuda.synchronize(device)
+        # size the timed loop from one measured step: about 50 ms, at least 10 steps
+        t1 = run_timed(reps, n_rep, 3, device, lambda: None) / 3
+        steps = int(max(10, min(2000, 50.0 / max(t1, 1e-3))))
+        us = run_timed(reps, n_rep, steps, device, lambda: None) * 1e3 / steps
+        reps[0].c.query_status()
+        kernels = sorted({tok for tok in reps[0].c.plan.replace("=", " ").split() if tok.startswith(("tcgen05", "cuda-core", "chain"))})
+        out.append({"case": label, "graph": w.name, "us": us, "steps": steps, "replicas": n_rep, "launches": reps[0].c.launches,
+                    "kernels": kernels, "ops": w.ops, "bytes": w.bytes, "t_hbm_us": w.bytes / (peaks["hbm_gbs"] * 1e9) * 1e6,
+                    "tops": w.ops / (us * 1e-6) / 1e12})
+        for r in reps:
+            r.c.close()
+        del reps, first
+        torch.cuda.empty_cache()
+    return out
+
+
 def run_e2e(w, rep, steps, warmup, device):
     """gc_execute_host with pinned host buffers: H2D of the non-constant inputs, execute, D2H, sync."""
     import torch
@@ -276,6 +321,8 @@ def main():
     ap.add_argument("--workload", default="c5", choices=list(W.CONFIGS))
     ap.add_argument("--only", action="store_true", help="time only the headline workload")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    ap.add_argument("--sweep", action="store_true",
+                    help="instead of the headline run, time every shape of the evaluation's workload table (1 GPU)")
     args = ap.parse_args()
     if args.impl == "reference":
         if args.steps == 0:
@@ -311,6 +358,13 @@ def main():
         return float(t.item())
 
     peaks, peak_src = load_peaks()
+    if args.sweep:
+        if rank == 0:
+            print(json.dumps({"sweep": run_sweep(B, local, peaks), "unit": "us per subgraph, cold L2", "data": "synthetic"}))
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
     head = args.workload
     names = [head] if args.only else [head] + [n for n in W.CONFIGS if n != head]
     results = {}

@@ -230,6 +230,7 @@ struct SdpaPlan {
   int q_input = -1, k_input = -1, v_input = -1, mask_input = -1, out_pos = 0;
   int p_out_pos = -1;        // graph output position of the probabilities tensor, if it is an output too
   bool use_tc = false;
+  bool wide = false;         // streaming kernel (wider heads, 512 keys) instead of the D = 64 kernel
   CUtensorMap tmQ, tmK, tmV, tmO;
   const void *q_ptr = nullptr, *k_ptr = nullptr, *v_ptr = nullptr, *o_ptr = nullptr;
 };
@@ -622,16 +623,22 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
     SdpaParams& s = c->sdpa.prm;
     bool tc = !c->opt.force_generic && s.D == 64 && s.S % 128 == 0 && s.S <= 384 &&
               sdpa_tc_smem_bytes(s.S, s.is_int8) <= static_cast<size_t>(prop.sharedMemPerBlockOptin);
-    if (!s.is_int8 && c->sdpa.p_out_pos >= 0) tc = false;   // the bf16 tcgen05 kernel never forms normalised P
+    bool wide = false;
+    if (!tc && !c->opt.force_generic) {
+      const size_t need = sdpa_wide_smem_bytes(s.S, s.D, s.is_int8);
+      wide = tc = need > 0 && need <= static_cast<size_t>(prop.sharedMemPerBlockOptin);
+    }
+    if (!s.is_int8 && c->sdpa.p_out_pos >= 0) tc = false;   // the bf16 tcgen05 kernels never form normalised P
     if (s.is_int8)
       // Q must be exactly centred (s8 / zero point 0, or u8 / zero point 128); a zero point on K only
       // shifts every score of a row by the same amount, which softmax cancels
       tc = tc && s.zp_p == 0 && ((s.q_signed && s.zp_q == 0) || (!s.q_signed && s.zp_q == 128));
     if (!tc && s.S > 8192) return bail(fail(GC_ERR_UNSUPPORTED, "attention: sequence length %d not supported", s.S));
     c->sdpa.use_tc = tc;
+    c->sdpa.wide = tc && wide;
     c->launches = 1;
     snprintf(line, sizeof(line), "pattern=attention %s B=%d H=%d S=%d D=%d kernel=%s\n", s.is_int8 ? "int8" : "bf16", s.B,
-             s.H, s.S, s.D, tc ? "tcgen05" : "cuda-core");
+             s.H, s.S, s.D, tc ? (wide ? "tcgen05.streaming" : "tcgen05") : "cuda-core");
     c->desc = line;
   } else {
     gc_status_t st = match_mlp(*p, *c);
@@ -1004,6 +1011,22 @@ static gc_status_t run_sdpa(gc_compiled& c, cudaStream_t st, const void* const* 
   const int dt = prm.is_int8 ? GC_U8 : GC_BF16;
   const int esz = prm.is_int8 ? 1 : 2;
   const uint64_t rows = static_cast<uint64_t>(prm.B) * prm.H * prm.S;
+  if (s.wide) {
+    int box = 0, swz = 0;
+    sdpa_wide_box(prm.D, prm.is_int8, &box, &swz);
+    const void* ptrs[3] = {prm.Q, prm.K, prm.V};
+    const void** cached[3] = {&s.q_ptr, &s.k_ptr, &s.v_ptr};
+    CUtensorMap* maps[3] = {&s.tmQ, &s.tmK, &s.tmV};
+    for (int i = 0; i < 3; ++i) {
+      if (*cached[i] == ptrs[i]) continue;
+      // a box wider than the head (D = 96) reads zeros past the tensor's edge
+      gc_status_t r = make_tmap(maps[i], ptrs[i], dt, prm.D, rows, static_cast<uint64_t>(prm.D) * esz, box, 128, swz);
+      if (r != GC_OK) return r;
+      *cached[i] = ptrs[i];
+    }
+    CUDA_TRY(launch_sdpa_wide(s.tmQ, s.tmK, s.tmV, prm, c.num_sms, st));
+    return GC_OK;
+  }
   const int swz = prm.is_int8 ? 64 : 128;
   if (s.q_ptr != prm.Q) {
     gc_status_t r = make_tmap(&s.tmQ, prm.Q, dt, prm.D, rows, static_cast<uint64_t>(prm.D) * esz, prm.D, 128, swz);

@@ -146,6 +146,13 @@ cudaError_t launch_gemm_tc2(int kind, int a_signed, const CUtensorMap& tmA, cons
                             const GemmTcParams& p, int grid, bool pdl, cudaStream_t s);
 
 size_t sdpa_tc_smem_bytes(int S, int is_int8);
+// Streaming attention kernel (head dimension 64 / 96 / 128, up to 512 keys): dynamic shared memory it needs
+// (0 = shape not supported), the TMA box (elements per row, swizzle bytes) its Q / K / V tensor maps must use
+// (128 rows per box), and the launcher.
+size_t sdpa_wide_smem_bytes(int S, int D, int is_int8);
+void sdpa_wide_box(int D, int is_int8, int* box_elems, int* swizzle_bytes);
+cudaError_t launch_sdpa_wide(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const SdpaParams& p,
+                             int num_sms, cudaStream_t s);
 // tmO: output [B*H*S, 64] with a [32 rows x 64 columns] box, swizzle = row bytes (64 for 8-bit, 128 for bf16)
 cudaError_t launch_sdpa_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmO,
                            const SdpaParams& p, int num_sms, cudaStream_t s);

@@ -213,6 +213,49 @@ def test_mha_bf16(B, b, h, s, d):
     assert np.abs(bf16_to_f64(got) - oracle(w)).max() <= 2e-2
 
 
+# the other head dimensions and sequence lengths of the evaluation's workload table, on the streaming kernel;
+# the larger cases give every CTA more than one work unit, so the rings and barrier phases wrap
+WIDE_SHAPES = [(1, 2, 128, 96), (1, 2, 384, 128), (1, 2, 512, 64), (2, 1, 256, 128), (1, 1, 512, 128), (1, 1, 256, 96),
+               (4, 40, 128, 96), (2, 30, 384, 128), (1, 50, 512, 64)]
+
+
+@pytest.mark.parametrize("b,h,s,d", WIDE_SHAPES)
+def test_mha_bf16_streaming_kernel(B, b, h, s, d):
+    w = W.mha_bf16(batch=b, heads=h, seq=s, head_dim=d)
+    got, plan = run_gpu(B, w)
+    assert "tcgen05.streaming" in plan
+    assert np.abs(bf16_to_f64(got) - oracle(w)).max() <= 2e-2
+
+
+@pytest.mark.parametrize("b,h,s,d", WIDE_SHAPES)
+def test_mha_int8_streaming_kernel(B, b, h, s, d):
+    w = W.mha_int8(batch=b, heads=h, seq=s, head_dim=d)
+    got, plan = run_gpu(B, w)
+    assert "tcgen05.streaming" in plan
+    check_int8_attention(got, oracle(w))
+
+
+def test_mha_int8_streaming_kernel_stages_around_the_softmax(B):
+    import torch
+    w = W.mha_int8(batch=2, heads=2, seq=512, head_dim=64, seed=9)
+    g = w.graph
+    g.mark_output(w.info["p_quant"])
+    c = B.CompiledPartition(g, 0)
+    assert "tcgen05.streaming" in c.plan
+    ins = B.device_inputs(w)
+    outs = B.device_outputs(g)
+    c.execute(ins, outs)
+    c.query_status()
+    torch.cuda.synchronize()
+    o_gpu = B.output_to_numpy(g, g.outputs[0], outs[0]).copy()
+    p_gpu = B.output_to_numpy(g, g.outputs[1], outs[1]).copy()
+    c.close()
+    ref = interp.run(g, w.feeds)
+    dp = np.abs(p_gpu.astype(np.int64) - ref[g.outputs[1]])
+    assert dp.max() <= 1 and (dp != 0).mean() <= 1e-3
+    assert_stage_after_softmax_exact(w, o_gpu, p_gpu)
+
+
 def test_mha_bf16_generic_kernel(B):
     w = W.mha_bf16(batch=2, heads=2, seq=128, head_dim=64)
     got, plan = run_gpu(B, w, force_generic=True)
