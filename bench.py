@@ -202,12 +202,14 @@ def sweep_cases():
     return cases
 
 
-def run_sweep(B, device, peaks):
+def run_sweep(B, device, peaks, only=""):
     """One line per shape: cold time (rotating replicas above the L2 size), kernels chosen, HBM-roofline time."""
     import torch
     out = []
     stream = torch.cuda.current_stream(device).cuda_stream
     for label, make in sweep_cases():
+        if only and only not in label:
+            continue
         w = make()
         first = Replica(B, w, 0, device)
         n_rep = int(min(32, max(2, -(-int(1.25 * L2_BYTES) // first.bytes))))
@@ -323,6 +325,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the headline run, time every shape of the evaluation's workload table (1 GPU)")
+    ap.add_argument("--sweep-filter", default="", help="with --sweep: only the cases whose name contains this text")
     args = ap.parse_args()
     if args.impl == "reference":
         if args.steps == 0:
@@ -360,7 +363,7 @@ def main():
     peaks, peak_src = load_peaks()
     if args.sweep:
         if rank == 0:
-            print(json.dumps({"sweep": run_sweep(B, local, peaks), "unit": "us per subgraph, cold L2", "data": "synthetic"}))
+            print(json.dumps({"sweep": run_sweep(B, local, peaks, args.sweep_filter), "unit": "us per subgraph, cold L2", "data": "synthetic"}))
         if world > 1:
             dist.barrier()
             dist.destroy_process_group()
@@ -368,7 +371,7 @@ def main():
     head = args.workload
     names = [head] if args.only else [head] + [n for n in W.CONFIGS if n != head]
     results = {}
-    floor_us = launch_floor_us(B, local) if rank == 0 else 0.0
+    floor_us = launch_floor_us(B, local) if (rank == 0 and not args.only) else 0.0
     sm_max_mhz = 1965.0
     clocks = None
     launches_total = 0

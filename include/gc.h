@@ -122,7 +122,10 @@ typedef struct {
                              (ablation / debugging; results obey the same contracts) */
   int32_t no_chain_fusion;/* 1: one launch per fused op with full stream ordering between them, the
                              analogue of running with coarse-grain fusion disabled (Section VII) */
-  int32_t reserved[6];
+  int32_t streaming_attention; /* 1: attention always runs on the streaming tcgen05 kernel (K/V and P rings),
+                             also for the shapes (head dimension 64, up to 384 keys) that by default use the
+                             kernel with resident K/V (ablation) */
+  int32_t reserved[5];
 } gc_compile_options_t;
 
 typedef struct gc_partition gc_partition_t;

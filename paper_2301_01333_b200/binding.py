@@ -49,7 +49,8 @@ class gc_op_t(C.Structure):
 
 
 class gc_compile_options_t(C.Structure):
-    _fields_ = [("force_generic", C.c_int32), ("no_chain_fusion", C.c_int32), ("reserved", C.c_int32 * 6)]
+    _fields_ = [("force_generic", C.c_int32), ("no_chain_fusion", C.c_int32), ("streaming_attention", C.c_int32),
+                ("reserved", C.c_int32 * 5)]
 
 
 class GcError(RuntimeError):
@@ -161,11 +162,13 @@ def gc_partition_destroy(p) -> None:
     load_library().gc_partition_destroy(p)
 
 
-def gc_compile(p, cuda_device: int = 0, force_generic: bool = False, no_chain_fusion: bool = False) -> C.c_void_p:
+def gc_compile(p, cuda_device: int = 0, force_generic: bool = False, no_chain_fusion: bool = False,
+               streaming_attention: bool = False) -> C.c_void_p:
     lib = load_library()
     opt = gc_compile_options_t()
     opt.force_generic = int(force_generic)
     opt.no_chain_fusion = int(no_chain_fusion)
+    opt.streaming_attention = int(streaming_attention)
     h = C.c_void_p()
     _check(lib.gc_compile(p, cuda_device, C.byref(opt), C.byref(h)))
     return h
@@ -238,13 +241,14 @@ def gc_matmul_s32_noalloc(stream: int, a_ptr: int, w_ptr: int, out_ptr: int, m: 
 class CompiledPartition:
     """Convenience owner: partition + compiled object + torch-allocated workspace."""
 
-    def __init__(self, g: Graph, device: int = 0, force_generic: bool = False, no_chain_fusion: bool = False):
+    def __init__(self, g: Graph, device: int = 0, force_generic: bool = False, no_chain_fusion: bool = False,
+                 streaming_attention: bool = False):
         import torch
         self.graph = g
         self.device = device
         self._part = gc_partition_create(g)
         try:
-            self._comp = gc_compile(self._part, device, force_generic, no_chain_fusion)
+            self._comp = gc_compile(self._part, device, force_generic, no_chain_fusion, streaming_attention)
         except Exception:
             gc_partition_destroy(self._part)
             self._part = None

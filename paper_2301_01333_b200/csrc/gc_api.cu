@@ -621,7 +621,7 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
     if (st != GC_OK) return bail(st);
     c->pattern = PAT_SDPA;
     SdpaParams& s = c->sdpa.prm;
-    bool tc = !c->opt.force_generic && s.D == 64 && s.S % 128 == 0 && s.S <= 384 &&
+    bool tc = !c->opt.force_generic && !c->opt.streaming_attention && s.D == 64 && s.S % 128 == 0 && s.S <= 384 &&
               sdpa_tc_smem_bytes(s.S, s.is_int8) <= static_cast<size_t>(prop.sharedMemPerBlockOptin);
     bool wide = false;
     if (!tc && !c->opt.force_generic) {

@@ -6,8 +6,11 @@
 // (512 keys).  That is what lets 128-wide heads and 512-key rows fit in 227 KB of shared memory.
 //
 // Persistent CTAs (one per SM, 704 threads) walk over work units (batch, head, 128-query tile):
-//   warp 0      TMA producer: Q tile, then K blocks 0..NB-1, then V blocks 0..NB-1 into the ring (no multicast)
-//   warp 1      MMA issuer (one thread): S_b = Q K_b^T per block, then O += P_b V_b per block
+//   warp 0      TMA producer: Q tile and 128-key blocks of K and V into the ring, in the order the MMA issuer
+//               consumes them (no multicast)
+//   warp 1      MMA issuer (one thread): S_b = Q K_b^T per block, O += P_b V_b per block; unless O shares
+//               columns with the scores, the next unit's S_b is issued right after this unit's P_b V_b, as
+//               soon as the softmax warps have released block b
 //   warps 2-5   per-unit preparation (mask row times log2(e), chunk flags, u8 -> s8 flip of Q) and the epilogue
 //               of the previous unit (O out of tensor memory, normalise or requantise, vector stores)
 //   warps 6-21  softmax, four threads per query row, 32 of every 128 key columns each (two passes)
@@ -177,22 +180,35 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (lane == 0) {
       int n = 0;
       uint32_t it = 0;                                          // ring position: stage it % stages, use it / stages
-      for (int unit = blockIdx.x; unit < num_units && !failed; unit += gridDim.x, ++n) {
-        const int bh = unit / q_tiles, qt = unit % q_tiles;
-        if (!mbar_wait(bar_q_empty, (n & 1) ^ 1)) { failed = true; break; }
+      auto load_q = [&](int u, int nn) -> bool {                 // Q tile of unit u, this CTA's nn-th unit
+        if (!mbar_wait(bar_q_empty, (nn & 1) ^ 1)) return false;
         mbar_arrive_expect_tx(bar_q_full, static_cast<uint32_t>(L::TILE_BYTES));
         for (int j = 0; j < L::NSUB; ++j)
-          tma_load_2d(smem_u32(sQ) + j * L::SUB_BYTES, &tmQ, j * L::SUB_ELEMS, bh * S + qt * W_BLOCK_Q, bar_q_full);
-        for (int kv = 0; kv < 2 && !failed; ++kv) {
-          const CUtensorMap* tm = kv == 0 ? &tmK : &tmV;
-          for (int b = 0; b < NB; ++b, ++it) {
-            const uint32_t st = it % stages, use = it / stages;
-            if (!mbar_wait(bar_kv_empty + 8 * st, (use & 1) ^ 1)) { failed = true; break; }
-            mbar_arrive_expect_tx(bar_kv_full + 8 * st, static_cast<uint32_t>(L::TILE_BYTES));
-            for (int j = 0; j < L::NSUB; ++j)
-              tma_load_2d(smem_u32(sKV) + st * L::TILE_BYTES + j * L::SUB_BYTES, tm, j * L::SUB_ELEMS, bh * S + b * 128,
-                          bar_kv_full + 8 * st);
-          }
+          tma_load_2d(smem_u32(sQ) + j * L::SUB_BYTES, &tmQ, j * L::SUB_ELEMS,
+                      (u / q_tiles) * S + (u % q_tiles) * W_BLOCK_Q, bar_q_full);
+        return true;
+      };
+      auto load_block = [&](const CUtensorMap* tm, int u, int b) -> bool {   // one 128-key block into the next stage
+        const uint32_t st = it % stages, use = it / stages;
+        ++it;
+        if (!mbar_wait(bar_kv_empty + 8 * st, (use & 1) ^ 1)) return false;
+        mbar_arrive_expect_tx(bar_kv_full + 8 * st, static_cast<uint32_t>(L::TILE_BYTES));
+        for (int j = 0; j < L::NSUB; ++j)
+          tma_load_2d(smem_u32(sKV) + st * L::TILE_BYTES + j * L::SUB_BYTES, tm, j * L::SUB_ELEMS, (u / q_tiles) * S + b * 128,
+                      bar_kv_full + 8 * st);
+        return true;
+      };
+      for (int unit = blockIdx.x; unit < num_units && !failed; unit += gridDim.x, ++n) {
+        const int next = unit + static_cast<int>(gridDim.x);
+        const bool ahead = !alias && next < num_units;          // next unit's K blocks interleaved with my V blocks
+        if (alias || n == 0) {
+          failed = !load_q(unit, n);
+          for (int b = 0; b < NB && !failed; ++b) failed = !load_block(&tmK, unit, b);
+        }
+        if (ahead && !failed) failed = !load_q(next, n + 1);
+        for (int b = 0; b < NB && !failed; ++b) {
+          failed = !load_block(&tmV, unit, b);
+          if (ahead && !failed) failed = !load_block(&tmK, next, b);
         }
       }
       if (failed) report(p.status, DEV_TIMEOUT_PRODUCER);
@@ -214,12 +230,14 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       uint32_t it = 0;
       for (int unit = blockIdx.x; unit < num_units && !failed; unit += gridDim.x, ++n) {
         const uint32_t upar = n & 1;
-        if (!mbar_wait(bar_q_ready, upar)) { failed = true; break; }
-        // S_b = Q K_b^T
-        for (int b = 0; b < NB; ++b, ++it) {
-          const uint32_t st = it % stages, use = it / stages;
-          if (!mbar_wait(bar_kv_full + 8 * st, use & 1) || !mbar_wait(bar_s_free + 8 * b, upar ^ 1)) { failed = true; break; }
-          if (alias && b == 0 && !mbar_wait(bar_o_free, upar ^ 1)) { failed = true; break; }
+        const bool ahead = !alias && unit + static_cast<int>(gridDim.x) < num_units;
+        // S_b = Q K_b^T for this CTA's nn-th unit (block b of the ring's next stage)
+        auto mma1 = [&](int nn, int b) -> bool {
+          const uint32_t st = it % stages, use = it / stages, par = nn & 1;
+          ++it;
+          if (b == 0 && !mbar_wait(bar_q_ready, par)) return false;
+          if (!mbar_wait(bar_kv_full + 8 * st, use & 1) || !mbar_wait(bar_s_free + 8 * b, par ^ 1)) return false;
+          if (alias && b == 0 && !mbar_wait(bar_o_free, par ^ 1)) return false;
           tc_fence_after();
           const uint32_t kb = smem_u32(sKV) + st * L::TILE_BYTES;
 #pragma unroll
@@ -230,12 +248,16 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           }
           umma_commit(bar_s_full + 8 * b);
           umma_commit(bar_kv_empty + 8 * st);
-        }
+          if (b == NB - 1) umma_commit(bar_q_empty);
+          return true;
+        };
+        if (alias || n == 0)
+          for (int b = 0; b < NB && !failed; ++b) failed = !mma1(n, b);
         if (failed) break;
-        umma_commit(bar_q_empty);
         // O += P_b V_b
-        for (int b = 0; b < NB; ++b, ++it) {
+        for (int b = 0; b < NB; ++b) {
           const uint32_t st = it % stages, use = it / stages;
+          ++it;
           const uint32_t pe = static_cast<uint32_t>(n * NB + b) % np;
           if (!mbar_wait(bar_p_full + 8 * b, upar) || !mbar_wait(bar_kv_full + 8 * st, use & 1)) { failed = true; break; }
           if (!alias && b == 0 && !mbar_wait(bar_o_free, upar ^ 1)) { failed = true; break; }
@@ -257,6 +279,7 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           umma_commit(bar_kv_empty + 8 * st);
           umma_commit(bar_p_free + 8 * pe);
           if (b == NB - 1) umma_commit(bar_o_full);
+          if (ahead && !mma1(n + 1, b)) { failed = true; break; }
         }
       }
       if (failed) report(p.status, DEV_TIMEOUT_MMA);
