@@ -854,6 +854,7 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
     cp.status = status;
     cp.barrier = reinterpret_cast<unsigned long long*>(ws + 64);
     cp.barrier_base = c.chain_arrivals;
+    cp.early_weights = need ? 0 : 1;
     const LayerPlan& L0 = c.layers[0];
     const void* a0 = in[L0.a_input];
     if (L0.need_pack) {
@@ -965,7 +966,9 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
         if (s != GC_OK) return s;
         L.tmD_ptr = O;
       }
-      const bool pdl = !c.opt.no_chain_fusion && l > 0 && !L.need_pack;
+      // Programmatic dependent launch, also for the first layer: whatever ran before on the stream, this kernel's
+      // set-up overlaps its tail and the kernel waits for it to complete before it touches global memory
+      const bool pdl = !c.opt.no_chain_fusion && !L.need_pack;
       if (L.cta2)
         CUDA_TRY(launch_gemm_tc2(L.kind, L.a_dtype == GC_S8, L.tmA, L.tmB, L.tmD, g, L.grid, pdl, st));
       else

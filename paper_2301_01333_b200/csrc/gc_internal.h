@@ -110,6 +110,8 @@ struct ChainParams {
   int64_t pack_src_pitch, pack_dst_pitch;   // bytes
   unsigned long long* barrier;              // grid-barrier counter (only grows)
   unsigned long long barrier_base;          // its value before this launch
+  int early_weights;                        // 1: the prepacked weights were written by an earlier call, so their loads
+                                            // need not wait for the kernel that precedes this one on the stream
   uint32_t* status;
   // TMA descriptors travel in the kernel parameter space (fetched once, cached by the TMA unit); descriptors
   // kept in global memory cost a fetch of several hundred clocks on every load instruction.

@@ -108,6 +108,12 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  // Programmatic dependent launch: everything above may overlap the tail of the preceding kernel on the stream.
+  // The prepacked weights are constants; unless this very call has just enqueued their prepack, their loads may
+  // start before the preceding kernel has finished, too.  Everything else waits for it.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (!p.early_weights) asm volatile("griddepcontrol.wait;" ::: "memory");
+
   // every layer's weight slice starts moving now (constants: they do not depend on earlier layers)
   if (warp == 0 && lane == 0) {
     for (int l = 0; l < p.n_layers; ++l) {
@@ -119,6 +125,8 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
                     cta * CH_BLOCK_N, bar_wfull + 8 * l);
     }
   }
+
+  if (p.early_weights) asm volatile("griddepcontrol.wait;" ::: "memory");
 
   bool failed = false;
   unsigned long long bar_count = p.barrier_base;                  // counter value before this launch
@@ -297,8 +305,13 @@ cudaError_t launch_mlp_chain(int kind, const ChainParams& p, int grid, cudaStrea
   // No cooperative-launch attribute: it costs tens of microseconds per launch, more than the whole chain.
   // The grid is at most one CTA per SM, so its CTAs become resident together whenever the SMs are free; if
   // they are not, the waiting CTAs only wait for unrelated work to finish, and every spin is bounded anyway.
-  cfg.attrs = nullptr;
-  cfg.numAttrs = 0;
+  // Programmatic dependent launch: the set-up may overlap the tail of whatever precedes on the stream; the
+  // kernel waits for that work to complete before its first global access.
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   void* args[] = {const_cast<ChainParams*>(&p)};
   return cudaLaunchKernelExC(&cfg, kern, args);
 }

@@ -168,6 +168,11 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  // Programmatic dependent launch: the set-up above may overlap the tail of the preceding kernel on the stream;
+  // nothing below touches global memory before that kernel has completed (no-op for an ordinary launch).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
   bool failed = false;
   auto slot_q = [&](int s) { return sSlots + s * L::slot_bytes(S); };
   auto slot_k = [&](int s) { return slot_q(s) + L::q_bytes(); };
@@ -464,14 +469,16 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       uint8_t* sP = sPall + buf * L::p_bytes(S);
       if (!mbar_wait(bar_kv_ready + 8 * s, (n / slots) & 1)) { failed = true; break; }
       // Mask-aware skipping (int8): with at least one unmasked key in the row, a chunk whose keys are all
-      // masked has exponentials that underflow to exactly zero, so neither pass touches it: its codes are zero.
-      uint32_t skip = 0;                                        // bit b: my chunk of key block b is skipped
+      // masked has exponentials that underflow to exactly zero, so neither pass needs to touch it: its codes are
+      // zero.  Only the trailing run of such chunks is left out (a padding mask is a valid-length prefix), which
+      // keeps the two passes free of per-chunk branches: they simply run over fewer blocks.
+      int nbp = NB;                                             // my chunks of key blocks nbp .. NB-1 are skipped
       if constexpr (INT8) {
         const uint32_t* fl = sChunk + s * 16;
         bool any_valid = false;
         for (int i = 0; i < NB * 4; ++i) any_valid = any_valid || fl[i] == 2u;
         if (any_valid)
-          for (int b = 0; b < NB; ++b) skip |= (fl[b * 4 + g] == 1u ? 1u : 0u) << b;
+          while (nbp > 0 && fl[(nbp - 1) * 4 + g] == 1u) --nbp;
       }
 
       // ---------------- pass A: one 32-column chunk per key block, transformed in place
@@ -479,12 +486,8 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       float m = -INFINITY, l = 0.f;
       float mc[3] = {0.f, 0.f, 0.f};                            // running max after each block (int8)
       uint32_t v[32];
-      for (int b = 0; b < NB; ++b) {
+      for (int b = 0; b < nbp; ++b) {
         const int col = b * 128 + g * 32;
-        if (INT8 && ((skip >> b) & 1u)) {
-          if (b == 0) mc[0] = m; else if (b == 1) mc[1] = m; else mc[2] = m;
-          continue;
-        }
         if (!mbar_wait(bar_s_full + 8 * bx(buf, b), fpar)) { failed = true; break; }
         tc_fence_after();
         if constexpr (INT8) tmem_wait_st();                     // v[] may still feed the previous block's store
@@ -545,14 +548,10 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       // ---------------- pass B: normalise, round, write P
       int psum = 0;
       float lsum = 0.f;
-      for (int b = 0; b < NB; ++b) {
+      for (int b = 0; b < nbp; ++b) {
         const int col = b * 128 + g * 32;
         if constexpr (INT8) {
           uint32_t w[8];
-          if ((skip >> b) & 1u) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) w[i] = 0u;
-          } else {
           tmem_ld32(t_row + col, v);
           tmem_wait_ld();
           const float f = ex2((b == 0 ? mc[0] : b == 1 ? mc[1] : mc[2]) - M) * scale;
@@ -566,7 +565,6 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             const uint32_t y3 = __float_as_uint(fmaf(__uint_as_float(v[4 * i + 3]), f, MAGIC_F));
             w[i] = __byte_perm(__byte_perm(y0, y1, 0x0040), __byte_perm(y2, y3, 0x0040), 0x5410);
             psum = static_cast<int>(__dp4a(w[i], 0x01010101u, static_cast<unsigned>(psum)));
-          }
           }
           uint8_t* blk = sP + b * P_BLOCK_BYTES + row_off;
           const int c0 = g * 2;                                 // 16-byte chunk index inside the 128-byte row
@@ -623,6 +621,28 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           mbar_arrive(bar_s_free + 8 * bx(buf, b));
         }
       }
+      if constexpr (INT8) {
+        for (int b = nbp; b < NB; ++b) {                        // skipped chunks: their codes are zero
+          const int col = b * 128 + g * 32;
+          uint8_t* blk = sP + b * P_BLOCK_BYTES + row_off;
+          const int c0 = g * 2;
+          *reinterpret_cast<uint4*>(blk + (((c0 + 0) ^ (r & 7)) * 16)) = make_uint4(0u, 0u, 0u, 0u);
+          *reinterpret_cast<uint4*>(blk + (((c0 + 1) ^ (r & 7)) * 16)) = make_uint4(0u, 0u, 0u, 0u);
+          if (p.P_out) {
+            const int64_t grow = static_cast<int64_t>(unit / q_tiles) * S + (unit % q_tiles) * SDPA_BLOCK_Q + r;
+            uint4* po = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.P_out) + grow * S + col);
+            po[0] = make_uint4(0u, 0u, 0u, 0u);
+            po[1] = make_uint4(0u, 0u, 0u, 0u);
+          }
+          fence_proxy_async_smem();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) {
+            mbar_arrive(bar_p_full + 8 * bx(buf, b));
+            mbar_arrive(bar_s_free + 8 * bx(buf, b));
+          }
+        }
+      }
       // my part of the row sum goes to the auxiliary warps, which finish and store the output; the slot is
       // free once they have read the sums of the unit that used it two units ago
       if (!mbar_wait(bar_st_free + 8 * upar, ((n >> 1) & 1) ^ 1)) { failed = true; break; }
@@ -652,17 +672,25 @@ cudaError_t launch_sdpa_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const
   if (!cfg.slots) return cudaErrorInvalidValue;
   const int units = p.B * p.H * (p.S / SDPA_BLOCK_Q);
   const int grid = units < num_sms ? units : num_sms;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(grid);
+  lc.blockDim = dim3(SDPA_THREADS);
+  lc.dynamicSmemBytes = cfg.smem;
+  lc.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = attr;
+  lc.numAttrs = 1;
   cudaError_t e;
   if (p.is_int8) {
     e = cudaFuncSetAttribute(sdpa_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(cfg.smem));
     if (e != cudaSuccess) return e;
-    sdpa_tc_kernel<true><<<grid, SDPA_THREADS, cfg.smem, s>>>(tmQ, tmK, tmV, tmO, p, cfg.slots, cfg.nsb, cfg.stage_out);
-  } else {
-    e = cudaFuncSetAttribute(sdpa_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(cfg.smem));
-    if (e != cudaSuccess) return e;
-    sdpa_tc_kernel<false><<<grid, SDPA_THREADS, cfg.smem, s>>>(tmQ, tmK, tmV, tmO, p, cfg.slots, cfg.nsb, cfg.stage_out);
+    return cudaLaunchKernelEx(&lc, sdpa_tc_kernel<true>, tmQ, tmK, tmV, tmO, p, cfg.slots, cfg.nsb, cfg.stage_out);
   }
-  return cudaGetLastError();
+  e = cudaFuncSetAttribute(sdpa_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(cfg.smem));
+  if (e != cudaSuccess) return e;
+  return cudaLaunchKernelEx(&lc, sdpa_tc_kernel<false>, tmQ, tmK, tmV, tmO, p, cfg.slots, cfg.nsb, cfg.stage_out);
 }
 
 }  // namespace gc

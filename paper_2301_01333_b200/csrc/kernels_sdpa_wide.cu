@@ -173,6 +173,11 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  // Programmatic dependent launch: the set-up above may overlap the tail of the preceding kernel on the stream;
+  // nothing below touches global memory before that kernel has completed (no-op for an ordinary launch).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
   bool failed = false;
 
   if (warp == 0) {
@@ -435,25 +440,21 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       const float* mk = sMask + (n & 1) * S;
       const uint32_t upar = n & 1;
       if (!mbar_wait(bar_q_ready, upar)) { failed = true; break; }
-      uint32_t skip = 0;                                        // bit b: my chunk of key block b is skipped
+      int nbp = NB;                                             // my chunks of key blocks nbp .. NB-1 are skipped
       if constexpr (INT8) {
         const uint32_t* fl = sChunk + (n & 1) * 16;
         bool any_valid = false;
         for (int i = 0; i < NB * 4; ++i) any_valid = any_valid || fl[i] == 2u;
         if (any_valid)
-          for (int b = 0; b < NB; ++b) skip |= (fl[b * 4 + g] == 1u ? 1u : 0u) << b;
+          while (nbp > 0 && fl[(nbp - 1) * 4 + g] == 1u) --nbp;
       }
 
       // ---------------- pass A: scale + mask, running row max [int8: exp2 and running sum, written back]
       float m = -INFINITY, l = 0.f;
       float mc[4] = {0.f, 0.f, 0.f, 0.f};                       // running max after each block (int8)
       uint32_t v[32];
-      for (int b = 0; b < NB; ++b) {
+      for (int b = 0; b < nbp; ++b) {
         const int col = b * 128 + g * 32;
-        if (INT8 && ((skip >> b) & 1u)) {
-          if (b == 0) mc[0] = m; else if (b == 1) mc[1] = m; else if (b == 2) mc[2] = m; else mc[3] = m;
-          continue;
-        }
         if (!mbar_wait(bar_s_full + 8 * b, upar)) { failed = true; break; }
         tc_fence_after();
         if constexpr (INT8) tmem_wait_st();                     // v[] may still feed the previous block's store
@@ -514,17 +515,14 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       // ---------------- pass B: normalise, round, write P into the ring
       int psum = 0;
       float lsum = 0.f;
-      for (int b = 0; b < NB; ++b) {
+      for (int b = 0; b < nbp; ++b) {
         const int col = b * 128 + g * 32;
         const uint32_t pseq = static_cast<uint32_t>(n * NB + b);
         const uint32_t pe = pseq % np, puse = pseq / np;
         uint8_t* sP = sPall + pe * L::P_BYTES;
         if constexpr (INT8) {
           uint32_t w[8];
-          if ((skip >> b) & 1u) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) w[i] = 0u;
-          } else {
+          {
             tmem_ld32(t_row + col, v);
             tmem_wait_ld();
             const float f = w_ex2((b == 0 ? mc[0] : b == 1 ? mc[1] : b == 2 ? mc[2] : mc[3]) - M) * scale;
@@ -597,6 +595,32 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         }
       }
       if (failed) break;
+      if constexpr (INT8) {
+        for (int b = nbp; b < NB; ++b) {                        // skipped chunks: their codes are zero
+          const int col = b * 128 + g * 32;
+          const uint32_t pseq = static_cast<uint32_t>(n * NB + b);
+          const uint32_t pe = pseq % np, puse = pseq / np;
+          if (!mbar_wait(bar_p_free + 8 * pe, (puse & 1) ^ 1)) { failed = true; break; }
+          uint8_t* blk = sPall + pe * L::P_BYTES + row_off;
+          const int c0 = g * 2;
+          *reinterpret_cast<uint4*>(blk + (((c0 + 0) ^ (r & 7)) * 16)) = make_uint4(0u, 0u, 0u, 0u);
+          *reinterpret_cast<uint4*>(blk + (((c0 + 1) ^ (r & 7)) * 16)) = make_uint4(0u, 0u, 0u, 0u);
+          if (p.P_out) {
+            const int64_t grow = static_cast<int64_t>(unit / q_tiles) * S + (unit % q_tiles) * W_BLOCK_Q + r;
+            uint4* po = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.P_out) + grow * S + col);
+            po[0] = make_uint4(0u, 0u, 0u, 0u);
+            po[1] = make_uint4(0u, 0u, 0u, 0u);
+          }
+          fence_proxy_async_smem();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) {
+            mbar_arrive(bar_p_full + 8 * b);
+            mbar_arrive(bar_s_free + 8 * b);
+          }
+        }
+        if (failed) break;
+      }
       // my part of the row sum goes to the auxiliary warps, which finish and store the output; the slot is
       // free once they have read the sums of the unit that used it two units ago
       if (!mbar_wait(bar_st_free + 8 * upar, ((n >> 1) & 1) ^ 1)) { failed = true; break; }
@@ -630,8 +654,17 @@ cudaError_t launch_wide_t(const CUtensorMap& tmQ, const CUtensorMap& tmK, const 
   cudaError_t e = cudaFuncSetAttribute(sdpa_wide_kernel<INT8, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(cfg.smem));
   if (e != cudaSuccess) return e;
-  sdpa_wide_kernel<INT8, D><<<grid, W_THREADS, cfg.smem, s>>>(tmQ, tmK, tmV, p, cfg.np, cfg.stages);
-  return cudaGetLastError();
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(grid);
+  lc.blockDim = dim3(W_THREADS);
+  lc.dynamicSmemBytes = cfg.smem;
+  lc.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+  return cudaLaunchKernelEx(&lc, sdpa_wide_kernel<INT8, D>, tmQ, tmK, tmV, p, cfg.np, cfg.stages);
 }
 
 }  // namespace
