@@ -179,6 +179,8 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   auto slot_v = [&](int s) { return slot_k(s) + L::kv_bytes(S); };
   // Unit n of this CTA uses score/output buffer buf(n); it is that buffer's cnt(n)-th use.  With one
   // buffer the per-key-block barriers are indexed by block, with two (one block per unit) by buffer.
+  auto slot_of = [&](int n) { return slots == 2 ? (n & 1) : 0; };   // slots is 1 or 2: no division needed
+  auto use_of = [&](int n) { return slots == 2 ? (n >> 1) : n; };
   auto buf_of = [&](int n) { return nsb == 2 ? (n & 1) : 0; };
   auto cnt_of = [&](int n) { return nsb == 2 ? (n >> 1) : n; };
   auto bx = [&](int buf, int b) { return nsb == 2 ? buf : b; };
@@ -188,8 +190,8 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     if (lane == 0) {
       int n = 0;
       for (int unit = blockIdx.x; unit < num_units; unit += gridDim.x, ++n) {
-        const int s = n % slots;
-        const uint32_t par = (n / slots) & 1;
+        const int s = slot_of(n);
+        const uint32_t par = use_of(n) & 1;
         if (!mbar_wait(bar_kv_empty + 8 * s, par ^ 1)) {
           report(p.status, DEV_TIMEOUT_PRODUCER);
           failed = true;
@@ -215,7 +217,7 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       constexpr int K2_STEPS = 128 / (INT8 ? 32 : 16);          // MMAs per 128-key block of P.V
       // S[:, 128b .. 128b+127] = Q K_b^T for unit n1 (waits until the softmax warps have released the columns)
       auto mma1 = [&](int n1, int b) -> bool {
-        const int s = n1 % slots, buf = buf_of(n1);
+        const int s = slot_of(n1), buf = buf_of(n1);
         if (!mbar_wait(bar_s_free + 8 * bx(buf, b), (cnt_of(n1) & 1) ^ 1)) return false;
         tc_fence_after();
         const uint64_t a_desc = make_smem_desc(smem_u32(slot_q(s)), 16, SBO, SWZ);
@@ -228,7 +230,7 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         return true;
       };
       auto mma2 = [&](int n0, int b) {                          // O += P_b V_b for unit n0
-        const int s = n0 % slots, buf = buf_of(n0);
+        const int s = slot_of(n0), buf = buf_of(n0);
         const uint32_t sP = smem_u32(sPall) + buf * L::p_bytes(S);
 #pragma unroll
         for (int ks = 0; ks < K2_STEPS; ++ks) {
@@ -242,13 +244,13 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         }
       };
       auto wait_inputs = [&](int n1) -> bool {
-        const int s = n1 % slots;
-        const uint32_t par = (n1 / slots) & 1;
+        const int s = slot_of(n1);
+        const uint32_t par = use_of(n1) & 1;
         return mbar_wait(bar_kv_ready + 8 * s, par) && mbar_wait(bar_kv_full + 8 * s, par);
       };
       int n = 0;
       for (int unit = blockIdx.x; unit < num_units && !failed; unit += gridDim.x, ++n) {
-        const int s = n % slots, buf = buf_of(n);
+        const int s = slot_of(n), buf = buf_of(n);
         const uint32_t fpar = cnt_of(n) & 1;
         const bool has_next = unit + static_cast<int>(gridDim.x) < num_units;
         if (n == 0) {
@@ -393,18 +395,28 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     int n = 0;
     int prev_unit = -1;
     for (int unit = blockIdx.x; unit < num_units && !failed; unit += gridDim.x, ++n) {
-      const int s = n % slots;
+      const int s = slot_of(n);
       const int b = (unit / q_tiles) / p.H;
       float* mk = sMask + s * S;
       // the mask slot is free once the unit that used this slot before has been fully consumed, which
       // the producer's own wait on kv_empty guarantees before kv_full can complete for this unit
-      if (!mbar_wait(bar_kv_full + 8 * s, (n / slots) & 1)) {
+      // the mask values are fetched before the wait so that their latency hides behind the unit's loads
+      float mreg[3];
+#pragma unroll
+      for (int i = 0; i < 3; ++i) {
+        const int j = t + 128 * i;
+        mreg[i] = (p.mask && j < S) ? __ldg(p.mask + static_cast<int64_t>(b) * S + j) * LOG2E : 0.0f;
+      }
+      if (!mbar_wait(bar_kv_full + 8 * s, use_of(n) & 1)) {
         report(p.status, DEV_TIMEOUT_OTHER);
         failed = true;
         break;
       }
-      for (int j = t; j < S; j += 128) {                        // a warp covers one aligned 32-key chunk per step
-        const float mv = p.mask ? __ldg(p.mask + static_cast<int64_t>(b) * S + j) * LOG2E : 0.0f;
+#pragma unroll
+      for (int i = 0; i < 3; ++i) {                             // a warp covers one aligned 32-key chunk per step
+        const int j = t + 128 * i;
+        if (j >= S) break;
+        const float mv = mreg[i];
         mk[j] = mv;
         if constexpr (INT8) {
           const bool all_masked = __all_sync(0xffffffffu, p.skip_thr > 0.f && mv <= -p.skip_thr);
@@ -461,13 +473,13 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 
     int n = 0;
     for (int unit = blockIdx.x; unit < num_units && !failed; unit += gridDim.x, ++n) {
-      const int s = n % slots, buf = buf_of(n);
+      const int s = slot_of(n), buf = buf_of(n);
       const float* mk = sMask + s * S;
       const uint32_t fpar = cnt_of(n) & 1;
       const int upar = n & 1;
       const uint32_t t_row = t_lane + buf * BUF_COLS;
       uint8_t* sP = sPall + buf * L::p_bytes(S);
-      if (!mbar_wait(bar_kv_ready + 8 * s, (n / slots) & 1)) { failed = true; break; }
+      if (!mbar_wait(bar_kv_ready + 8 * s, use_of(n) & 1)) { failed = true; break; }
       // Mask-aware skipping (int8): with at least one unmasked key in the row, a chunk whose keys are all
       // masked has exponentials that underflow to exactly zero, so neither pass needs to touch it: its codes are
       // zero.  Only the trailing run of such chunks is left out (a padding mask is a valid-length prefix), which

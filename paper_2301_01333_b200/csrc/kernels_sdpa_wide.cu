@@ -378,13 +378,23 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       float* mk = sMask + (n & 1) * S;
       // Q(n) lands only after every Q K^T of unit n-1 has completed, which needed the softmax warps to be done
       // with unit n-2: the mask buffer and chunk flags of that unit are free
+      // the mask values are fetched before the wait so that their latency hides behind the unit's loads
+      float mreg[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int j = t + 128 * i;
+        mreg[i] = (p.mask && j < S) ? __ldg(p.mask + static_cast<int64_t>(b) * S + j) * W_LOG2E : 0.0f;
+      }
       if (!mbar_wait(bar_q_full, n & 1)) {
         report(p.status, DEV_TIMEOUT_OTHER);
         failed = true;
         break;
       }
-      for (int j = t; j < S; j += 128) {                        // a warp covers one aligned 32-key chunk per step
-        const float mv = p.mask ? __ldg(p.mask + static_cast<int64_t>(b) * S + j) * W_LOG2E : 0.0f;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {                             // a warp covers one aligned 32-key chunk per step
+        const int j = t + 128 * i;
+        if (j >= S) break;
+        const float mv = mreg[i];
         mk[j] = mv;
         if constexpr (INT8) {
           const bool all_masked = __all_sync(0xffffffffu, p.skip_thr > 0.f && mv <= -p.skip_thr);
