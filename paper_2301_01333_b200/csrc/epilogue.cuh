@@ -48,64 +48,71 @@ __device__ __forceinline__ int quantize_value(float t, float inv, int zp, int lo
   return min(max(r + zp, lo), hi);
 }
 
-// Store 16 consecutive outputs of one row (columns n0..n0+15) from 16 raw accumulator words.
-// `dst_row` points at column 0 of the row; n0 is a multiple of 16 and the row pitch keeps 16-byte
-// alignment of (dst_row + n0) for every supported dtype.
-__device__ __forceinline__ void epi_store16(const uint32_t* raw, void* dst_row, int n0, const Epilogue& e) {
-  // zero-point compensation of the integer accumulator (exact in s32)
+// Per-column constants of 16 consecutive output columns (bias, dequantisation scale, zero-point compensation).
+// Loading them is separated from using them so that a kernel can issue the loads before it waits for its
+// accumulators.
+struct EpiCols16 {
+  float b[16];
+  float dq[16];
   int c[16];
+};
+
+__device__ __forceinline__ void epi_load_cols16(EpiCols16& k, int n0, const Epilogue& e) {
   if (e.comp) {
     const int4* cp = reinterpret_cast<const int4*>(e.comp + n0);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int4 v = __ldg(cp + i);
-      c[4 * i] = v.x; c[4 * i + 1] = v.y; c[4 * i + 2] = v.z; c[4 * i + 3] = v.w;
+      k.c[4 * i] = v.x; k.c[4 * i + 1] = v.y; k.c[4 * i + 2] = v.z; k.c[4 * i + 3] = v.w;
     }
   } else {
 #pragma unroll
-    for (int i = 0; i < 16; ++i) c[i] = 0;
+    for (int i = 0; i < 16; ++i) k.c[i] = 0;
   }
-  if (e.acc_is_int && !e.has_dq) {   // raw s32 accumulators
-    int4* d = reinterpret_cast<int4*>(static_cast<int*>(dst_row) + n0);
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-      d[i] = make_int4(static_cast<int>(raw[4 * i]) - c[4 * i], static_cast<int>(raw[4 * i + 1]) - c[4 * i + 1],
-                       static_cast<int>(raw[4 * i + 2]) - c[4 * i + 2], static_cast<int>(raw[4 * i + 3]) - c[4 * i + 3]);
-    return;
-  }
-  // Fetch the 16 bias values with four vector loads up front: per-element loads behind per-element branches
-  // serialise into 16 dependent memory latencies.
-  float b[16];
   if (e.bias) {
     const float4* bp = reinterpret_cast<const float4*>(e.bias + n0);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const float4 v = __ldg(bp + i);
-      b[4 * i] = v.x; b[4 * i + 1] = v.y; b[4 * i + 2] = v.z; b[4 * i + 3] = v.w;
+      k.b[4 * i] = v.x; k.b[4 * i + 1] = v.y; k.b[4 * i + 2] = v.z; k.b[4 * i + 3] = v.w;
     }
   } else {
 #pragma unroll
-    for (int i = 0; i < 16; ++i) b[i] = 0.f;
+    for (int i = 0; i < 16; ++i) k.b[i] = 0.f;
   }
-  const bool has_bias = e.bias != nullptr, acc_int = e.acc_is_int != 0;
-  float dq[16];
   if (e.dqv) {
     const float4* dp = reinterpret_cast<const float4*>(e.dqv + n0);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const float4 v = __ldg(dp + i);
-      dq[4 * i] = v.x; dq[4 * i + 1] = v.y; dq[4 * i + 2] = v.z; dq[4 * i + 3] = v.w;
+      k.dq[4 * i] = v.x; k.dq[4 * i + 1] = v.y; k.dq[4 * i + 2] = v.z; k.dq[4 * i + 3] = v.w;
     }
   } else {
 #pragma unroll
-    for (int i = 0; i < 16; ++i) dq[i] = e.dq;
+    for (int i = 0; i < 16; ++i) k.dq[i] = e.dq;
   }
+}
+
+// Store 16 consecutive outputs of one row (columns n0..n0+15) from 16 raw accumulator words.
+// `dst_row` points at column 0 of the row; n0 is a multiple of 16 and the row pitch keeps 16-byte
+// alignment of (dst_row + n0) for every supported dtype.
+__device__ __forceinline__ void epi_store16_cols(const uint32_t* raw, void* dst_row, int n0, const Epilogue& e,
+                                                 const EpiCols16& k) {
+  if (e.acc_is_int && !e.has_dq) {   // raw s32 accumulators (zero-point compensation is exact in s32)
+    int4* d = reinterpret_cast<int4*>(static_cast<int*>(dst_row) + n0);
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      d[i] = make_int4(static_cast<int>(raw[4 * i]) - k.c[4 * i], static_cast<int>(raw[4 * i + 1]) - k.c[4 * i + 1],
+                       static_cast<int>(raw[4 * i + 2]) - k.c[4 * i + 2], static_cast<int>(raw[4 * i + 3]) - k.c[4 * i + 3]);
+    return;
+  }
+  const bool has_bias = e.bias != nullptr, acc_int = e.acc_is_int != 0;
   const int act = e.act;
   float t[16];
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
-    float x = acc_int ? __fmul_rn(__int2float_rn(static_cast<int>(raw[i]) - c[i]), dq[i]) : __uint_as_float(raw[i]);
-    x = has_bias ? __fadd_rn(x, b[i]) : x;      // separately rounded: exact on the integer path
+    float x = acc_int ? __fmul_rn(__int2float_rn(static_cast<int>(raw[i]) - k.c[i]), k.dq[i]) : __uint_as_float(raw[i]);
+    x = has_bias ? __fadd_rn(x, k.b[i]) : x;      // separately rounded: exact on the integer path
     t[i] = x;
   }
   if (act == ACT_RELU) {
@@ -142,6 +149,12 @@ __device__ __forceinline__ void epi_store16(const uint32_t* raw, void* dst_row, 
     }
     *reinterpret_cast<uint4*>(static_cast<uint8_t*>(dst_row) + n0) = make_uint4(w[0], w[1], w[2], w[3]);
   }
+}
+
+__device__ __forceinline__ void epi_store16(const uint32_t* raw, void* dst_row, int n0, const Epilogue& e) {
+  EpiCols16 k;
+  epi_load_cols16(k, n0, e);
+  epi_store16_cols(raw, dst_row, n0, e, k);
 }
 
 // Scalar store of one output (generic kernels).

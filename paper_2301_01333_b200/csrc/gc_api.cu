@@ -254,7 +254,7 @@ struct gc_compiled {
   std::string desc;
   // fused small-batch chain (one persistent kernel for all layers)
   bool chain_fused = false;
-  int chain_kind = 0, chain_grid = 0, chain_barriers = 0;
+  int chain_kind = 0, chain_grid = 0, chain_barriers = 0, chain_ks = 1;
   size_t chain_tmap_off = 0;                 // workspace offset of the tensor-map array
   uint32_t chain_w_smem = 0;
   int chain_a_stages = 0, chain_a_stage_bytes = 0, chain_a_rows = 0;
@@ -715,49 +715,66 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
     // Small-batch chains run as one persistent kernel when every layer fits one MMA row tile and all
     // weight slices of a CTA fit in shared memory next to the activation ring.
     bool ok = true;
-    int kind = -1, max_ctas = 0;
-    uint32_t w_smem = 0;
     c->chain_w_off.assign(c->layers.size(), 0);
+    int kind = -1, max_ctas = 0, max_nkb = 1, a_rows = 8;
     for (size_t l = 0; l < c->layers.size() && ok; ++l) {
       LayerPlan& L = c->layers[l];
       ok = L.M <= 128;
       const int lk = is_int8(L.a_dtype) ? 0 : (L.a_dtype == GC_BF16 ? 1 : 2);
       if (kind < 0) kind = lk;
       ok = ok && lk == kind;
+      a_rows = ((L.M + 7) / 8 * 8) > a_rows ? ((L.M + 7) / 8 * 8) : a_rows;
       if (L.use_tc) {
         const int ctas = (L.N + 31) / 32;
         max_ctas = ctas > max_ctas ? ctas : max_ctas;
-        c->chain_w_off[l] = w_smem;
-        w_smem += static_cast<uint32_t>(L.nkb) * 32 * 128;
+        max_nkb = L.nkb > max_nkb ? L.nkb : max_nkb;
       }
     }
-    // A-operand ring: round_up(M, 8) rows per stage, as many stages as fit (all k-blocks of the deepest
-    // layer if possible, so every layer fetches its whole A operand in one burst)
-    int a_rows = 8, max_nkb = 1;
-    for (auto& L : c->layers) {
-      a_rows = ((L.M + 7) / 8 * 8) > a_rows ? ((L.M + 7) / 8 * 8) : a_rows;
-      if (L.use_tc && L.nkb > max_nkb) max_nkb = L.nkb;
-    }
+    // The reduction axis is split over a cluster of ks CTAs (each multiplies its share of the k-blocks, the
+    // partial sums meet in distributed shared memory): worth it when the longest reduction has enough k-blocks.
+    // A-operand ring: round_up(M, 8) rows per stage and one stage per k-block a CTA handles in the deepest
+    // layer, so every layer fetches its whole A operand in one burst.
     const int a_stage_bytes = a_rows * 128;
-    int a_stages = max_nkb < 32 ? max_nkb : 32;
-    while (a_stages > 2 && mlp_chain_smem_bytes(w_smem, a_stages, a_stage_bytes) > static_cast<size_t>(prop.sharedMemPerBlockOptin))
-      --a_stages;
-    ok = ok && max_ctas > 0 && max_ctas <= c->num_sms && a_stages >= max_nkb &&
-         mlp_chain_smem_bytes(w_smem, a_stages, a_stage_bytes) <= static_cast<size_t>(prop.sharedMemPerBlockOptin);
+    int ks = max_nkb >= 8 ? 4 : (max_nkb >= 4 ? 2 : 1);
+    int a_stages = 0;
+    uint32_t w_smem = 0;
+    ok = ok && max_ctas > 0;
+    for (; ok; ks >>= 1) {
+      w_smem = 0;
+      for (size_t l = 0; l < c->layers.size(); ++l) {
+        const LayerPlan& L = c->layers[l];
+        c->chain_w_off[l] = w_smem;
+        if (L.use_tc) w_smem += static_cast<uint32_t>((L.nkb + ks - 1) / ks) * 32 * 128;
+      }
+      a_stages = (max_nkb + ks - 1) / ks;
+      const size_t smem = mlp_chain_smem_bytes(w_smem, a_stages, a_stage_bytes);
+      bool fits = a_stages <= 32 && max_ctas * ks <= c->num_sms && smem <= static_cast<size_t>(prop.sharedMemPerBlockOptin);
+      // all clusters must be resident together (the layers are separated by a grid-wide barrier)
+      if (fits && ks > 1 && cuda_device != GC_DEVICE_PLAN_ONLY) {
+        int cur = -1;
+        cudaGetDevice(&cur);
+        if (cur != cuda_device) cudaSetDevice(cuda_device);     // the occupancy query answers for the current device
+        fits = mlp_chain_max_clusters(kind, ks, smem) >= max_ctas;
+        if (cur >= 0 && cur != cuda_device) cudaSetDevice(cur);
+      }
+      if (fits) break;
+      if (ks == 1) ok = false;
+    }
     if (ok) {
       c->chain_a_stages = a_stages;
       c->chain_a_stage_bytes = a_stage_bytes;
       c->chain_a_rows = a_rows;
       c->chain_fused = true;
       c->chain_kind = kind;
-      c->chain_grid = max_ctas;
+      c->chain_grid = max_ctas * ks;
+      c->chain_ks = ks;
       c->chain_w_smem = w_smem;
       c->chain_barriers = (c->layers[0].need_pack ? 1 : 0) + static_cast<int>(c->layers.size()) - 1;
       c->chain_tmap_off = ws;
       ws = align_up(ws + 2 * CHAIN_MAX_LAYERS * sizeof(CUtensorMap), 1024);
       c->launches = 1;
-      snprintf(line, sizeof(line), "  fused chain: one persistent kernel, %d CTAs, %u KB of resident weight slices per CTA, %d grid barriers\n",
-               max_ctas, w_smem / 1024, c->chain_barriers);
+      snprintf(line, sizeof(line), "  fused chain: one persistent kernel, %d CTAs in clusters of %d (split reduction axis), %u KB of resident weight slices per CTA, %d grid barriers\n",
+               max_ctas * ks, ks, w_smem / 1024, c->chain_barriers);
       c->desc += line;
     }
   }
@@ -855,6 +872,7 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
     cp.barrier = reinterpret_cast<unsigned long long*>(ws + 64);
     cp.barrier_base = c.chain_arrivals;
     cp.early_weights = need ? 0 : 1;
+    cp.ks = c.chain_ks;
     const LayerPlan& L0 = c.layers[0];
     const void* a0 = in[L0.a_input];
     if (L0.need_pack) {

@@ -110,6 +110,7 @@ struct ChainParams {
   int64_t pack_src_pitch, pack_dst_pitch;   // bytes
   unsigned long long* barrier;              // grid-barrier counter (only grows)
   unsigned long long barrier_base;          // its value before this launch
+  int ks;                                   // CTAs per cluster = parts the reduction axis of every layer is split into
   int early_weights;                        // 1: the prepacked weights were written by an earlier call, so their loads
                                             // need not wait for the kernel that precedes this one on the stream
   uint32_t* status;
@@ -119,6 +120,8 @@ struct ChainParams {
 };
 size_t mlp_chain_smem_bytes(size_t w_smem_bytes, int a_stages, int a_stage_bytes);
 cudaError_t launch_mlp_chain(int kind, const ChainParams& p, int grid, cudaStream_t s);
+// clusters of `ks` CTAs of the chain kernel that can be resident together on the current device (0 on error)
+int mlp_chain_max_clusters(int kind, int ks, size_t smem);
 
 // ---- launchers (each enqueues exactly one kernel on the stream and returns cudaGetLastError) ----
 cudaError_t launch_pack_rows(const void* src, void* dst, int rows, int64_t src_pitch_bytes, int64_t dst_pitch_bytes,

@@ -12,11 +12,17 @@
 //     32 columns of the next activation.  A stage holds only round_up(M, 8) rows; the MMA still reads 128
 //     rows, the surplus rows come from whatever follows in shared memory and only feed accumulator rows
 //     that are never stored (rows of a matmul are independent);
+//   * the reduction axis of every layer is split over the KS CTAs of a thread-block cluster (KS = 1, 2 or 4): each
+//     CTA loads, holds and multiplies only its share of the k-blocks, which divides the serial chain of MMAs
+//     (about 120 clocks each however narrow the tile) and the A-operand traffic per CTA by KS.  The partial
+//     accumulators meet in distributed shared memory: every CTA of the cluster finishes 128 / KS rows, so warp q
+//     sends its 32 rows to the CTA that owns them and signals that CTA's mbarrier; the owner adds the KS partials
+//     in a fixed order (exact for s32, deterministic for fp32), applies the post-ops and stores;
 //   * a grid-wide barrier (epoch-counted atomic in global memory, bounded spin) separates the layers;
 //   * layers the tensor-core path does not take (N not a multiple of 16, e.g. the 256 -> 1 tail) run on
 //     CUDA cores inside the same kernel, one warp per output;
 //   * an input whose row pitch TMA cannot address is first copied to a padded buffer by all threads.
-// At most one CTA per SM (<= 148 CTAs of 192 threads), so all CTAs of the grid are resident together.
+// At most one CTA per SM, and the host checks that all clusters of the grid can be resident together.
 #include <cuda_bf16.h>
 
 #include "epilogue.cuh"
@@ -32,6 +38,7 @@ constexpr int CH_BLOCK_N = 32;
 // narrow the tile is, so the four 32-byte k-steps of a k-block go to four independent 32-column accumulators
 // that the epilogue adds up (exact for s32; a fixed summation order for fp32).
 constexpr int CH_NACC = 4;
+constexpr int CH_RED_BYTES = 128 * 32 * 4;   // partial-sum exchange buffer: 128 rows x 32 columns x 4 bytes
 
 __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
   unsigned long long v;
@@ -45,9 +52,10 @@ __device__ __forceinline__ bool grid_barrier(unsigned long long* ctr, unsigned l
   __syncthreads();
   int ok = 1;
   if (threadIdx.x == 0) {
-    asm volatile("fence.proxy.async;" ::: "memory");   // async-proxy (TMA) accesses vs. generic stores
-    __threadfence();
-    atomicAdd(ctr, 1ULL);
+    // generic-proxy stores of this CTA (made CTA-visible by the barrier above) must be visible to the other CTAs'
+    // TMA loads: proxy fence on the global space, then a releasing reduction (no return value to wait for)
+    asm volatile("fence.proxy.async.global;" ::: "memory");
+    asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(ctr), "l"(1ULL) : "memory");
     const uint64_t t0 = globaltimer_ns();
     uint32_t i = 0;
     while (ld_acquire_u64(ctr) < target) {
@@ -56,7 +64,7 @@ __device__ __forceinline__ bool grid_barrier(unsigned long long* ctr, unsigned l
         break;
       }
     }
-    asm volatile("fence.proxy.async;" ::: "memory");
+    asm volatile("fence.proxy.async.global;" ::: "memory");
   }
   return __syncthreads_and(ok) != 0;
 }
@@ -70,6 +78,34 @@ __device__ __forceinline__ int ch_load_i(const void* p, int64_t i, int dtype) {
   return static_cast<const int8_t*>(p)[i];
 }
 
+// 16 bytes into the shared memory of a CTA of the cluster; the store itself reports its bytes to that CTA's
+// mbarrier (complete_tx), so the sender neither waits for the store nor issues a separate releasing arrive
+__device__ __forceinline__ void st_async_cluster_v4(uint32_t cluster_addr, uint32_t cluster_bar, uint32_t x, uint32_t y,
+                                                    uint32_t z, uint32_t w) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(
+                   cluster_addr),
+               "r"(x), "r"(y), "r"(z), "r"(w), "r"(cluster_bar)
+               : "memory");
+}
+// Bounded wait on an mbarrier of this CTA that CTAs of the cluster arrive on: acquire at cluster scope, so the
+// remote shared-memory stores made before those arrivals are visible afterwards.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity) {
+  const uint64_t t0 = globaltimer_ns();
+  for (uint32_t i = 0; i < (1u << 22); ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred P;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 P, [%1], %2, %3;\n\t"
+        "selp.b32 %0, 1, 0, P;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(20000u)
+        : "memory");
+    if (ok) return true;
+    if ((i & 15u) == 15u && globaltimer_ns() - t0 > 2000000000ull) break;
+  }
+  return false;
+}
+
 template <int KIND>
 __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_constant__ ChainParams p) {
   constexpr int K_ELEMS = KIND == KIND_I8 ? 128 : (KIND == KIND_BF16 ? 64 : 32);
@@ -78,17 +114,22 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int CH_STAGES = p.a_stages;
   const int CH_A_STAGE_BYTES = p.a_stage_bytes;
+  const int KS = p.ks;                                            // CTAs per cluster = parts of the reduction axis
   uint8_t* sA = smem;                                             // a_stages x a_stage_bytes
   // the weight slices (padded to at least 16 KB) follow the ring, so the 128-row MMA reads of the last stages
   // stay inside this CTA's shared memory
   uint8_t* sW = sA + ((CH_STAGES * CH_A_STAGE_BYTES + 1023) & ~1023);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sW + (p.w_smem_bytes < 16384u ? 16384u : p.w_smem_bytes));
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * CH_MAX_STAGES + 1 + CHAIN_MAX_LAYERS);
+  // partial sums from the cluster: [KS sources][128 / KS rows][32 columns] s32 / fp32, 16-byte chunks XOR-swizzled
+  uint8_t* sRed = sW + (p.w_smem_bytes < 16384u ? 16384u : p.w_smem_bytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sRed + CH_RED_BYTES);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * CH_MAX_STAGES + 2 + CHAIN_MAX_LAYERS);
   const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * CH_MAX_STAGES;
   const uint32_t bar_tfull = bar_empty + 8 * CH_MAX_STAGES;       // [1]
-  const uint32_t bar_wfull = bar_tfull + 8;                       // [CHAIN_MAX_LAYERS]
+  const uint32_t bar_red = bar_tfull + 8;                         // [1] partials of the cluster have arrived
+  const uint32_t bar_wfull = bar_red + 8;                         // [CHAIN_MAX_LAYERS]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int cta = blockIdx.x;
+  const int ksr = KS > 1 ? static_cast<int>(cluster_ctarank()) : 0;   // my part of the reduction axis
+  const int cta = blockIdx.x / KS;                                // my 32-column slice
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < CH_STAGES; ++s) {
@@ -96,6 +137,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
       mbar_init(bar_empty + 8 * s, 1);
     }
     mbar_init(bar_tfull, 1);
+    mbar_init(bar_red, 1);                                        // armed per layer with the bytes the cluster will send
     for (int l = 0; l < CHAIN_MAX_LAYERS; ++l) mbar_init(bar_wfull + 8 * l, 1);
     fence_mbar_init();
   }
@@ -107,6 +149,8 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // nobody may signal a barrier of another CTA before that CTA has initialised it
+  if (KS > 1) cluster_sync_all();
 
   // Programmatic dependent launch: everything above may overlap the tail of the preceding kernel on the stream.
   // The prepacked weights are constants; unless this very call has just enqueued their prepack, their loads may
@@ -114,14 +158,20 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (!p.early_weights) asm volatile("griddepcontrol.wait;" ::: "memory");
 
+  // my k-blocks of layer L: [kb_lo, kb_hi)
+  auto kb_lo = [&](const ChainLayer& L) { return ksr * L.nkb / KS; };
+  auto kb_hi = [&](const ChainLayer& L) { return (ksr + 1) * L.nkb / KS; };
+
   // every layer's weight slice starts moving now (constants: they do not depend on earlier layers)
   if (warp == 0 && lane == 0) {
     for (int l = 0; l < p.n_layers; ++l) {
       const ChainLayer& L = p.L[l];
       if (L.active_ctas == 0 || cta >= L.active_ctas) continue;
-      mbar_arrive_expect_tx(bar_wfull + 8 * l, static_cast<uint32_t>(L.nkb) * (CH_BLOCK_N * 128));
-      for (int kb = 0; kb < L.nkb; ++kb)
-        tma_load_2d(smem_u32(sW) + L.w_smem_off + kb * (CH_BLOCK_N * 128), p.tmaps + L.b_tm, kb * K_ELEMS,
+      const int lo = kb_lo(L), hi = kb_hi(L);
+      if (hi == lo) continue;
+      mbar_arrive_expect_tx(bar_wfull + 8 * l, static_cast<uint32_t>(hi - lo) * (CH_BLOCK_N * 128));
+      for (int kb = lo; kb < hi; ++kb)
+        tma_load_2d(smem_u32(sW) + L.w_smem_off + (kb - lo) * (CH_BLOCK_N * 128), p.tmaps + L.b_tm, kb * K_ELEMS,
                     cta * CH_BLOCK_N, bar_wfull + 8 * l);
     }
   }
@@ -144,7 +194,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
     const int64_t total = static_cast<int64_t>(p.pack_rows) * words_per_row;
     const uint8_t* src = static_cast<const uint8_t*>(p.pack_src);
     uint8_t* dst = static_cast<uint8_t*>(p.pack_dst);
-    for (int64_t i = static_cast<int64_t>(cta) * CH_THREADS + threadIdx.x; i < total;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * CH_THREADS + threadIdx.x; i < total;
          i += static_cast<int64_t>(gridDim.x) * CH_THREADS) {
       const int64_t r = i / words_per_row, c = (i % words_per_row) * 4;
       uint32_t w = 0;
@@ -159,18 +209,21 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
   int stage = 0;                 // ring position, shared by construction between producer and MMA thread
   uint32_t phase = 0;
   uint32_t tphase = 0;           // parity of the accumulator-ready barrier (one completion per active layer)
+  const int rows_per = 128 / KS; // rows of the tile this CTA finishes
   for (int l = 0; l < p.n_layers && !failed; ++l) {
     // A by-value copy: fields read through a reference into the parameter space are re-fetched around every
     // store (possible aliasing) at a few hundred clocks each, which made a 16-element epilogue cost thousands.
     const ChainLayer L = p.L[l];
     if (L.active_ctas > 0) {
       if (cta < L.active_ctas) {
+        const int lo = kb_lo(L), my_nkb = kb_hi(L) - lo;
         if (warp == 0) {
           if (lane == 0) {
-            asm volatile("fence.proxy.async;" ::: "memory");     // activations were written with generic stores
-            // a_stages >= nkb (planner): a stage is never reused within a layer, and between layers the
+            // (this thread is the one that ran the grid barrier: its proxy fence after the acquire already ordered
+            // the other CTAs' generic stores before the TMA loads below)
+            // a_stages >= my_nkb (planner): a stage is never reused within a layer, and between layers the
             // accumulator-ready commit plus the grid barrier guarantee that every MMA has read its stage
-            for (int kb = 0; kb < L.nkb; ++kb) {
+            for (int kb = lo; kb < lo + my_nkb; ++kb) {
               mbar_arrive_expect_tx(bar_full + 8 * stage, CH_A_STAGE_BYTES);
               tma_load_2d(smem_u32(sA) + stage * CH_A_STAGE_BYTES, p.tmaps + L.a_tm, kb * K_ELEMS, 0, bar_full + 8 * stage);
               if (++stage == CH_STAGES) {
@@ -181,34 +234,47 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
           }
         } else if (warp == 1) {
           if (lane == 0) {
-            bool ok = mbar_wait(bar_wfull + 8 * l, 0);
-            const uint32_t idesc = L.idesc;
-            const int nkb = L.nkb;
-            const uint64_t a_desc0 = make_smem_desc(smem_u32(sA), 16, 1024, SWZ_128B);
-            uint64_t b_desc = make_smem_desc(smem_u32(sW) + L.w_smem_off, 16, 1024, SWZ_128B);
-            const uint32_t a_step = static_cast<uint32_t>(CH_A_STAGE_BYTES) >> 4;   // descriptor address units of 16 bytes
-            for (int kb = 0; kb < nkb && ok; ++kb, b_desc += (CH_BLOCK_N * 128) >> 4) {
-              ok = mbar_wait(bar_full + 8 * stage, phase);
-              if (!ok) break;
-              tc_fence_after();
-              const uint64_t a_desc = a_desc0 + static_cast<uint64_t>(stage) * a_step;
+            if (my_nkb == 0) {
+              mbar_arrive(bar_tfull);                             // nothing to multiply: my partial sums are zero
+            } else {
+              bool ok = mbar_wait(bar_wfull + 8 * l, 0);
+              const uint32_t idesc = L.idesc;
+              const uint64_t a_desc0 = make_smem_desc(smem_u32(sA), 16, 1024, SWZ_128B);
+              uint64_t b_desc = make_smem_desc(smem_u32(sW) + L.w_smem_off, 16, 1024, SWZ_128B);
+              const uint32_t a_step = static_cast<uint32_t>(CH_A_STAGE_BYTES) >> 4;   // descriptor address units of 16 bytes
+              for (int i = 0; i < my_nkb && ok; ++i, b_desc += (CH_BLOCK_N * 128) >> 4) {
+                ok = mbar_wait(bar_full + 8 * stage, phase);
+                if (!ok) break;
+                tc_fence_after();
+                const uint64_t a_desc = a_desc0 + static_cast<uint64_t>(stage) * a_step;
 #pragma unroll
-              for (int k = 0; k < 4; ++k)
-                umma_ss<KIND>(tmem_base + k * CH_BLOCK_N, a_desc + 2 * k, b_desc + 2 * k, idesc, kb != 0);
-              if (++stage == CH_STAGES) {
-                stage = 0;
-                phase ^= 1;
+                for (int k = 0; k < 4; ++k)
+                  umma_ss<KIND>(tmem_base + k * CH_BLOCK_N, a_desc + 2 * k, b_desc + 2 * k, idesc, i != 0);
+                if (++stage == CH_STAGES) {
+                  stage = 0;
+                  phase ^= 1;
+                }
               }
+              if (ok) umma_commit(bar_tfull);
+              else report(p.status, DEV_TIMEOUT_MMA);
             }
-            if (ok) umma_commit(bar_tfull);
-            else report(p.status, DEV_TIMEOUT_MMA);
           }
         } else {
           const int q = warp & 3;
+          // expect the partial sums of the whole cluster for my rows of the tile (senders may be ahead of this)
+          if (KS > 1 && threadIdx.x == 64) mbar_arrive_expect_tx(bar_red, CH_RED_BYTES);
+          // the per-column constants of the outputs this thread will finish: fetched now, used after the waits
+          const int ft = threadIdx.x - 64;
+          const int fcol = cta * CH_BLOCK_N + 16 * (ft & 1);
+          const bool finisher = KS > 1 && ft < 2 * rows_per && fcol < L.N;
+          EpiCols16 fk;
+          if (finisher) epi_load_cols16(fk, fcol, L.epi);
+          if (KS == 1 && L.epi.bias && lane < 2 && cta * CH_BLOCK_N + 16 * lane < L.N)
+            asm volatile("prefetch.global.L1 [%0];" ::"l"(L.epi.bias + cta * CH_BLOCK_N + 16 * lane));
           if (mbar_wait(bar_tfull, tphase)) {
             tc_fence_after();
             uint32_t r[32];
-            {
+            if (my_nkb > 0) {
               uint32_t r1[32], r2[32], r3[32];
               const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
               tmem_ld32(t_row, r);
@@ -224,14 +290,59 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
                   r[i] = __float_as_uint((__uint_as_float(r[i]) + __uint_as_float(r1[i])) +
                                          (__uint_as_float(r2[i]) + __uint_as_float(r3[i])));
               }
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) r[i] = 0u;
             }
             tc_fence_before();
-            const int row = q * 32 + lane;
             const int n0 = cta * CH_BLOCK_N;
-            if (row < L.M) {
-              char* dst_row = static_cast<char*>(L.out) + static_cast<int64_t>(row) * L.out_pitch * L.out_elem;
-              if (n0 < L.N) epi_store16(r, dst_row, n0, L.epi);
-              if (n0 + 16 < L.N) epi_store16(r + 16, dst_row, n0 + 16, L.epi);
+            if (KS == 1) {
+              const int row = q * 32 + lane;
+              if (row < L.M) {
+                char* dst_row = static_cast<char*>(L.out) + static_cast<int64_t>(row) * L.out_pitch * L.out_elem;
+                if (n0 < L.N) epi_store16(r, dst_row, n0, L.epi);
+                if (n0 + 16 < L.N) epi_store16(r + 16, dst_row, n0 + 16, L.epi);
+              }
+            } else {
+              // my warp's 32 rows belong to CTA `dest` of the cluster: 128 bytes per row into its buffer
+              const int row = q * 32 + lane;
+              const int dest = row / rows_per, lrow = row % rows_per;
+              const uint32_t base = mapa_shared(smem_u32(sRed) + static_cast<uint32_t>((ksr * rows_per + lrow) * 128), dest);
+              const uint32_t rbar = mapa_shared(bar_red, dest);
+#pragma unroll
+              for (int c = 0; c < 8; ++c)
+                st_async_cluster_v4(base + ((c ^ (lrow & 7)) << 4), rbar, r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);
+              // finish my rows of the tile: thread t handles row t / 2, columns 16 (t % 2) .. + 16
+              if (mbar_wait_cluster(bar_red, tphase)) {
+                if (finisher) {
+                  const int frow = ft >> 1, half = ft & 1;
+                  uint32_t a[16];
+#pragma unroll
+                  for (int i = 0; i < 16; ++i) a[i] = 0u;
+                  for (int s = 0; s < KS; ++s) {
+                    const uint8_t* src = sRed + (s * rows_per + frow) * 128;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                      const uint4 v = *reinterpret_cast<const uint4*>(src + (((half * 4 + c) ^ (frow & 7)) << 4));
+                      if constexpr (KIND == KIND_I8) {
+                        a[4 * c] += v.x; a[4 * c + 1] += v.y; a[4 * c + 2] += v.z; a[4 * c + 3] += v.w;
+                      } else {
+                        a[4 * c] = __float_as_uint(__uint_as_float(a[4 * c]) + __uint_as_float(v.x));
+                        a[4 * c + 1] = __float_as_uint(__uint_as_float(a[4 * c + 1]) + __uint_as_float(v.y));
+                        a[4 * c + 2] = __float_as_uint(__uint_as_float(a[4 * c + 2]) + __uint_as_float(v.z));
+                        a[4 * c + 3] = __float_as_uint(__uint_as_float(a[4 * c + 3]) + __uint_as_float(v.w));
+                      }
+                    }
+                  }
+                  const int grow = ksr * rows_per + frow;
+                  if (grow < L.M) {
+                    char* dst_row = static_cast<char*>(L.out) + static_cast<int64_t>(grow) * L.out_pitch * L.out_elem;
+                    epi_store16_cols(a, dst_row, fcol, L.epi, fk);
+                  }
+                }
+              } else {
+                report(p.status, DEV_TIMEOUT_EPILOGUE);
+              }
             }
           } else {
             report(p.status, DEV_TIMEOUT_EPILOGUE);
@@ -239,8 +350,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
         }
         // the ring position advances identically in the threads that did not walk it
         if (!(warp <= 1 && lane == 0)) {
-          const int adv = L.nkb;
-          const int pos = stage + adv;
+          const int pos = stage + my_nkb;
           phase ^= (pos / CH_STAGES) & 1;
           stage = pos % CH_STAGES;
         }
@@ -249,7 +359,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
     } else {
       // CUDA-core layer: one warp per output element, lanes stride the reduction axis
       const int64_t outputs = static_cast<int64_t>(L.M) * L.N;
-      for (int64_t o = static_cast<int64_t>(cta) * (CH_THREADS / 32) + warp; o < outputs;
+      for (int64_t o = static_cast<int64_t>(blockIdx.x) * (CH_THREADS / 32) + warp; o < outputs;
            o += static_cast<int64_t>(gridDim.x) * (CH_THREADS / 32)) {
         const int m = static_cast<int>(o / L.N), n = static_cast<int>(o % L.N);
         const char* A = static_cast<const char*>(L.a_ptr) + static_cast<int64_t>(m) * L.a_pitch * ESZ;
@@ -283,11 +393,13 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
     tc_fence_after();
     tmem_dealloc(tmem_base, CH_NACC * CH_BLOCK_N);
   }
+  // no CTA leaves while another one of its cluster may still write into its shared memory
+  if (KS > 1) cluster_sync_all();
 }
 
 size_t mlp_chain_smem_bytes(size_t w_smem_bytes, int a_stages, int a_stage_bytes) {
   return ((static_cast<size_t>(a_stages) * a_stage_bytes + 1023) & ~size_t(1023)) +
-         (w_smem_bytes < 16384 ? size_t(16384) : w_smem_bytes) + 1024 + 1024;
+         (w_smem_bytes < 16384 ? size_t(16384) : w_smem_bytes) + CH_RED_BYTES + 1024 + 1024;
 }
 
 cudaError_t launch_mlp_chain(int kind, const ChainParams& p, int grid, cudaStream_t s) {
@@ -307,13 +419,38 @@ cudaError_t launch_mlp_chain(int kind, const ChainParams& p, int grid, cudaStrea
   // they are not, the waiting CTAs only wait for unrelated work to finish, and every spin is bounded anyway.
   // Programmatic dependent launch: the set-up may overlap the tail of whatever precedes on the stream; the
   // kernel waits for that work to complete before its first global access.
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = static_cast<unsigned>(p.ks);
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = p.ks > 1 ? 2 : 1;
   void* args[] = {const_cast<ChainParams*>(&p)};
   return cudaLaunchKernelExC(&cfg, kern, args);
+}
+
+int mlp_chain_max_clusters(int kind, int ks, size_t smem) {
+  void* kern = kind == KIND_I8 ? reinterpret_cast<void*>(mlp_chain_kernel<KIND_I8>)
+               : kind == KIND_BF16 ? reinterpret_cast<void*>(mlp_chain_kernel<KIND_BF16>)
+                                   : reinterpret_cast<void*>(mlp_chain_kernel<KIND_TF32>);
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) return 0;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(ks));
+  cfg.blockDim = dim3(CH_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = static_cast<unsigned>(ks);
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) return 0;
+  return n;
 }
 
 }  // namespace gc
