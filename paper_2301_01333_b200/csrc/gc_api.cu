@@ -769,7 +769,7 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
       c->chain_grid = max_ctas * ks;
       c->chain_ks = ks;
       c->chain_w_smem = w_smem;
-      c->chain_barriers = (c->layers[0].need_pack ? 1 : 0) + static_cast<int>(c->layers.size()) - 1;
+      c->chain_barriers = static_cast<int>(c->layers.size()) - 1;   // one grid barrier between consecutive layers
       c->chain_tmap_off = ws;
       ws = align_up(ws + 2 * CHAIN_MAX_LAYERS * sizeof(CUtensorMap), 1024);
       c->launches = 1;
@@ -878,10 +878,8 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
     if (L0.need_pack) {
       const int esz0 = dtype_bytes(L0.a_dtype);
       cp.pack_src = a0;
-      cp.pack_dst = ws + L0.pack_off;
       cp.pack_rows = L0.M;
       cp.pack_src_pitch = L0.a_pitch * esz0;
-      cp.pack_dst_pitch = L0.pack_pitch * esz0;
     }
     const bool rebuild = !c.chain_tmaps_valid || (!L0.need_pack && c.chain_a0_ptr != a0);
     if (rebuild) c.chain_tmaps.assign(2 * CHAIN_MAX_LAYERS, CUtensorMap());

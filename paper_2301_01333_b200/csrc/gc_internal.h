@@ -104,10 +104,9 @@ struct ChainParams {
   uint32_t w_smem_bytes;   // shared memory taken by the resident weight slices
   int a_stages;            // A-operand ring: stages and bytes per stage (round_up(M, 8) rows of 128 bytes)
   int a_stage_bytes;
-  const void* pack_src;    // graph-entry reorder (pack_rows == 0: none)
-  void* pack_dst;
-  int pack_rows;
-  int64_t pack_src_pitch, pack_dst_pitch;   // bytes
+  const void* pack_src;    // graph-entry reorder: the first layer's input when TMA cannot address its row pitch
+  int pack_rows;           // its rows (0: the first layer is fed by TMA like the others)
+  int64_t pack_src_pitch;  // bytes
   unsigned long long* barrier;              // grid-barrier counter (only grows)
   unsigned long long barrier_base;          // its value before this launch
   int ks;                                   // CTAs per cluster = parts the reduction axis of every layer is split into

@@ -21,7 +21,9 @@
 //   * a grid-wide barrier (epoch-counted atomic in global memory, bounded spin) separates the layers;
 //   * layers the tensor-core path does not take (N not a multiple of 16, e.g. the 256 -> 1 tail) run on
 //     CUDA cores inside the same kernel, one warp per output;
-//   * an input whose row pitch TMA cannot address is first copied to a padded buffer by all threads.
+//   * an input whose row pitch TMA cannot address (the graph-entry reorder, Section V: pre-op fusion "only at the
+//     entry point of the graph") is read with plain loads by the four epilogue warps, which are idle at that point,
+//     realigned in registers and written straight into the swizzled A-operand stages of the first layer.
 // At most one CTA per SM, and the host checks that all clusters of the grid can be resident together.
 #include <cuda_bf16.h>
 
@@ -78,13 +80,13 @@ __device__ __forceinline__ int ch_load_i(const void* p, int64_t i, int dtype) {
   return static_cast<const int8_t*>(p)[i];
 }
 
-// 16 bytes into the shared memory of a CTA of the cluster; the store itself reports its bytes to that CTA's
-// mbarrier (complete_tx), so the sender neither waits for the store nor issues a separate releasing arrive
-__device__ __forceinline__ void st_async_cluster_v4(uint32_t cluster_addr, uint32_t cluster_bar, uint32_t x, uint32_t y,
-                                                    uint32_t z, uint32_t w) {
-  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(
-                   cluster_addr),
-               "r"(x), "r"(y), "r"(z), "r"(w), "r"(cluster_bar)
+// Bulk copy from this CTA's shared memory into the shared memory of a CTA of the cluster; the copy reports its
+// bytes to that CTA's mbarrier (complete_tx).  Addresses and size are multiples of 16 bytes.
+__device__ __forceinline__ void bulk_copy_to_cluster(uint32_t dst_cluster_addr, uint32_t src_cta_addr, uint32_t bytes,
+                                                     uint32_t cluster_bar) {
+  asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   dst_cluster_addr),
+               "r"(src_cta_addr), "r"(bytes), "r"(cluster_bar)
                : "memory");
 }
 // Bounded wait on an mbarrier of this CTA that CTAs of the cluster arrive on: acquire at cluster scope, so the
@@ -121,12 +123,14 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
   uint8_t* sW = sA + ((CH_STAGES * CH_A_STAGE_BYTES + 1023) & ~1023);
   // partial sums from the cluster: [KS sources][128 / KS rows][32 columns] s32 / fp32, 16-byte chunks XOR-swizzled
   uint8_t* sRed = sW + (p.w_smem_bytes < 16384u ? 16384u : p.w_smem_bytes);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sRed + CH_RED_BYTES);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * CH_MAX_STAGES + 2 + CHAIN_MAX_LAYERS);
+  uint8_t* sSend = sRed + CH_RED_BYTES;                           // my own partial sums, staged for the bulk copies
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sSend + CH_RED_BYTES);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * CH_MAX_STAGES + 3 + CHAIN_MAX_LAYERS);
   const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * CH_MAX_STAGES;
   const uint32_t bar_tfull = bar_empty + 8 * CH_MAX_STAGES;       // [1]
   const uint32_t bar_red = bar_tfull + 8;                         // [1] partials of the cluster have arrived
-  const uint32_t bar_wfull = bar_red + 8;                         // [CHAIN_MAX_LAYERS]
+  const uint32_t bar_a0 = bar_red + 8;                            // [1] first layer's A operand written by the epilogue warps
+  const uint32_t bar_wfull = bar_a0 + 8;                          // [CHAIN_MAX_LAYERS]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int ksr = KS > 1 ? static_cast<int>(cluster_ctarank()) : 0;   // my part of the reduction axis
   const int cta = blockIdx.x / KS;                                // my 32-column slice
@@ -137,6 +141,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
       mbar_init(bar_empty + 8 * s, 1);
     }
     mbar_init(bar_tfull, 1);
+    mbar_init(bar_a0, 4);                                         // one arrival per epilogue warp
     mbar_init(bar_red, 1);                                        // armed per layer with the bytes the cluster will send
     for (int l = 0; l < CHAIN_MAX_LAYERS; ++l) mbar_init(bar_wfull + 8 * l, 1);
     fence_mbar_init();
@@ -178,6 +183,17 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
 
   if (p.early_weights) asm volatile("griddepcontrol.wait;" ::: "memory");
 
+  // the per-column constants this CTA's epilogues will need: start them on their way from DRAM now
+  if (warp >= 2 && threadIdx.x - 64 < p.n_layers) {
+    const ChainLayer& L = p.L[threadIdx.x - 64];
+    const int col = cta * CH_BLOCK_N;
+    if (L.active_ctas > 0 && cta < L.active_ctas) {
+      if (L.epi.bias) asm volatile("prefetch.global.L2 [%0];" ::"l"(L.epi.bias + col));
+      if (L.epi.dqv) asm volatile("prefetch.global.L2 [%0];" ::"l"(L.epi.dqv + col));
+      if (L.epi.comp) asm volatile("prefetch.global.L2 [%0];" ::"l"(L.epi.comp + col));
+    }
+  }
+
   bool failed = false;
   unsigned long long bar_count = p.barrier_base;                  // counter value before this launch
   auto next_barrier = [&]() {
@@ -187,24 +203,6 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
       report(p.status, DEV_TIMEOUT_OTHER);
     }
   };
-
-  // graph-entry reorder: copy the input into a buffer whose row pitch TMA can address
-  if (p.pack_rows > 0) {
-    const int64_t words_per_row = p.pack_dst_pitch / 4;
-    const int64_t total = static_cast<int64_t>(p.pack_rows) * words_per_row;
-    const uint8_t* src = static_cast<const uint8_t*>(p.pack_src);
-    uint8_t* dst = static_cast<uint8_t*>(p.pack_dst);
-    for (int64_t i = static_cast<int64_t>(blockIdx.x) * CH_THREADS + threadIdx.x; i < total;
-         i += static_cast<int64_t>(gridDim.x) * CH_THREADS) {
-      const int64_t r = i / words_per_row, c = (i % words_per_row) * 4;
-      uint32_t w = 0;
-#pragma unroll
-      for (int b = 0; b < 4; ++b)
-        if (c + b < p.pack_src_pitch) w |= static_cast<uint32_t>(src[r * p.pack_src_pitch + c + b]) << (8 * b);
-      *reinterpret_cast<uint32_t*>(dst + r * p.pack_dst_pitch + c) = w;
-    }
-    next_barrier();
-  }
 
   int stage = 0;                 // ring position, shared by construction between producer and MMA thread
   uint32_t phase = 0;
@@ -217,8 +215,10 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
     if (L.active_ctas > 0) {
       if (cta < L.active_ctas) {
         const int lo = kb_lo(L), my_nkb = kb_hi(L) - lo;
+        // first layer fed by plain loads (graph-entry reorder): its blocks use stages 0 .. my_nkb-1 outside the ring
+        const bool manual_a = l == 0 && p.pack_rows > 0;
         if (warp == 0) {
-          if (lane == 0) {
+          if (lane == 0 && !manual_a) {
             // (this thread is the one that ran the grid barrier: its proxy fence after the acquire already ordered
             // the other CTAs' generic stores before the TMA loads below)
             // a_stages >= my_nkb (planner): a stage is never reused within a layer, and between layers the
@@ -238,19 +238,20 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
               mbar_arrive(bar_tfull);                             // nothing to multiply: my partial sums are zero
             } else {
               bool ok = mbar_wait(bar_wfull + 8 * l, 0);
+              if (manual_a) ok = ok && mbar_wait(bar_a0, 0);
               const uint32_t idesc = L.idesc;
               const uint64_t a_desc0 = make_smem_desc(smem_u32(sA), 16, 1024, SWZ_128B);
               uint64_t b_desc = make_smem_desc(smem_u32(sW) + L.w_smem_off, 16, 1024, SWZ_128B);
               const uint32_t a_step = static_cast<uint32_t>(CH_A_STAGE_BYTES) >> 4;   // descriptor address units of 16 bytes
               for (int i = 0; i < my_nkb && ok; ++i, b_desc += (CH_BLOCK_N * 128) >> 4) {
-                ok = mbar_wait(bar_full + 8 * stage, phase);
+                if (!manual_a) ok = mbar_wait(bar_full + 8 * stage, phase);
                 if (!ok) break;
                 tc_fence_after();
-                const uint64_t a_desc = a_desc0 + static_cast<uint64_t>(stage) * a_step;
+                const uint64_t a_desc = a_desc0 + static_cast<uint64_t>(manual_a ? i : stage) * a_step;
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
                   umma_ss<KIND>(tmem_base + k * CH_BLOCK_N, a_desc + 2 * k, b_desc + 2 * k, idesc, i != 0);
-                if (++stage == CH_STAGES) {
+                if (!manual_a && ++stage == CH_STAGES) {
                   stage = 0;
                   phase ^= 1;
                 }
@@ -261,6 +262,47 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
           }
         } else {
           const int q = warp & 3;
+          if (manual_a) {
+            // Row r of my k-blocks (thread per row): 16-byte chunks assembled from aligned 32-bit words of the
+            // (arbitrarily aligned) source row with funnel shifts, zero beyond the row's K bytes and beyond row M,
+            // stored where TMA would have put them (128-byte rows, 8-row groups of 1024 bytes, 16-byte chunk index
+            // XOR row mod 8).  All loads of a thread are independent, so one memory round trip covers them.
+            const int r = q * 32 + lane;
+            const int a_rows = CH_A_STAGE_BYTES / 128;
+            const int64_t kbytes = static_cast<int64_t>(L.K) * ESZ;
+            const uint8_t* src_row = static_cast<const uint8_t*>(p.pack_src) + static_cast<int64_t>(r) * p.pack_src_pitch;
+            if (r < a_rows) {
+              for (int i = 0; i < my_nkb; ++i) {
+                uint8_t* dst = sA + i * CH_A_STAGE_BYTES + (r >> 3) * 1024 + (r & 7) * 128;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                  const int64_t off = static_cast<int64_t>(lo + i) * 128 + c * 16;     // byte offset inside the row
+                  int64_t nv = kbytes - off;                                             // valid bytes of this chunk
+                  nv = r < L.M ? (nv > 16 ? 16 : nv) : 0;
+                  uint32_t o[4] = {0u, 0u, 0u, 0u};
+                  if (nv > 0) {
+                    const uintptr_t a = reinterpret_cast<uintptr_t>(src_row + off);
+                    const uint32_t sh = static_cast<uint32_t>(a & 3);
+                    const uint32_t* aw = reinterpret_cast<const uint32_t*>(a - sh);
+                    uint32_t w[5];
+#pragma unroll
+                    for (int j = 0; j < 5; ++j)   // word j holds chunk bytes [4j - sh, 4j - sh + 4): load it only if one is valid
+                      w[j] = (4 * j - static_cast<int>(sh) < nv) ? __ldg(aw + j) : 0u;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                      const uint32_t v = __funnelshift_r(w[j], w[j + 1], sh * 8);
+                      const int64_t left = nv - 4 * j;
+                      o[j] = left >= 4 ? v : (left <= 0 ? 0u : (v & ((1u << (8 * static_cast<int>(left))) - 1u)));
+                    }
+                  }
+                  *reinterpret_cast<uint4*>(dst + ((c ^ (r & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                }
+              }
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_a0);
+          }
           // expect the partial sums of the whole cluster for my rows of the tile (senders may be ahead of this)
           if (KS > 1 && threadIdx.x == 64) mbar_arrive_expect_tx(bar_red, CH_RED_BYTES);
           // the per-column constants of the outputs this thread will finish: fetched now, used after the waits
@@ -307,11 +349,17 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
               // my warp's 32 rows belong to CTA `dest` of the cluster: 128 bytes per row into its buffer
               const int row = q * 32 + lane;
               const int dest = row / rows_per, lrow = row % rows_per;
-              const uint32_t base = mapa_shared(smem_u32(sRed) + static_cast<uint32_t>((ksr * rows_per + lrow) * 128), dest);
-              const uint32_t rbar = mapa_shared(bar_red, dest);
+              // stage the row locally (16-byte chunks XOR-swizzled by the row), then one bulk copy per warp: its 32
+              // rows are contiguous here and in the owner's buffer
+              uint8_t* my = sSend + row * 128;
 #pragma unroll
               for (int c = 0; c < 8; ++c)
-                st_async_cluster_v4(base + ((c ^ (lrow & 7)) << 4), rbar, r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);
+                *reinterpret_cast<uint4*>(my + ((c ^ (row & 7)) << 4)) = make_uint4(r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);
+              fence_proxy_async_smem();
+              __syncwarp();
+              if (lane == 0)
+                bulk_copy_to_cluster(mapa_shared(smem_u32(sRed) + static_cast<uint32_t>((ksr * rows_per + lrow) * 128), dest),
+                                     smem_u32(sSend) + static_cast<uint32_t>(row * 128), 32 * 128, mapa_shared(bar_red, dest));
               // finish my rows of the tile: thread t handles row t / 2, columns 16 (t % 2) .. + 16
               if (mbar_wait_cluster(bar_red, tphase)) {
                 if (finisher) {
@@ -349,7 +397,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
           }
         }
         // the ring position advances identically in the threads that did not walk it
-        if (!(warp <= 1 && lane == 0)) {
+        if (!manual_a && !(warp <= 1 && lane == 0)) {
           const int pos = stage + my_nkb;
           phase ^= (pos / CH_STAGES) & 1;
           stage = pos % CH_STAGES;
@@ -399,7 +447,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
 
 size_t mlp_chain_smem_bytes(size_t w_smem_bytes, int a_stages, int a_stage_bytes) {
   return ((static_cast<size_t>(a_stages) * a_stage_bytes + 1023) & ~size_t(1023)) +
-         (w_smem_bytes < 16384 ? size_t(16384) : w_smem_bytes) + CH_RED_BYTES + 1024 + 1024;
+         (w_smem_bytes < 16384 ? size_t(16384) : w_smem_bytes) + 2 * CH_RED_BYTES + 1024 + 1024;
 }
 
 cudaError_t launch_mlp_chain(int kind, const ChainParams& p, int grid, cudaStream_t s) {
