@@ -270,17 +270,20 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           if (!mbar_wait(bar_p_full + 8 * bx(buf, b), fpar)) { failed = true; break; }
           if (b == 0 && !mbar_wait(bar_o_free + 8 * buf, fpar ^ 1)) { failed = true; break; }
           tc_fence_after();
-          mma2(n, b);
-          if (b == NB - 1) {
-            umma_commit(bar_o_full + 8 * buf);
-            umma_commit(bar_kv_empty + 8 * s);
-          }
-          if (has_next && !next_issued && slots == 2) {         // same buffer: block by block as it frees up
+          // Same buffer: the next unit's scores block by block as the columns free up - and BEFORE this unit's
+          // P.V for the block: the softmax warps will wait for those scores, nobody waits for this O yet, and
+          // the tensor pipe runs the MMAs in issue order.
+          if (has_next && !next_issued && slots == 2) {
             if (!next_ready) {
               if (!wait_inputs(n + 1)) { failed = true; break; }
               next_ready = true;
             }
             if (!mma1(n + 1, b)) { failed = true; break; }
+          }
+          mma2(n, b);
+          if (b == NB - 1) {
+            umma_commit(bar_o_full + 8 * buf);
+            umma_commit(bar_kv_empty + 8 * s);
           }
         }
         if (!failed && has_next && !next_issued && slots == 1) {
@@ -421,7 +424,9 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         if constexpr (INT8) {
           const bool all_masked = __all_sync(0xffffffffu, p.skip_thr > 0.f && mv <= -p.skip_thr);
           const bool any_valid = __any_sync(0xffffffffu, mv >= -1.0f);
-          if (lane == 0) sChunk[s * 16 + (j >> 5)] = all_masked ? 1u : (any_valid ? 2u : 0u);
+          // bit 2: all 32 keys of the chunk carry the same mask value, so the largest score is the largest accumulator
+          const bool uniform = __all_sync(0xffffffffu, __float_as_uint(mv) == __shfl_sync(0xffffffffu, __float_as_uint(mv), 0));
+          if (lane == 0) sChunk[s * 16 + (j >> 5)] = (all_masked ? 1u : (any_valid ? 2u : 0u)) | (uniform ? 4u : 0u);
         }
       }
       if (INT8 && !p.q_signed) {
@@ -458,6 +463,8 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     const int r = q * 32 + lane;                                // query row within the tile = TMEM lane
     const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
     const float c2 = (INT8 ? __fmul_rn(p.dq1, p.scalar) : p.scalar) * LOG2E;
+    const float neg_c0 = -__fmul_rn(MAGIC_F, c2);                // cancels the bias of the int -> float trick inside an FMA
+    const float rho = fmaf(MAGIC_F, c2, neg_c0);                 // ... up to this rounding residue, a launch-wide constant
     const uint32_t row_off = (r >> 3) * 1024 + (r & 7) * 128;
     uint32_t xphase = 0;
     // statistics shared between the four threads of a row and the auxiliary warps: [kind][unit parity][group][row]
@@ -488,15 +495,15 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       if constexpr (INT8) {
         const uint32_t* fl = sChunk + s * 16;
         bool any_valid = false;
-        for (int i = 0; i < NB * 4; ++i) any_valid = any_valid || fl[i] == 2u;
+        for (int i = 0; i < NB * 4; ++i) any_valid = any_valid || (fl[i] & 3u) == 2u;
         if (any_valid)
-          while (nbp > 0 && fl[(nbp - 1) * 4 + g] == 1u) --nbp;
+          while (nbp > 0 && (fl[(nbp - 1) * 4 + g] & 3u) == 1u) --nbp;
       }
 
       // ---------------- pass A: one 32-column chunk per key block, transformed in place
       // (accumulator -> scaled, masked score [-> exponential, stored back to tensor memory on the int8 path])
       float m = -INFINITY, l = 0.f;
-      float mc[3] = {0.f, 0.f, 0.f};                            // running max after each block (int8)
+      float mc[3] = {0.f, 0.f, 0.f};                            // int8: the exponent the stored exponentials of block b refer to
       uint32_t v[32];
       for (int b = 0; b < nbp; ++b) {
         const int col = b * 128 + g * 32;
@@ -505,6 +512,39 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         if constexpr (INT8) tmem_wait_st();                     // v[] may still feed the previous block's store
         tmem_ld32(t_row + col, v);
         tmem_wait_ld();
+        if (INT8 && (sChunk[s * 16 + b * 4 + g] & 4u)) {
+          // Uniform mask over my 32 keys (the usual case: unmasked, or padding): the largest score belongs to the
+          // largest accumulator, found with integer compares.  With it as the reference, each exponential is
+          // 2^((a - a_max) c2): the integer difference goes through the 1.5 * 2^23 bias trick in ONE add
+          // (|a - a_max| < 2^22 for 64-wide heads), the FMA's addend cancels the bias (its rounding residue is the
+          // same factor for every score of the launch and drops out of the softmax), and no per-score
+          // max or subtraction is left.
+          int vm[4] = {static_cast<int>(v[0]), static_cast<int>(v[1]), static_cast<int>(v[2]), static_cast<int>(v[3])};
+#pragma unroll
+          for (int i = 4; i < 32; i += 4) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) vm[j] = max(vm[j], static_cast<int>(v[i + j]));
+          }
+          const int vmax = max(max(vm[0], vm[1]), max(vm[2], vm[3]));
+          const float tmax = fmaf(__int2float_rn(vmax), c2, mk[col]);    // largest scaled, masked score of the chunk
+          const float m_new = fmaxf(m, tmax);
+          const int kadd = MAGIC_I - vmax;
+          float sm[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+          for (int i = 0; i < 32; i += 4) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const float e = ex2(fmaf(__int_as_float(static_cast<int>(v[i + j]) + kadd), c2, neg_c0));
+              v[i + j] = __float_as_uint(e);
+              sm[j] += e;
+            }
+          }
+          l = l * ex2(m - m_new) + ((sm[0] + sm[1]) + (sm[2] + sm[3])) * ex2(tmax - m_new);
+          m = m_new;
+          if (b == 0) mc[0] = tmax; else if (b == 1) mc[1] = tmax; else mc[2] = tmax;
+          tmem_st32(t_row + col, v);
+          continue;
+        }
         const float4* mk4 = reinterpret_cast<const float4*>(mk + col);
         float cm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
@@ -522,12 +562,13 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const float cmax = fmaxf(fmaxf(cm[0], cm[1]), fmaxf(cm[2], cm[3]));
         if constexpr (INT8) {
           const float m_new = fmaxf(m, cmax);
+          const float m_sub = m_new - rho;                       // same constant factor 2^rho as the fast path above
           float sm[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
           for (int i = 0; i < 32; i += 4) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-              const float e = ex2(__uint_as_float(v[i + j]) - m_new);
+              const float e = ex2(__uint_as_float(v[i + j]) - m_sub);
               v[i + j] = __float_as_uint(e);
               sm[j] += e;
             }

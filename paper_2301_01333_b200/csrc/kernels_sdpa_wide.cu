@@ -211,9 +211,9 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           for (int b = 0; b < NB && !failed; ++b) failed = !load_block(&tmK, unit, b);
         }
         if (ahead && !failed) failed = !load_q(next, n + 1);
-        for (int b = 0; b < NB && !failed; ++b) {
-          failed = !load_block(&tmV, unit, b);
-          if (ahead && !failed) failed = !load_block(&tmK, next, b);
+        for (int b = 0; b < NB && !failed; ++b) {                // the order the MMA issuer consumes them in
+          if (ahead) failed = !load_block(&tmK, next, b);
+          if (!failed) failed = !load_block(&tmV, unit, b);
         }
       }
       if (failed) report(p.status, DEV_TIMEOUT_PRODUCER);
@@ -261,10 +261,14 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (failed) break;
         // O += P_b V_b
         for (int b = 0; b < NB; ++b) {
+          if (!mbar_wait(bar_p_full + 8 * b, upar)) { failed = true; break; }
+          // the next unit's scores for this block first: the softmax warps will wait for them, nobody waits for
+          // this O yet, and the tensor pipe runs the MMAs in issue order
+          if (ahead && !mma1(n + 1, b)) { failed = true; break; }
           const uint32_t st = it % stages, use = it / stages;
           ++it;
           const uint32_t pe = static_cast<uint32_t>(n * NB + b) % np;
-          if (!mbar_wait(bar_p_full + 8 * b, upar) || !mbar_wait(bar_kv_full + 8 * st, use & 1)) { failed = true; break; }
+          if (!mbar_wait(bar_kv_full + 8 * st, use & 1)) { failed = true; break; }
           if (!alias && b == 0 && !mbar_wait(bar_o_free, upar ^ 1)) { failed = true; break; }
           tc_fence_after();
           const uint32_t sP = smem_u32(sPall) + pe * L::P_BYTES;
@@ -284,7 +288,6 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           umma_commit(bar_kv_empty + 8 * st);
           umma_commit(bar_p_free + 8 * pe);
           if (b == NB - 1) umma_commit(bar_o_full);
-          if (ahead && !mma1(n + 1, b)) { failed = true; break; }
         }
       }
       if (failed) report(p.status, DEV_TIMEOUT_MMA);
