@@ -204,17 +204,22 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         return true;
       };
       for (int unit = blockIdx.x; unit < num_units && !failed; unit += gridDim.x, ++n) {
+        // Blocks go into the ring in the order the MMA issuer consumes them: the next unit's K block b right before
+        // this unit's V block b.  When O shares the columns of score block 0, that block's K comes last: its
+        // Q.K^T has to wait for the previous unit's output to be read, the others need not.
         const int next = unit + static_cast<int>(gridDim.x);
-        const bool ahead = !alias && next < num_units;          // next unit's K blocks interleaved with my V blocks
-        if (alias || n == 0) {
-          failed = !load_q(unit, n);
-          for (int b = 0; b < NB && !failed; ++b) failed = !load_block(&tmK, unit, b);
+        const bool ahead = next < num_units;
+        const int b_first = alias ? 1 : 0;
+        if (n == 0) {
+          failed = !load_q(unit, 0);
+          for (int i = 0; i < NB && !failed; ++i) failed = !load_block(&tmK, unit, (b_first + i) % NB);
         }
         if (ahead && !failed) failed = !load_q(next, n + 1);
-        for (int b = 0; b < NB && !failed; ++b) {                // the order the MMA issuer consumes them in
-          if (ahead) failed = !load_block(&tmK, next, b);
+        for (int b = 0; b < NB && !failed; ++b) {
+          if (ahead && b >= b_first) failed = !load_block(&tmK, next, b);
           if (!failed) failed = !load_block(&tmV, unit, b);
         }
+        if (ahead && alias && !failed) failed = !load_block(&tmK, next, 0);
       }
       if (failed) report(p.status, DEV_TIMEOUT_PRODUCER);
     }
@@ -235,12 +240,14 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       uint32_t it = 0;
       for (int unit = blockIdx.x; unit < num_units && !failed; unit += gridDim.x, ++n) {
         const uint32_t upar = n & 1;
-        const bool ahead = !alias && unit + static_cast<int>(gridDim.x) < num_units;
+        const bool ahead = unit + static_cast<int>(gridDim.x) < num_units;
+        const int b_first = alias ? 1 : 0;                      // first / last score block of a unit in issue order
+        const int b_last = alias ? 0 : NB - 1;
         // S_b = Q K_b^T for this CTA's nn-th unit (block b of the ring's next stage)
         auto mma1 = [&](int nn, int b) -> bool {
           const uint32_t st = it % stages, use = it / stages, par = nn & 1;
           ++it;
-          if (b == 0 && !mbar_wait(bar_q_ready, par)) return false;
+          if (b == b_first && !mbar_wait(bar_q_ready, par)) return false;
           if (!mbar_wait(bar_kv_full + 8 * st, use & 1) || !mbar_wait(bar_s_free + 8 * b, par ^ 1)) return false;
           if (alias && b == 0 && !mbar_wait(bar_o_free, par ^ 1)) return false;
           tc_fence_after();
@@ -253,18 +260,18 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           }
           umma_commit(bar_s_full + 8 * b);
           umma_commit(bar_kv_empty + 8 * st);
-          if (b == NB - 1) umma_commit(bar_q_empty);
+          if (b == b_last) umma_commit(bar_q_empty);
           return true;
         };
-        if (alias || n == 0)
-          for (int b = 0; b < NB && !failed; ++b) failed = !mma1(n, b);
+        if (n == 0)
+          for (int i = 0; i < NB && !failed; ++i) failed = !mma1(0, (b_first + i) % NB);
         if (failed) break;
         // O += P_b V_b
         for (int b = 0; b < NB; ++b) {
           if (!mbar_wait(bar_p_full + 8 * b, upar)) { failed = true; break; }
           // the next unit's scores for this block first: the softmax warps will wait for them, nobody waits for
           // this O yet, and the tensor pipe runs the MMAs in issue order
-          if (ahead && !mma1(n + 1, b)) { failed = true; break; }
+          if (ahead && b >= b_first && !mma1(n + 1, b)) { failed = true; break; }
           const uint32_t st = it % stages, use = it / stages;
           ++it;
           const uint32_t pe = static_cast<uint32_t>(n * NB + b) % np;
@@ -289,6 +296,8 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           umma_commit(bar_p_free + 8 * pe);
           if (b == NB - 1) umma_commit(bar_o_full);
         }
+        // score block 0 of the next unit overwrites this unit's O: issued once the epilogue has read it
+        if (!failed && ahead && alias && !mma1(n + 1, 0)) failed = true;
       }
       if (failed) report(p.status, DEV_TIMEOUT_MMA);
     }
@@ -466,7 +475,9 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       float m = -INFINITY, l = 0.f;
       float mc[4] = {0.f, 0.f, 0.f, 0.f};                       // running max after each block (int8)
       uint32_t v[32];
-      for (int b = 0; b < nbp; ++b) {
+      for (int i = 0; i < nbp; ++i) {
+        // when O shares columns with score block 0, that block's Q.K^T is the last one issued: take it last
+        const int b = alias ? (i + 1 < nbp ? i + 1 : 0) : i;
         const int col = b * 128 + g * 32;
         if (!mbar_wait(bar_s_full + 8 * b, upar)) { failed = true; break; }
         tc_fence_after();

@@ -167,6 +167,33 @@ def test_int8_matmul_nonzero_zero_point_on_tensor_cores_exact(B, m, k, n, zp):
     assert np.array_equal(got.astype(np.int64), oracle(w))
 
 
+@pytest.mark.parametrize("batch,dims,ks", [(64, (600, 256, 64), 2), (77, (700, 128, 32), 2), (33, (131, 64, 16), 1),
+                                           (128, (1030, 512, 256, 32), 4), (1, (479, 1024, 16), 4)])
+def test_mlp_int8_chain_kernel_cluster_sizes_and_entry_reorder(B, batch, dims, ks):
+    # the fused chain kernel with the reduction axis split over 1, 2 and 4 CTAs, inputs whose rows start at every
+    # byte alignment (the graph-entry reorder inside the kernel) and reductions that end inside a k-block
+    w = W.mlp_int8(batch=batch, dims=dims, final="none", per_channel=True, x_zp=3, act_zp=7)
+    got, plan = run_gpu(B, w)
+    assert f"clusters of {ks}" in plan
+    assert np.array_equal(got, oracle(w))
+
+
+@pytest.mark.parametrize("batch,dims,ks", [(16, (160, 64, 32), 2), (100, (13, 1024, 48), 4), (128, (37, 32, 16), 1)])
+def test_mlp_f32_chain_kernel_cluster_sizes(B, batch, dims, ks):
+    w = W.mlp_f32(batch=batch, dims=dims)
+    got, plan = run_gpu(B, w)
+    assert f"clusters of {ks}" in plan
+    ref = oracle(w)
+    assert np.abs(got.astype(np.float64) - ref).max() <= 5e-3 * np.abs(ref).max()
+
+
+def test_ffn_bf16_chain_kernel_with_split_reduction(B):
+    w = W.ffn_bf16(tokens=96, d_model=512, d_ff=256)
+    got, plan = run_gpu(B, w)
+    assert "clusters of 4" in plan
+    assert np.abs(bf16_to_f64(got) - oracle(w)).max() <= 2e-2
+
+
 def test_mlp_int8_hidden_layer_codes_bit_exact(B):
     # a chain that ends on a requantised u8 tensor: compares the codes themselves
     w = W.mlp_int8(batch=128, dims=(479, 1024, 512), final="none")
