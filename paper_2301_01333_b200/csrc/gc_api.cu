@@ -216,6 +216,12 @@ struct LayerPlan {
   int Kp = 0;
   std::vector<float> dqv_host;   // per-channel weights: float32(a_scale) * float32(w_scale[n]) per output column
   size_t dqv_off = 0;            // workspace offset of their device copy
+  // this layer and the next one run as one launch of the CTA-pair GEMM (kernels_gemm_tc2_fused.cu)
+  bool fused_first = false;
+  std::vector<int> pair_sched;   // [clusters][pair_pitch] tile lists: (layer << 24) | tile, -1 terminated
+  int pair_pitch = 0, pair_clusters = 0;
+  size_t pair_sched_off = 0, pair_ready_off = 0;
+  unsigned long long pair_execs = 0;   // launches since the counters were cleared
   bool need_comp = false;        // tcgen05 path with a non-zero activation zero point
   size_t comp_off = 0;           // workspace offset of a_zp * colsum(W), s32 per output column
   // cached tensor maps
@@ -778,6 +784,101 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
       c->desc += line;
     }
   }
+  // Two consecutive large layers on CTA pairs: one launch with a tile schedule over both (see the kernel's header).
+  if (c->pattern == PAT_MLP && !c->chain_fused && !c->opt.no_chain_fusion && !c->opt.force_generic) {
+    auto out_kind = [](const LayerPlan& L) {
+      return L.epi.out_dtype == GC_BF16 ? 1 : (L.epi.out_dtype == GC_F32 ? 2 : ((L.epi.acc_is_int && !L.epi.has_dq) ? 3 : 0));
+    };
+    for (size_t l = 0; l + 1 < c->layers.size(); ++l) {
+      LayerPlan& A = c->layers[l];
+      LayerPlan& B = c->layers[l + 1];
+      if (l > 0 && c->layers[l - 1].fused_first) continue;       // A is already the second half of a pair
+      const bool kinds_ok = A.use_tc && B.use_tc && A.cta2 && B.cta2 && A.kind == B.kind && A.M == B.M && !B.need_pack &&
+                            out_kind(A) == out_kind(B) && out_kind(A) == A.kind;   // i8 -> 8-bit, bf16 -> bf16, tf32 -> f32
+      if (!kinds_ok) continue;
+      const int C = c->num_sms / 2;
+      const int m_pairs = (A.m_tiles + 1) / 2;
+      const long T0 = static_cast<long>(m_pairs) * A.n_tiles, T1 = static_cast<long>(m_pairs) * B.n_tiles;
+      const long w0 = A.nkb, w1 = B.nkb;
+      if (T0 + T1 < 2L * C || T0 >= (1L << 24) || T1 >= (1L << 24)) continue;
+      // Schedule (static, built here): first-layer tiles in row-block order, round robin over the clusters that
+      // still have quota; second-layer tiles in row-block order, each to the cluster that is free first, starting
+      // no earlier than its row block is ready.  A row block is ready a while after its last first-layer tile's
+      // main loop ends (epilogue, store completion, counter, the poll: about 24 k-block times measured on this
+      // workload), so first-layer work must not end everywhere at the last moment.  The clusters that will take
+      // one second-layer tile fewer take e extra first-layer tiles instead; e is chosen by simulating the step.
+      const long lat = 24;
+      const int heavy = T1 % C ? C - static_cast<int>(T1 % C) : 0;   // clusters with one second-layer tile fewer
+      long best_span = -1;
+      std::vector<int> best_sched;
+      int best_pitch = 0;
+      for (int e = 0; e <= 4; ++e) {
+        if (e > 0 && heavy == 0) break;
+        // first-layer quotas: heavy clusters (the last ones) get e more than the light ones
+        std::vector<long> n0(C, 0);
+        const long light = C - heavy;
+        long base = (T0 - static_cast<long>(heavy) * e) / C;
+        if (base < 0) break;
+        long rest = T0 - base * C - static_cast<long>(heavy) * e;
+        for (int k = 0; k < C; ++k) n0[k] = base + (k >= light ? e : 0);
+        for (int k = 0; rest > 0; k = (k + 1) % C, --rest) ++n0[k];
+        // first layer: tile index -> (cluster, position); finish time of each tile
+        std::vector<std::vector<int>> list(C);
+        std::vector<long> done0(T0);
+        long next0 = 0;
+        while (next0 < T0)
+          for (int k = 0; k < C && next0 < T0; ++k)
+            if (static_cast<long>(list[k].size()) < n0[k]) {
+              list[k].push_back(static_cast<int>(next0));
+              done0[next0] = static_cast<long>(list[k].size()) * w0;
+              ++next0;
+            }
+        std::vector<long> ready(m_pairs, 0), avail(C);
+        for (long t = 0; t < T0; ++t) {
+          const long mp = t / A.n_tiles;
+          ready[mp] = done0[t] + lat > ready[mp] ? done0[t] + lat : ready[mp];
+        }
+        for (int k = 0; k < C; ++k) avail[k] = n0[k] * w0;
+        for (long t = 0; t < T1; ++t) {
+          int bestk = 0;
+          for (int k = 1; k < C; ++k)
+            if (avail[k] < avail[bestk]) bestk = k;
+          const long mp = t / B.n_tiles;
+          const long start = avail[bestk] > ready[mp] ? avail[bestk] : ready[mp];
+          avail[bestk] = start + w1;
+          list[bestk].push_back((1 << 24) | static_cast<int>(t));
+        }
+        long span = 0;
+        size_t longest = 0;
+        for (int k = 0; k < C; ++k) {
+          span = avail[k] > span ? avail[k] : span;
+          longest = list[k].size() > longest ? list[k].size() : longest;
+        }
+        if (best_span < 0 || span < best_span) {
+          best_span = span;
+          best_pitch = static_cast<int>(longest) + 1;
+          best_sched.assign(static_cast<size_t>(C) * best_pitch, -1);
+          for (int k = 0; k < C; ++k)
+            for (size_t i = 0; i < list[k].size(); ++i) best_sched[static_cast<size_t>(k) * best_pitch + i] = list[k][i];
+        }
+      }
+      if (best_span < 0) continue;
+      A.pair_pitch = best_pitch;
+      A.pair_clusters = C;
+      A.pair_sched = best_sched;
+      const long worst = best_span;
+      const double target = static_cast<double>(T0 * w0 + T1 * w1) / C;
+      A.fused_first = true;
+      A.pair_sched_off = ws;
+      ws = align_up(ws + A.pair_sched.size() * sizeof(int), 256);
+      A.pair_ready_off = ws;
+      ws = align_up(ws + static_cast<size_t>(m_pairs) * sizeof(unsigned long long), 256);
+      c->launches -= 1;
+      snprintf(line, sizeof(line), "  layers %zu+%zu: one launch, %d clusters, tile schedule over both (longest list %ld of %.1f k-blocks ideal)\n",
+               l, l + 1, C, worst, target);
+      c->desc += line;
+    }
+  }
   c->ws_bytes = align_up(ws, 1024);
   // host staging layout
   size_t so = 0;
@@ -859,6 +960,13 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
       if (L.need_comp)
         CUDA_TRY(launch_weight_compensation(ws + L.wt_off, L.N, L.Kp, L.a_zp, reinterpret_cast<int*>(ws + L.comp_off), st));
       c.const_ptrs[L.w_input] = in[L.w_input];
+      if (L.fused_first) {
+        CUDA_TRY(cudaMemcpyAsync(ws + L.pair_sched_off, L.pair_sched.data(), L.pair_sched.size() * sizeof(int),
+                                 cudaMemcpyHostToDevice, st));
+        const int m_pairs = (L.m_tiles + 1) / 2;
+        CUDA_TRY(cudaMemsetAsync(ws + L.pair_ready_off, 0, static_cast<size_t>(m_pairs) * sizeof(unsigned long long), st));
+        L.pair_execs = 0;
+      }
     }
     c.prepacked = true;
   }
@@ -936,6 +1044,7 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
     c.chain_arrivals += static_cast<unsigned long long>(c.chain_barriers) * c.chain_grid;
     return GC_OK;
   }
+  GemmTcParams pair_first = {};
   for (size_t l = 0; l < c.layers.size(); ++l) {
     LayerPlan& L = c.layers[l];
     const int esz = dtype_bytes(L.a_dtype);
@@ -985,6 +1094,34 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
       // Programmatic dependent launch, also for the first layer: whatever ran before on the stream, this kernel's
       // set-up overlaps its tail and the kernel waits for it to complete before it touches global memory
       const bool pdl = !c.opt.no_chain_fusion && !L.need_pack;
+      if (L.fused_first) {
+        pair_first = g;                                            // launched together with the next layer
+        continue;
+      }
+      if (l > 0 && c.layers[l - 1].fused_first) {
+        LayerPlan& F = c.layers[l - 1];
+        GemmPairParams pp = {};
+        const GemmTcParams* gs[2] = {&pair_first, &g};
+        const LayerPlan* ls[2] = {&F, &L};
+        for (int k = 0; k < 2; ++k) {
+          pp.L[k].N = gs[k]->N;
+          pp.L[k].num_k_blocks = gs[k]->num_k_blocks;
+          pp.L[k].n_tiles = gs[k]->n_tiles;
+          pp.L[k].epi = gs[k]->epi;
+          pp.tm[3 * k] = ls[k]->tmA;
+          pp.tm[3 * k + 1] = ls[k]->tmB;
+          pp.tm[3 * k + 2] = ls[k]->tmD;
+        }
+        pp.sched = reinterpret_cast<const int*>(ws + F.pair_sched_off);
+        pp.sched_pitch = F.pair_pitch;
+        pp.ready = reinterpret_cast<unsigned long long*>(ws + F.pair_ready_off);
+        // every epilogue warp of both CTAs adds one per first-layer tile of the row block
+        pp.ready_target = (F.pair_execs + 1) * static_cast<unsigned long long>(F.n_tiles) * 16ull;
+        pp.status = status;
+        CUDA_TRY(launch_gemm_tc2_fused(L.kind, F.a_dtype == GC_S8, pp, 2 * F.pair_clusters, st));
+        ++F.pair_execs;
+        continue;
+      }
       if (L.cta2)
         CUDA_TRY(launch_gemm_tc2(L.kind, L.a_dtype == GC_S8, L.tmA, L.tmB, L.tmD, g, L.grid, pdl, st));
       else

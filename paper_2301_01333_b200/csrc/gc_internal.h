@@ -81,6 +81,23 @@ struct SdpaParams {
   uint32_t* status;
 };
 
+// Two consecutive large fused ops in one launch of the CTA-pair GEMM (kernels_gemm_tc2_fused.cu).
+struct GemmPairLayer {
+  int N, num_k_blocks, n_tiles;   // n_tiles: 256-column tiles per 256-row block
+  uint32_t idesc;                 // tcgen05 instruction descriptor (filled by the launcher)
+  Epilogue epi;
+};
+struct GemmPairParams {
+  GemmPairLayer L[2];
+  const int* sched;               // [clusters][sched_pitch]: (layer << 24) | tile, a negative entry ends a list
+  int sched_pitch;
+  unsigned long long* ready;      // per 256-row block: completed stores of the first layer (only grows)
+  unsigned long long ready_target;   // the value a block's counter reaches in this launch
+  uint32_t* status;
+  alignas(64) CUtensorMap tm[6];  // A, Wt, D of the first layer, then of the second
+};
+cudaError_t launch_gemm_tc2_fused(int kind, int a_signed, const GemmPairParams& p, int grid, cudaStream_t s);
+
 // One layer of the fused small-batch chain kernel (kernels_chain.cu).
 constexpr int CHAIN_MAX_LAYERS = 8;
 struct ChainLayer {

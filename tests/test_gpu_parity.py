@@ -187,6 +187,26 @@ def test_mlp_f32_chain_kernel_cluster_sizes(B, batch, dims, ks):
     assert np.abs(got.astype(np.float64) - ref).max() <= 5e-3 * np.abs(ref).max()
 
 
+def test_two_large_layers_in_one_launch_bf16(B):
+    # both GEMMs on CTA pairs in one persistent launch (row-block counters between them); 39 row tiles: the last
+    # pair is half empty
+    w = W.ffn_bf16(tokens=4900, d_model=1024, d_ff=1024)
+    got, plan = run_gpu(B, w, n_runs=2)
+    assert "one launch" in plan
+    assert np.array_equal(got[0], got[1])
+    assert np.abs(bf16_to_f64(got[0]) - oracle(w)).max() <= 2e-2
+    sep, plan2 = run_gpu(B, w, no_chain_fusion=True)
+    assert "one launch" not in plan2
+    assert np.array_equal(sep, got[0])                   # same tiles, same arithmetic: identical bits
+
+
+def test_two_large_layers_in_one_launch_int8_bit_exact(B):
+    w = W.mlp_int8(batch=4900, dims=(1024, 1024, 1024, 16), final="none", per_channel=True, x_zp=9, act_zp=4)
+    got, plan = run_gpu(B, w)
+    assert "layers 0+1: one launch" in plan
+    assert np.array_equal(got, oracle(w))
+
+
 def test_ffn_bf16_chain_kernel_with_split_reduction(B):
     w = W.ffn_bf16(tokens=96, d_model=512, d_ff=256)
     got, plan = run_gpu(B, w)
