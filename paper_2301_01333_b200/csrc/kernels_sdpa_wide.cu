@@ -184,7 +184,13 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       int n = 0;
-      uint32_t it = 0;                                          // ring position: stage it % stages, use it / stages
+      uint32_t ring_st = 0, ring_use = 0;                        // ring position: stage and how often the ring has wrapped
+      auto ring_next = [&]() {
+        if (++ring_st == static_cast<uint32_t>(stages)) {
+          ring_st = 0;
+          ++ring_use;
+        }
+      };
       auto load_q = [&](int u, int nn) -> bool {                 // Q tile of unit u, this CTA's nn-th unit
         if (!mbar_wait(bar_q_empty, (nn & 1) ^ 1)) return false;
         mbar_arrive_expect_tx(bar_q_full, static_cast<uint32_t>(L::TILE_BYTES));
@@ -194,8 +200,8 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         return true;
       };
       auto load_block = [&](const CUtensorMap* tm, int u, int b) -> bool {   // one 128-key block into the next stage
-        const uint32_t st = it % stages, use = it / stages;
-        ++it;
+        const uint32_t st = ring_st, use = ring_use;
+        ring_next();
         if (!mbar_wait(bar_kv_empty + 8 * st, (use & 1) ^ 1)) return false;
         mbar_arrive_expect_tx(bar_kv_full + 8 * st, static_cast<uint32_t>(L::TILE_BYTES));
         for (int j = 0; j < L::NSUB; ++j)
@@ -237,7 +243,13 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                          : make_idesc(ACC_F32, FMT_BF16, FMT_BF16, 128, nj, 0, 1);
       }
       int n = 0;
-      uint32_t it = 0;
+      uint32_t ring_st = 0, ring_use = 0, pe = 0;                // K/V ring position; P ring entry of the next block
+      auto ring_next = [&]() {
+        if (++ring_st == static_cast<uint32_t>(stages)) {
+          ring_st = 0;
+          ++ring_use;
+        }
+      };
       for (int unit = blockIdx.x; unit < num_units && !failed; unit += gridDim.x, ++n) {
         const uint32_t upar = n & 1;
         const bool ahead = unit + static_cast<int>(gridDim.x) < num_units;
@@ -245,8 +257,8 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const int b_last = alias ? 0 : NB - 1;
         // S_b = Q K_b^T for this CTA's nn-th unit (block b of the ring's next stage)
         auto mma1 = [&](int nn, int b) -> bool {
-          const uint32_t st = it % stages, use = it / stages, par = nn & 1;
-          ++it;
+          const uint32_t st = ring_st, use = ring_use, par = nn & 1;
+          ring_next();
           if (b == b_first && !mbar_wait(bar_q_ready, par)) return false;
           if (!mbar_wait(bar_kv_full + 8 * st, use & 1) || !mbar_wait(bar_s_free + 8 * b, par ^ 1)) return false;
           if (alias && b == 0 && !mbar_wait(bar_o_free, par ^ 1)) return false;
@@ -272,9 +284,8 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           // the next unit's scores for this block first: the softmax warps will wait for them, nobody waits for
           // this O yet, and the tensor pipe runs the MMAs in issue order
           if (ahead && b >= b_first && !mma1(n + 1, b)) { failed = true; break; }
-          const uint32_t st = it % stages, use = it / stages;
-          ++it;
-          const uint32_t pe = static_cast<uint32_t>(n * NB + b) % np;
+          const uint32_t st = ring_st, use = ring_use;
+          ring_next();
           if (!mbar_wait(bar_kv_full + 8 * st, use & 1)) { failed = true; break; }
           if (!alias && b == 0 && !mbar_wait(bar_o_free, upar ^ 1)) { failed = true; break; }
           tc_fence_after();
@@ -294,6 +305,7 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           }
           umma_commit(bar_kv_empty + 8 * st);
           umma_commit(bar_p_free + 8 * pe);
+          if (++pe == static_cast<uint32_t>(np)) pe = 0;
           if (b == NB - 1) umma_commit(bar_o_full);
         }
         // score block 0 of the next unit overwrites this unit's O: issued once the epilogue has read it
@@ -411,7 +423,9 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if constexpr (INT8) {
           const bool all_masked = __all_sync(0xffffffffu, p.skip_thr > 0.f && mv <= -p.skip_thr);
           const bool any_valid = __any_sync(0xffffffffu, mv >= -1.0f);
-          if (lane == 0) sChunk[(n & 1) * 16 + (j >> 5)] = all_masked ? 1u : (any_valid ? 2u : 0u);
+          // bit 2: all 32 keys of the chunk carry the same mask value, so the largest score is the largest accumulator
+          const bool uniform = __all_sync(0xffffffffu, __float_as_uint(mv) == __shfl_sync(0xffffffffu, __float_as_uint(mv), 0));
+          if (lane == 0) sChunk[(n & 1) * 16 + (j >> 5)] = (all_masked ? 1u : (any_valid ? 2u : 0u)) | (uniform ? 4u : 0u);
         }
       }
       if (INT8 && !p.q_signed) {
@@ -446,8 +460,11 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const int r = q * 32 + lane;                                // query row within the tile = TMEM lane
     const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
     const float c2 = (INT8 ? __fmul_rn(p.dq1, p.scalar) : p.scalar) * W_LOG2E;
+    const float neg_c0 = -__fmul_rn(W_MAGIC_F, c2);              // cancels the bias of the int -> float trick inside an FMA
+    const float rho = fmaf(W_MAGIC_F, c2, neg_c0);               // ... up to this rounding residue, a launch-wide constant
     const uint32_t row_off = (r >> 3) * 1024 + (r & 7) * 128;
     uint32_t xphase = 0;
+    uint32_t p_entry = 0, p_use = 0;                              // P ring: entry of the next block, wraps so far
     auto stat = [&](int kind, int par, int grp) { return sStat + ((kind * 2 + par) * 4 + grp) * 128 + r; };
     auto xchg_sync = [&]() -> bool {
       __syncwarp();
@@ -466,9 +483,9 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       if constexpr (INT8) {
         const uint32_t* fl = sChunk + (n & 1) * 16;
         bool any_valid = false;
-        for (int i = 0; i < NB * 4; ++i) any_valid = any_valid || fl[i] == 2u;
+        for (int i = 0; i < NB * 4; ++i) any_valid = any_valid || (fl[i] & 3u) == 2u;
         if (any_valid)
-          while (nbp > 0 && fl[(nbp - 1) * 4 + g] == 1u) --nbp;
+          while (nbp > 0 && (fl[(nbp - 1) * 4 + g] & 3u) == 1u) --nbp;
       }
 
       // ---------------- pass A: scale + mask, running row max [int8: exp2 and running sum, written back]
@@ -484,6 +501,37 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if constexpr (INT8) tmem_wait_st();                     // v[] may still feed the previous block's store
         tmem_ld32(t_row + col, v);
         tmem_wait_ld();
+        if (INT8 && D <= 64 && (sChunk[(n & 1) * 16 + b * 4 + g] & 4u)) {
+          // Uniform mask over my 32 keys: the largest score belongs to the largest accumulator (integer compares);
+          // with it as the reference each exponential is 2^((a - a_max) c2), the integer difference going through
+          // the 1.5 * 2^23 bias trick in one add (|a - a_max| < 2^22 for heads up to 64 wide) and the FMA's addend
+          // cancelling the bias; its rounding residue is the same factor for every score of the launch.
+          int vm[4] = {static_cast<int>(v[0]), static_cast<int>(v[1]), static_cast<int>(v[2]), static_cast<int>(v[3])};
+#pragma unroll
+          for (int ii = 4; ii < 32; ii += 4) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) vm[j] = max(vm[j], static_cast<int>(v[ii + j]));
+          }
+          const int vmax = max(max(vm[0], vm[1]), max(vm[2], vm[3]));
+          const float tmax = fmaf(__int2float_rn(vmax), c2, mk[col]);
+          const float m_new = fmaxf(m, tmax);
+          const int kadd = W_MAGIC_I - vmax;
+          float sm[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+          for (int ii = 0; ii < 32; ii += 4) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const float e = w_ex2(fmaf(__int_as_float(static_cast<int>(v[ii + j]) + kadd), c2, neg_c0));
+              v[ii + j] = __float_as_uint(e);
+              sm[j] += e;
+            }
+          }
+          l = l * w_ex2(m - m_new) + ((sm[0] + sm[1]) + (sm[2] + sm[3])) * w_ex2(tmax - m_new);
+          m = m_new;
+          if (b == 0) mc[0] = tmax; else if (b == 1) mc[1] = tmax; else if (b == 2) mc[2] = tmax; else mc[3] = tmax;
+          tmem_st32(t_row + col, v);
+          continue;
+        }
         const float4* mk4 = reinterpret_cast<const float4*>(mk + col);
         float cm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
@@ -501,12 +549,13 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const float cmax = fmaxf(fmaxf(cm[0], cm[1]), fmaxf(cm[2], cm[3]));
         if constexpr (INT8) {
           const float m_new = fmaxf(m, cmax);
+          const float m_sub = D <= 64 ? m_new - rho : m_new;      // same constant factor 2^rho as the fast path above
           float sm[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
           for (int i = 0; i < 32; i += 4) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-              const float e = w_ex2(__uint_as_float(v[i + j]) - m_new);
+              const float e = w_ex2(__uint_as_float(v[i + j]) - m_sub);
               v[i + j] = __float_as_uint(e);
               sm[j] += e;
             }
@@ -541,8 +590,11 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       float lsum = 0.f;
       for (int b = 0; b < nbp; ++b) {
         const int col = b * 128 + g * 32;
-        const uint32_t pseq = static_cast<uint32_t>(n * NB + b);
-        const uint32_t pe = pseq % np, puse = pseq / np;
+        const uint32_t pe = p_entry, puse = p_use;
+        if (++p_entry == static_cast<uint32_t>(np)) {
+          p_entry = 0;
+          ++p_use;
+        }
         uint8_t* sP = sPall + pe * L::P_BYTES;
         if constexpr (INT8) {
           uint32_t w[8];
@@ -622,8 +674,11 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       if constexpr (INT8) {
         for (int b = nbp; b < NB; ++b) {                        // skipped chunks: their codes are zero
           const int col = b * 128 + g * 32;
-          const uint32_t pseq = static_cast<uint32_t>(n * NB + b);
-          const uint32_t pe = pseq % np, puse = pseq / np;
+          const uint32_t pe = p_entry, puse = p_use;
+          if (++p_entry == static_cast<uint32_t>(np)) {
+            p_entry = 0;
+            ++p_use;
+          }
           if (!mbar_wait(bar_p_free + 8 * pe, (puse & 1) ^ 1)) { failed = true; break; }
           uint8_t* blk = sPall + pe * L::P_BYTES + row_off;
           const int c0 = g * 2;
