@@ -43,7 +43,7 @@ DEFAULT_STEPS = {"c1": 2000, "c2": 2000, "c3": 500, "c4": 100, "c5": 8000}
 # (dram__bytes_read.sum + dram__bytes_write.sum; c5: one launch per step, the 64 MiB hidden tensor is written back)
 TRAFFIC_BYTES_PER_LAUNCH = {"c5": 135.4e6, "c3": None, "c4": 84.8e6}
 DOMINANT_KERNEL = {"c1": "mlp_chain_kernel<tf32>", "c2": "mlp_chain_kernel<i8>", "c3": "sdpa_tc_kernel<bf16>",
-                   "c4": "sdpa_tc_kernel<int8>", "c5": "gemm_tc2_fused_kernel<bf16, bf16 out>"}
+                   "c4": "sdpa_tc_kernel<int8>", "c5": "gemm_tc2_kernel<bf16, bf16 out> (both FFN GEMMs in one launch)"}
 
 
 def load_peaks():

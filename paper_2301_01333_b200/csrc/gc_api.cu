@@ -216,7 +216,7 @@ struct LayerPlan {
   int Kp = 0;
   std::vector<float> dqv_host;   // per-channel weights: float32(a_scale) * float32(w_scale[n]) per output column
   size_t dqv_off = 0;            // workspace offset of their device copy
-  // this layer and the next one run as one launch of the CTA-pair GEMM (kernels_gemm_tc2_fused.cu)
+  // this layer and the next one run as one launch of the CTA-pair GEMM (kernels_gemm_tc2.cu)
   bool fused_first = false;
   std::vector<int> pair_sched;   // [clusters][pair_pitch] tile lists: (layer << 24) | tile, -1 terminated
   int pair_pitch = 0, pair_clusters = 0;

@@ -81,7 +81,7 @@ struct SdpaParams {
   uint32_t* status;
 };
 
-// Two consecutive large fused ops in one launch of the CTA-pair GEMM (kernels_gemm_tc2_fused.cu).
+// One layer, or two consecutive large fused ops in one launch, of the CTA-pair GEMM (kernels_gemm_tc2.cu).
 struct GemmPairLayer {
   int N, num_k_blocks, n_tiles;   // n_tiles: 256-column tiles per 256-row block
   uint32_t idesc;                 // tcgen05 instruction descriptor (filled by the launcher)
@@ -89,9 +89,10 @@ struct GemmPairLayer {
 };
 struct GemmPairParams {
   GemmPairLayer L[2];
-  const int* sched;               // [clusters][sched_pitch]: (layer << 24) | tile, a negative entry ends a list
-  int sched_pitch;
-  unsigned long long* ready;      // per 256-row block: completed stores of the first layer (only grows)
+  const int* sched;               // [clusters][sched_pitch]: (layer << 24) | tile, a negative entry ends a list;
+  int sched_pitch;                // null: one layer whose implicit_tiles tiles the clusters take round robin
+  int implicit_tiles;
+  unsigned long long* ready;      // per 256-row block: completed stores of the first layer (only grows); null for one layer
   unsigned long long ready_target;   // the value a block's counter reaches in this launch
   uint32_t* status;
   alignas(64) CUtensorMap tm[6];  // A, Wt, D of the first layer, then of the second

@@ -1,5 +1,6 @@
-// tcgen05 GEMM on CTA pairs (cta_group::2) with the same fused epilogue as kernels_gemm_tc.cu, for large
-// problems:  D[M,N] = A[M,K] * Wt[N,K]^T  ->  post-ops  ->  store.
+// tcgen05 GEMM on CTA pairs (cta_group::2) with the fused epilogue of kernels_gemm_tc.cu, for large problems:
+//   D[M,N] = A[M,K] * Wt[N,K]^T  ->  post-ops  ->  store,
+// for one layer or for two consecutive layers in ONE persistent launch.
 //
 // A cluster of two CTAs (two SMs) owns a 256 x 256 output tile.  Each CTA loads its own 128 rows of A and its
 // own 128 of the tile's 256 Wt rows per k-block (32 KB instead of the 48 KB a lone CTA needs for a 128 x 256
@@ -14,45 +15,69 @@
 //   tempty[a]  in the leader; the epilogue warps of both CTAs arrive on it (peer: remote arrive)
 // Cluster-wide barriers bracket the kernel so that neither CTA touches the other's barriers before they are
 // initialised nor retires while its peer can still read its shared memory.
+//
+// Two layers in one launch (the bf16 FFN: matmul + bias + GELU, matmul + bias) are the analogue of the paper's
+// coarse-grain fusion for the large-batch case (Section V: consecutive fused ops merged so that the intermediate
+// stays in cache and the per-op synchronisation disappears).  What one launch buys over two:
+//   * no second ramp (set-up, first loads) and no tail in between (the last tiles' epilogues of the first matmul
+//     overlap the first main loops of the second);
+//   * a tile schedule over BOTH matmuls, built by the host: each cluster walks its own list of tiles;
+//   * the hidden tensor is read back soon after it was written, while it is still in L2.
+// Dependency: a tile of the second matmul reads 256 rows of the hidden tensor, which the n_tiles tiles of that
+// row block of the first matmul write (TMA stores of 2 CTAs x 8 epilogue warps each).  Every epilogue warp, once its
+// stores of a first-matmul tile have COMPLETED, adds one to the row block's counter in global memory (releasing);
+// the producer thread of a second-matmul tile polls the counter (acquiring, bounded) before it issues the loads of
+// its A operand.  The counters only grow; the host passes the value they reach in this launch.  The schedule puts
+// every first-matmul tile before every second-matmul tile in each cluster's list and all clusters are resident
+// (one CTA per SM), so the waits cannot deadlock.  Without a schedule (one layer) the clusters take the tiles
+// round robin.
+#include <type_traits>
+
 #include "gemm_epilogue.cuh"
 
 namespace gc {
 
-constexpr int G2_BLOCK_M = 128;          // rows per CTA (256 per pair)
-constexpr int G2_BLOCK_N = 256;
-constexpr int G2_B_ROWS = 128;           // Wt rows each CTA loads
-constexpr int G2_STAGES = 5;
-constexpr int G2_STAGE_BYTES = (G2_BLOCK_M + G2_B_ROWS) * 128;
-constexpr int G2_EPI_WARPS = 8;
-constexpr int G2_THREADS = 64 + 32 * G2_EPI_WARPS;
-constexpr int G2_STAGING_BYTES = G2_EPI_WARPS * 4096;       // one [32 rows x 128 B] box per epilogue warp
-constexpr int G2_BIAS_BYTES = G2_EPI_WARPS * G2_BLOCK_N * 4;  // per epilogue warp: the tile's 256 bias values
-constexpr int G2_TMEM_COLS = 512;
+namespace {
 
-size_t gemm_tc2_smem_bytes() {
-  return static_cast<size_t>(G2_STAGES) * G2_STAGE_BYTES + G2_STAGING_BYTES + G2_BIAS_BYTES + 1024 + 256;
+constexpr int F2_BLOCK_M = 128;          // rows per CTA (256 per pair)
+constexpr int F2_BLOCK_N = 256;
+constexpr int F2_B_ROWS = 128;           // Wt rows each CTA loads
+constexpr int F2_STAGES = 5;
+constexpr int F2_STAGE_BYTES = (F2_BLOCK_M + F2_B_ROWS) * 128;
+constexpr int F2_EPI_WARPS = 8;
+constexpr int F2_THREADS = 64 + 32 * F2_EPI_WARPS;
+constexpr int F2_STAGING_BYTES = F2_EPI_WARPS * 4096;
+constexpr int F2_BIAS_BYTES = F2_EPI_WARPS * F2_BLOCK_N * 4;
+constexpr int F2_TMEM_COLS = 512;
+
+size_t fused_smem_bytes() {
+  return static_cast<size_t>(F2_STAGES) * F2_STAGE_BYTES + F2_STAGING_BYTES + F2_BIAS_BYTES + 1024 + 256;
+}
+
+__device__ __forceinline__ unsigned long long f2_ld_acquire(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
 }
 
 template <int KIND, int OUT>
-__global__ void __launch_bounds__(G2_THREADS, 1)
-gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                const __grid_constant__ CUtensorMap tmD, const GemmTcParams p) {
-  constexpr int A_BYTES = G2_BLOCK_M * 128;
+__global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_constant__ GemmPairParams p) {
+  constexpr int A_BYTES = F2_BLOCK_M * 128;
   constexpr int K_ELEMS = KIND == KIND_I8 ? 128 : (KIND == KIND_BF16 ? 64 : 32);
   constexpr int OUT_BYTES = out_bytes(OUT);
   constexpr int BOX_COLS = 128 / OUT_BYTES;
-  constexpr int NUM_BOXES = G2_BLOCK_N / BOX_COLS;
+  constexpr int NUM_BOXES = F2_BLOCK_N / BOX_COLS;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* staging = smem + G2_STAGES * G2_STAGE_BYTES;
-  float* bias_smem = reinterpret_cast<float*>(staging + G2_STAGING_BYTES);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(staging + G2_STAGING_BYTES + G2_BIAS_BYTES);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * G2_STAGES + 4);
+  uint8_t* staging = smem + F2_STAGES * F2_STAGE_BYTES;
+  float* bias_smem = reinterpret_cast<float*>(staging + F2_STAGING_BYTES);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(staging + F2_STAGING_BYTES + F2_BIAS_BYTES);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * F2_STAGES + 4);
   const uint32_t smem_base = smem_u32(smem);
   const uint32_t bar_full = smem_u32(bars);                       // [STAGES]  (used in the leader)
-  const uint32_t bar_empty = bar_full + 8 * G2_STAGES;            // [STAGES]
-  const uint32_t bar_tfull = bar_empty + 8 * G2_STAGES;           // [2]
+  const uint32_t bar_empty = bar_full + 8 * F2_STAGES;            // [STAGES]
+  const uint32_t bar_tfull = bar_empty + 8 * F2_STAGES;           // [2]
   const uint32_t bar_tempty = bar_tfull + 16;                     // [2]       (used in the leader)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -60,21 +85,19 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   const bool leader = rank == 0;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < G2_STAGES; ++s) {
+    for (int s = 0; s < F2_STAGES; ++s) {
       mbar_init(bar_full + 8 * s, 1);
       mbar_init(bar_empty + 8 * s, 1);
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_tfull + 8 * a, 1);
-      mbar_init(bar_tempty + 8 * a, 2 * G2_EPI_WARPS);
+      mbar_init(bar_tempty + 8 * a, 2 * F2_EPI_WARPS);
     }
     fence_mbar_init();
-    tma_prefetch_desc(&tmA);
-    tma_prefetch_desc(&tmB);
-    tma_prefetch_desc(&tmD);
+    for (int i = 0; i < 6; ++i) tma_prefetch_desc(&p.tm[i]);
   }
   if (warp == 1) {
-    tmem_alloc2(smem_u32(tmem_slot), G2_TMEM_COLS);
+    tmem_alloc2(smem_u32(tmem_slot), F2_TMEM_COLS);
     tmem_relinquish2();
   }
   tc_fence_before();
@@ -85,10 +108,16 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
-  // pair tiles: m_pairs x n_tiles; this CTA handles 128-row block 2 * m_pair + rank
-  const int m_pairs = (p.m_tiles + 1) / 2;
-  const int num_tiles = m_pairs * p.n_tiles;
+  // this cluster's tile list: entries (layer << 24) | tile, terminated by a negative entry; without a list the
+  // clusters take the tiles of the (single) layer round robin
   const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
+  const int* sched = p.sched ? p.sched + static_cast<int64_t>(cluster_id) * p.sched_pitch : nullptr;
+  const int list_len = p.sched ? p.sched_pitch : (p.implicit_tiles + num_clusters - 1) / num_clusters;
+  auto entry = [&](int i) -> int {
+    if (sched) return __ldg(sched + i);
+    const int t = cluster_id + i * num_clusters;
+    return t < p.implicit_tiles ? t : -1;
+  };
   bool failed = false;
 
   if (warp == 0) {
@@ -97,20 +126,41 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       int stage = 0;
       uint32_t phase = 0;
       const uint32_t leader_full = leader ? bar_full : mapa_shared(bar_full, 0);
-      for (int tile = cluster_id; tile < num_tiles && !failed; tile += num_clusters) {
-        const int m_blk = (tile / p.n_tiles) * 2 + static_cast<int>(rank), n_blk = tile % p.n_tiles;
-        for (int kb = 0; kb < p.num_k_blocks; ++kb) {
+      for (int i = 0; i < list_len && !failed; ++i) {
+        const int e = entry(i);
+        if (e < 0) break;
+        const int l = e >> 24, tile = e & 0xFFFFFF;
+        const int n_tiles = p.L[l].n_tiles, nkb = p.L[l].num_k_blocks;
+        const int m_pair = tile / n_tiles, n_blk = tile % n_tiles;
+        const int m_blk = m_pair * 2 + static_cast<int>(rank);
+        if (l == 1) {
+          // the 256 hidden rows this tile reads: wait until every store of that row block has completed
+          const uint64_t t0 = globaltimer_ns();
+          uint32_t spins = 0;
+          while (f2_ld_acquire(p.ready + m_pair) < p.ready_target) {
+            if ((++spins & 255u) == 0 && globaltimer_ns() - t0 > 2000000000ull) {
+              report(p.status, DEV_TIMEOUT_PRODUCER);
+              failed = true;
+              break;
+            }
+          }
+          if (failed) break;
+          asm volatile("fence.proxy.async.global;" ::: "memory");   // acquire (generic) before the TMA loads (async proxy)
+        }
+        const CUtensorMap* tmA = &p.tm[3 * l];
+        const CUtensorMap* tmB = &p.tm[3 * l + 1];
+        for (int kb = 0; kb < nkb; ++kb) {
           if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1)) {
             report(p.status, DEV_TIMEOUT_PRODUCER);
             failed = true;
             break;
           }
-          const uint32_t sA = smem_base + stage * G2_STAGE_BYTES, sB = sA + A_BYTES;
-          if (leader) mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * G2_STAGE_BYTES);   // both CTAs' bytes
-          tma_load_2d_pair(sA, &tmA, kb * K_ELEMS, m_blk * G2_BLOCK_M, leader_full + 8 * stage);
-          tma_load_2d_pair(sB, &tmB, kb * K_ELEMS, n_blk * G2_BLOCK_N + static_cast<int>(rank) * G2_B_ROWS,
+          const uint32_t sA = smem_base + stage * F2_STAGE_BYTES, sB = sA + A_BYTES;
+          if (leader) mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * F2_STAGE_BYTES);   // both CTAs' bytes
+          tma_load_2d_pair(sA, tmA, kb * K_ELEMS, m_blk * F2_BLOCK_M, leader_full + 8 * stage);
+          tma_load_2d_pair(sB, tmB, kb * K_ELEMS, n_blk * F2_BLOCK_N + static_cast<int>(rank) * F2_B_ROWS,
                            leader_full + 8 * stage);
-          if (++stage == G2_STAGES) {
+          if (++stage == F2_STAGES) {
             stage = 0;
             phase ^= 1;
           }
@@ -122,29 +172,34 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     if (leader && lane == 0) {
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
-      for (int tile = cluster_id; tile < num_tiles && !failed; tile += num_clusters) {
+      for (int i = 0; i < list_len && !failed; ++i) {
+        const int e = entry(i);
+        if (e < 0) break;
+        const int l = e >> 24;
+        const int nkb = p.L[l].num_k_blocks;
+        const uint32_t idesc = p.L[l].idesc;
         if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1)) {
           report(p.status, DEV_TIMEOUT_MMA);
           failed = true;
           break;
         }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * G2_BLOCK_N;
-        for (int kb = 0; kb < p.num_k_blocks; ++kb) {
+        const uint32_t d_tmem = tmem_base + acc * F2_BLOCK_N;
+        for (int kb = 0; kb < nkb; ++kb) {
           if (!mbar_wait(bar_full + 8 * stage, phase)) {
             report(p.status, DEV_TIMEOUT_MMA);
             failed = true;
             break;
           }
           tc_fence_after();
-          const uint32_t sA = smem_base + stage * G2_STAGE_BYTES, sB = sA + A_BYTES;
+          const uint32_t sA = smem_base + stage * F2_STAGE_BYTES, sB = sA + A_BYTES;
           const uint64_t a_desc = make_smem_desc(sA, 16, 1024, SWZ_128B);
           const uint64_t b_desc = make_smem_desc(sB, 16, 1024, SWZ_128B);
 #pragma unroll
           for (int k = 0; k < 4; ++k)
-            umma_ss2<KIND>(d_tmem, a_desc + 2 * k, b_desc + 2 * k, p.idesc, (kb | k) != 0 ? 1u : 0u);
+            umma_ss2<KIND>(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
           umma_commit2(bar_empty + 8 * stage, 3);                // frees the stage in both CTAs
-          if (++stage == G2_STAGES) {
+          if (++stage == F2_STAGES) {
             stage = 0;
             phase ^= 1;
           }
@@ -164,24 +219,30 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     uint32_t acc_phase = 0;
     uint8_t* my_stage = staging + ew * 4096;
     const uint32_t my_stage_u32 = smem_u32(my_stage);
-    float* my_bias = bias_smem + ew * G2_BLOCK_N;
+    float* my_bias = bias_smem + ew * F2_BLOCK_N;
     const uint32_t row_off = (lane >> 3) * 1024 + (lane & 7) * 128;
     const uint32_t leader_tempty = leader ? bar_tempty : mapa_shared(bar_tempty, 0);
-    for (int tile = cluster_id; tile < num_tiles; tile += num_clusters) {
-      const int m_blk = (tile / p.n_tiles) * 2 + static_cast<int>(rank), n_blk = tile % p.n_tiles;
+    for (int i = 0; i < list_len; ++i) {
+      const int e = entry(i);
+      if (e < 0) break;
+      const int l = e >> 24, tile = e & 0xFFFFFF;
+      const int n_tiles = p.L[l].n_tiles, N = p.L[l].N;
+      const int m_pair = tile / n_tiles, n_blk = tile % n_tiles;
+      const int m_blk = m_pair * 2 + static_cast<int>(rank);
+      const CUtensorMap* tmD = &p.tm[3 * l + 2];
       // Copy this tile's bias slice into shared memory while the accumulator is still being produced: a
       // global load in the per-chunk loop would put its full latency on the critical path of every chunk.
-      Epilogue epi = p.epi;
-      if (p.epi.bias) {
+      Epilogue epi = p.L[l].epi;
+      if (epi.bias) {
         __syncwarp();
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          const int c = n_blk * G2_BLOCK_N + (lane + 32 * i) * 4;
-          const float4 v = c < p.N ? __ldg(reinterpret_cast<const float4*>(p.epi.bias + c)) : make_float4(0.f, 0.f, 0.f, 0.f);
-          reinterpret_cast<float4*>(my_bias)[lane + 32 * i] = v;
+        for (int j = 0; j < 2; ++j) {
+          const int c = n_blk * F2_BLOCK_N + (lane + 32 * j) * 4;
+          const float4 v = c < N ? __ldg(reinterpret_cast<const float4*>(epi.bias + c)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          reinterpret_cast<float4*>(my_bias)[lane + 32 * j] = v;
         }
         __syncwarp();
-        epi.bias = my_bias - n_blk * G2_BLOCK_N;                   // indexed by absolute column below
+        epi.bias = my_bias - n_blk * F2_BLOCK_N;                   // indexed by absolute column below
       }
       if (!mbar_wait(bar_tfull + 8 * acc, acc_phase)) {
         report(p.status, DEV_TIMEOUT_EPILOGUE);
@@ -189,7 +250,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         break;
       }
       tc_fence_after();
-      const uint32_t t_row = tmem_base + acc * G2_BLOCK_N + (static_cast<uint32_t>(q * 32) << 16);
+      const uint32_t t_row = tmem_base + acc * F2_BLOCK_N + (static_cast<uint32_t>(q * 32) << 16);
       for (int box = half; box < NUM_BOXES; box += 2) {
         // the previous store out of this warp's staging buffer must have read it completely
         if (lane == 0) tma_store_wait_read<0>();
@@ -201,17 +262,17 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           tmem_wait_ld();
           constexpr int NW = 32 * OUT_BYTES / 4;
           uint32_t w[NW];
-          epi_chunk32<KIND, OUT>(r, w, n_blk * G2_BLOCK_N + box * BOX_COLS + sub * 32, p.N, epi);
+          epi_chunk32<KIND, OUT>(r, w, n_blk * F2_BLOCK_N + box * BOX_COLS + sub * 32, N, epi);
           const int c0 = sub * (NW / 4);
 #pragma unroll
-          for (int i = 0; i < NW / 4; ++i)
-            *reinterpret_cast<uint4*>(my_stage + row_off + (((c0 + i) ^ (lane & 7)) * 16)) =
-                make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+          for (int j = 0; j < NW / 4; ++j)
+            *reinterpret_cast<uint4*>(my_stage + row_off + (((c0 + j) ^ (lane & 7)) * 16)) =
+                make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
         }
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
-          tma_store_2d(&tmD, n_blk * G2_BLOCK_N + box * BOX_COLS, m_blk * G2_BLOCK_M + q * 32, my_stage_u32);
+          tma_store_2d(tmD, n_blk * F2_BLOCK_N + box * BOX_COLS, m_blk * F2_BLOCK_M + q * 32, my_stage_u32);
           tma_store_commit();
         }
       }
@@ -220,6 +281,12 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       if (lane == 0) {
         if (leader) mbar_arrive(bar_tempty + 8 * acc);
         else mbar_arrive_cluster(leader_tempty + 8 * acc);
+        if (l == 0 && p.ready) {
+          // my part of the hidden row block is in memory once my stores have completed (not merely been read)
+          tma_store_wait_all<0>();
+          asm volatile("fence.proxy.async.global;" ::: "memory");
+          asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p.ready + m_pair), "l"(1ULL) : "memory");
+        }
       }
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1;
@@ -232,7 +299,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   cluster_sync_all();                                             // the peer no longer reads this CTA's smem
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc2(tmem_base, G2_TMEM_COLS);
+    tmem_dealloc2(tmem_base, F2_TMEM_COLS);
   }
   if (failed) {
     const uint64_t t0 = globaltimer_ns();
@@ -242,21 +309,14 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 }
 
 template <int KIND, int OUT>
-static cudaError_t launch_one2(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmD,
-                               const GemmTcParams& p, int grid, bool pdl, cudaStream_t s) {
-  const size_t smem = gemm_tc2_smem_bytes();
+cudaError_t launch_fused_t(const GemmPairParams& p, int grid, bool pdl, cudaStream_t s) {
+  const size_t smem = fused_smem_bytes();
   auto kern = gemm_tc2_kernel<KIND, OUT>;
-  static bool attr_set[64] = {};
-  int dev = 0;
-  cudaGetDevice(&dev);
-  if (!attr_set[dev & 63]) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
-    attr_set[dev & 63] = true;
-  }
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
-  cfg.blockDim = dim3(G2_THREADS);
+  cfg.blockDim = dim3(F2_THREADS);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
   cudaLaunchAttribute attr[2];
@@ -268,43 +328,66 @@ static cudaError_t launch_one2(const CUtensorMap& tmA, const CUtensorMap& tmB, c
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 2 : 1;
-  return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmD, p);
+  return cudaLaunchKernelEx(&cfg, kern, p);
 }
 
-template <int KIND>
-static cudaError_t launch_out2(int out, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmD,
-                               const GemmTcParams& p, int grid, bool pdl, cudaStream_t s) {
-  switch (out) {
-    case OUT_F32: return launch_one2<KIND, OUT_F32>(tmA, tmB, tmD, p, grid, pdl, s);
-    case OUT_BF16: return launch_one2<KIND, OUT_BF16>(tmA, tmB, tmD, p, grid, pdl, s);
-    case OUT_Q8: return launch_one2<KIND, OUT_Q8>(tmA, tmB, tmD, p, grid, pdl, s);
-    case OUT_RAW32:
-      if constexpr (KIND == KIND_I8) return launch_one2<KIND, OUT_RAW32>(tmA, tmB, tmD, p, grid, pdl, s);
-      return launch_one2<KIND, OUT_F32>(tmA, tmB, tmD, p, grid, pdl, s);
-    default: return cudaErrorInvalidValue;
+}  // namespace
+
+size_t gemm_tc2_smem_bytes() { return fused_smem_bytes(); }
+
+// kind: 0 = i8, 1 = bf16, 2 = tf32; both layers share the MMA kind and the output element type.
+cudaError_t launch_gemm_tc2_fused(int kind, int a_signed, const GemmPairParams& p_in, int grid, cudaStream_t s) {
+  GemmPairParams p = p_in;
+  const int out_dtype = p.L[0].epi.out_dtype;
+  for (int l = 0; l < 2; ++l) {
+    p.L[l].idesc = kind == KIND_I8     ? make_idesc(ACC_S32, (l == 0 ? a_signed : (out_dtype == GC_S8)) ? FMT_S8 : FMT_U8, FMT_S8, 256, F2_BLOCK_N)
+                   : kind == KIND_BF16 ? make_idesc(ACC_F32, FMT_BF16, FMT_BF16, 256, F2_BLOCK_N)
+                                       : make_idesc(ACC_F32, FMT_TF32, FMT_TF32, 256, F2_BLOCK_N);
   }
+  if (kind == KIND_BF16 && out_dtype == GC_BF16) return launch_fused_t<KIND_BF16, OUT_BF16>(p, grid, true, s);
+  if (kind == KIND_I8 && (out_dtype == GC_U8 || out_dtype == GC_S8)) return launch_fused_t<KIND_I8, OUT_Q8>(p, grid, true, s);
+  if (kind == KIND_TF32 && out_dtype == GC_F32) return launch_fused_t<KIND_TF32, OUT_F32>(p, grid, true, s);
+  return cudaErrorInvalidValue;
 }
 
+// One layer: the clusters take its tiles round robin (no schedule table, no counters).
 cudaError_t launch_gemm_tc2(int kind, int a_signed, const CUtensorMap& tmA, const CUtensorMap& tmB,
-                            const CUtensorMap& tmD, const GemmTcParams& p_in, int grid, bool pdl, cudaStream_t s) {
-  GemmTcParams p = p_in;
-  const Epilogue& e = p.epi;
+                            const CUtensorMap& tmD, const GemmTcParams& g, int grid, bool pdl, cudaStream_t s) {
+  GemmPairParams p = {};
+  p.L[0].N = g.N;
+  p.L[0].num_k_blocks = g.num_k_blocks;
+  p.L[0].n_tiles = g.n_tiles;
+  p.L[0].epi = g.epi;
+  p.implicit_tiles = ((g.m_tiles + 1) / 2) * g.n_tiles;
+  p.status = g.status;
+  p.tm[0] = tmA;
+  p.tm[1] = tmB;
+  p.tm[2] = tmD;
+  p.tm[3] = tmA;                                                  // unused; valid descriptors for the prefetch
+  p.tm[4] = tmB;
+  p.tm[5] = tmD;
+  p.L[0].idesc = kind == KIND_I8     ? make_idesc(ACC_S32, a_signed ? FMT_S8 : FMT_U8, FMT_S8, 256, F2_BLOCK_N)
+                 : kind == KIND_BF16 ? make_idesc(ACC_F32, FMT_BF16, FMT_BF16, 256, F2_BLOCK_N)
+                                     : make_idesc(ACC_F32, FMT_TF32, FMT_TF32, 256, F2_BLOCK_N);
+  const Epilogue& e = g.epi;
   const int out = (e.acc_is_int && !e.has_dq) ? OUT_RAW32
                   : e.out_dtype == GC_F32    ? OUT_F32
                   : e.out_dtype == GC_BF16   ? OUT_BF16
                                              : OUT_Q8;
-  if (kind == KIND_I8) {
-    p.idesc = make_idesc(ACC_S32, a_signed ? FMT_S8 : FMT_U8, FMT_S8, 256, G2_BLOCK_N);
-    return launch_out2<KIND_I8>(out, tmA, tmB, tmD, p, grid, pdl, s);
-  }
-  if (kind == KIND_BF16) {
-    p.idesc = make_idesc(ACC_F32, FMT_BF16, FMT_BF16, 256, G2_BLOCK_N);
-    return launch_out2<KIND_BF16>(out, tmA, tmB, tmD, p, grid, pdl, s);
-  }
-  if (kind == KIND_TF32) {
-    p.idesc = make_idesc(ACC_F32, FMT_TF32, FMT_TF32, 256, G2_BLOCK_N);
-    return launch_out2<KIND_TF32>(out, tmA, tmB, tmD, p, grid, pdl, s);
-  }
+  auto dispatch = [&](auto kind_tag) -> cudaError_t {
+    constexpr int K = decltype(kind_tag)::value;
+    switch (out) {
+      case OUT_F32: return launch_fused_t<K, OUT_F32>(p, grid, pdl, s);
+      case OUT_BF16: return launch_fused_t<K, OUT_BF16>(p, grid, pdl, s);
+      case OUT_Q8: return launch_fused_t<K, OUT_Q8>(p, grid, pdl, s);
+      default:
+        if constexpr (K == KIND_I8) return launch_fused_t<K, OUT_RAW32>(p, grid, pdl, s);
+        return launch_fused_t<K, OUT_F32>(p, grid, pdl, s);
+    }
+  };
+  if (kind == KIND_I8) return dispatch(std::integral_constant<int, KIND_I8>());
+  if (kind == KIND_BF16) return dispatch(std::integral_constant<int, KIND_BF16>());
+  if (kind == KIND_TF32) return dispatch(std::integral_constant<int, KIND_TF32>());
   return cudaErrorInvalidValue;
 }
 
