@@ -50,7 +50,10 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
 
 // Grid-wide barrier: every CTA adds one to a counter that only grows; the caller passes the value the
 // counter reaches when all CTAs of this launch have arrived at this barrier.  Bounded: gives up after 2 s.
-__device__ __forceinline__ bool grid_barrier(unsigned long long* ctr, unsigned long long target) {
+// `on_release` runs in thread 0 as soon as the barrier opens, before the CTA's other threads are released: the
+// place to issue the loads that only waited for the other CTAs' stores.
+template <typename F>
+__device__ __forceinline__ bool grid_barrier(unsigned long long* ctr, unsigned long long target, F on_release) {
   __syncthreads();
   int ok = 1;
   if (threadIdx.x == 0) {
@@ -67,6 +70,7 @@ __device__ __forceinline__ bool grid_barrier(unsigned long long* ctr, unsigned l
       }
     }
     asm volatile("fence.proxy.async.global;" ::: "memory");
+    if (ok) on_release();
   }
   return __syncthreads_and(ok) != 0;
 }
@@ -196,17 +200,37 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
 
   bool failed = false;
   unsigned long long bar_count = p.barrier_base;                  // counter value before this launch
-  auto next_barrier = [&]() {
+  int stage = 0;                 // ring position, shared by construction between producer and MMA thread
+  uint32_t phase = 0;
+  uint32_t tphase = 0;           // parity of the accumulator-ready barrier (one completion per active layer)
+  bool a_issued = false;         // thread 0: the A loads of the coming layer went out from inside the barrier
+
+  // Thread 0 (the TMA producer) issues my k-blocks of layer l's A operand.  a_stages >= my k-blocks (planner): a
+  // stage is never reused within a layer, and between layers the accumulator-ready commit plus the grid barrier
+  // guarantee that every MMA has read its stage.
+  auto issue_a_loads = [&](int l) {
+    const ChainLayer& L = p.L[l];
+    if (L.active_ctas == 0 || cta >= L.active_ctas || (l == 0 && p.pack_rows > 0)) return;
+    const int lo = kb_lo(L), hi = kb_hi(L);
+    for (int kb = lo; kb < hi; ++kb) {
+      mbar_arrive_expect_tx(bar_full + 8 * stage, CH_A_STAGE_BYTES);
+      tma_load_2d(smem_u32(sA) + stage * CH_A_STAGE_BYTES, p.tmaps + L.a_tm, kb * K_ELEMS, 0, bar_full + 8 * stage);
+      if (++stage == CH_STAGES) {
+        stage = 0;
+        phase ^= 1;
+      }
+    }
+    a_issued = true;
+  };
+  // Grid barrier before layer l_next: its A operand is what the other CTAs have just stored, so thread 0 sends the
+  // loads the moment the barrier opens (its proxy fence after the acquire orders those stores before the loads).
+  auto next_barrier = [&](int l_next) {
     bar_count += gridDim.x;
-    if (!grid_barrier(p.barrier, bar_count)) {
+    if (!grid_barrier(p.barrier, bar_count, [&]() { issue_a_loads(l_next); })) {
       failed = true;
       report(p.status, DEV_TIMEOUT_OTHER);
     }
   };
-
-  int stage = 0;                 // ring position, shared by construction between producer and MMA thread
-  uint32_t phase = 0;
-  uint32_t tphase = 0;           // parity of the accumulator-ready barrier (one completion per active layer)
   const int rows_per = 128 / KS; // rows of the tile this CTA finishes
   for (int l = 0; l < p.n_layers && !failed; ++l) {
     // A by-value copy: fields read through a reference into the parameter space are re-fetched around every
@@ -218,19 +242,9 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
         // first layer fed by plain loads (graph-entry reorder): its blocks use stages 0 .. my_nkb-1 outside the ring
         const bool manual_a = l == 0 && p.pack_rows > 0;
         if (warp == 0) {
-          if (lane == 0 && !manual_a) {
-            // (this thread is the one that ran the grid barrier: its proxy fence after the acquire already ordered
-            // the other CTAs' generic stores before the TMA loads below)
-            // a_stages >= my_nkb (planner): a stage is never reused within a layer, and between layers the
-            // accumulator-ready commit plus the grid barrier guarantee that every MMA has read its stage
-            for (int kb = lo; kb < lo + my_nkb; ++kb) {
-              mbar_arrive_expect_tx(bar_full + 8 * stage, CH_A_STAGE_BYTES);
-              tma_load_2d(smem_u32(sA) + stage * CH_A_STAGE_BYTES, p.tmaps + L.a_tm, kb * K_ELEMS, 0, bar_full + 8 * stage);
-              if (++stage == CH_STAGES) {
-                stage = 0;
-                phase ^= 1;
-              }
-            }
+          if (lane == 0) {
+            if (!a_issued) issue_a_loads(l);                     // first layer: no barrier preceded it
+            a_issued = false;
           }
         } else if (warp == 1) {
           if (lane == 0) {
@@ -432,7 +446,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
         }
       }
     }
-    if (l + 1 < p.n_layers) next_barrier();
+    if (l + 1 < p.n_layers) next_barrier(l + 1);
   }
 
   tc_fence_before();
