@@ -168,9 +168,23 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  // Programmatic dependent launch: the set-up above may overlap the tail of the preceding kernel on the stream;
-  // nothing below touches global memory before that kernel has completed (no-op for an ordinary launch).
+  // Programmatic dependent launch: the set-up above may overlap the tail of the preceding kernel on the stream.
+  // While waiting for it, the first units' operands are pulled into L2 (a prefetch has no destination the kernel
+  // could read too early, and L2 stays coherent with whatever the preceding kernel still writes); nothing else
+  // touches global memory before that kernel has completed (the wait is a no-op for an ordinary launch).
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (tid == 0) {
+    const int q_tiles0 = S / SDPA_BLOCK_Q;
+    int unit = blockIdx.x;
+    for (int n0 = 0; n0 < slots && unit < p.B * p.H * q_tiles0; ++n0, unit += gridDim.x) {
+      const int bh = unit / q_tiles0, qt = unit % q_tiles0;
+      tma_prefetch_2d(&tmQ, 0, bh * S + qt * SDPA_BLOCK_Q);
+      for (int j = 0; j < NB; ++j) {
+        tma_prefetch_2d(&tmK, 0, bh * S + j * 128);
+        tma_prefetch_2d(&tmV, 0, bh * S + j * 128);
+      }
+    }
+  }
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
   bool failed = false;

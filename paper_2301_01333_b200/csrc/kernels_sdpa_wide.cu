@@ -173,9 +173,21 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  // Programmatic dependent launch: the set-up above may overlap the tail of the preceding kernel on the stream;
-  // nothing below touches global memory before that kernel has completed (no-op for an ordinary launch).
+  // Programmatic dependent launch: the set-up above may overlap the tail of the preceding kernel on the stream.
+  // While waiting for it, the first unit's operands are pulled into L2 (a prefetch has no destination the kernel
+  // could read too early, and L2 stays coherent with whatever the preceding kernel still writes); nothing else
+  // touches global memory before that kernel has completed (the wait is a no-op for an ordinary launch).
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (threadIdx.x == 0 && static_cast<int>(blockIdx.x) < p.B * p.H * (S / W_BLOCK_Q)) {
+    const int unit = blockIdx.x, qt0 = S / W_BLOCK_Q;
+    const int row0 = (unit / qt0) * S;
+    for (int j = 0; j < L::NSUB; ++j) tma_prefetch_2d(&tmQ, j * L::SUB_ELEMS, row0 + (unit % qt0) * W_BLOCK_Q);
+    for (int b = 0; b < NB; ++b)
+      for (int j = 0; j < L::NSUB; ++j) {
+        tma_prefetch_2d(&tmK, j * L::SUB_ELEMS, row0 + b * 128);
+        tma_prefetch_2d(&tmV, j * L::SUB_ELEMS, row0 + b * 128);
+      }
+  }
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
   bool failed = false;
