@@ -303,6 +303,63 @@ def test_mha_int8_streaming_kernel_stages_around_the_softmax(B):
     assert_stage_after_softmax_exact(w, o_gpu, p_gpu)
 
 
+def _attention_variant(kind, b, h, s, d, mask, mul, q_signed, seed=1):
+    """An attention partition with optional pieces left out (no mask, no scaling) or s8 queries."""
+    from paper_2301_01333_b200.graph import Graph
+    from paper_2301_01333_b200.workloads import Workload, _mask_from_valid, f32_to_bf16_bits
+    rng = np.random.default_rng(seed)
+    g = Graph(name="attention_variant")
+    feeds = {}
+    shp, ss = (b, h, s, d), (b, h, s, s)
+    if kind == "bf16":
+        q, k, v = (g.input("bf16", shp) for _ in range(3))
+        for t in (q, k, v):
+            feeds[t] = f32_to_bf16_bits(rng.standard_normal(shp, dtype=np.float32))
+        x = g.op("matmul", (q, k), g.tensor("f32", ss), transpose_b=True)
+    else:
+        q = g.input("s8" if q_signed else "u8", shp, scale=0.03, zero_point=0 if q_signed else 128)
+        k = g.input("u8", shp, scale=0.03, zero_point=128)
+        v = g.input("u8", shp, scale=0.03, zero_point=128)
+        feeds[q] = rng.integers(-128, 128, size=shp).astype(np.int8) if q_signed else rng.integers(0, 256, size=shp).astype(np.uint8)
+        feeds[k] = rng.integers(0, 256, size=shp).astype(np.uint8)
+        feeds[v] = rng.integers(0, 256, size=shp).astype(np.uint8)
+        a = g.op("matmul", (q, k), g.tensor("s32", ss), transpose_b=True)
+        x = g.op("dequantize", (a,), g.tensor("f32", ss))
+    if mul:
+        x = g.op("mul", (x,), g.tensor("f32", ss), scalar=float(1 / np.sqrt(d)))
+    if mask:
+        m = g.input("f32", (b, 1, 1, s))
+        feeds[m] = _mask_from_valid(rng.integers(s // 2, s + 1, size=(b,)), s)
+        x = g.op("add", (x, m), g.tensor("f32", ss))
+    p = g.op("softmax", (x,), g.tensor("f32", ss), axis=-1)
+    if kind == "bf16":
+        pb = g.op("typecast", (p,), g.tensor("bf16", ss))
+        o = g.op("matmul", (pb, v), g.tensor("f32", shp))
+        o = g.op("typecast", (o,), g.tensor("bf16", shp))
+    else:
+        pq = g.op("quantize", (p,), g.tensor("u8", ss, scale=float(np.float32(1 / 255)), zero_point=0))
+        a2 = g.op("matmul", (pq, v), g.tensor("s32", shp))
+        o = g.op("dequantize", (a2,), g.tensor("f32", shp))
+        o = g.op("quantize", (o,), g.tensor("u8", shp, scale=0.02, zero_point=128))
+    g.mark_output(o)
+    return Workload(g.name, g, feeds).finish()
+
+
+@pytest.mark.parametrize("kind,s,d,mask,mul,q_signed", [
+    ("bf16", 128, 64, False, True, False), ("bf16", 256, 128, True, False, False), ("bf16", 512, 64, False, False, False),
+    ("int8", 384, 64, False, False, True), ("int8", 512, 64, True, True, True), ("int8", 128, 96, False, True, False),
+    ("int8", 256, 128, True, False, True)])
+def test_attention_graph_variants(B, kind, s, d, mask, mul, q_signed):
+    # the optional ops of the pattern left out (no mask, no scaling) and signed queries, on both tcgen05 kernels
+    w = _attention_variant(kind, 2, 3, s, d, mask, mul, q_signed)
+    got, plan = run_gpu(B, w)
+    assert "tcgen05" in plan
+    if kind == "bf16":
+        assert np.abs(bf16_to_f64(got) - oracle(w)).max() <= 2e-2
+    else:
+        check_int8_attention(got, oracle(w))
+
+
 def test_mha_bf16_generic_kernel(B):
     w = W.mha_bf16(batch=2, heads=2, seq=128, head_dim=64)
     got, plan = run_gpu(B, w, force_generic=True)
