@@ -207,6 +207,81 @@ def test_two_large_layers_in_one_launch_int8_bit_exact(B):
     assert np.array_equal(got, oracle(w))
 
 
+def _mlp_variant(kind, batch, dims, bias=True, act="relu", transposed=False, hidden="u8", per_channel=False, seed=3):
+    """An MLP chain with optional pieces changed: no bias, another activation, weights stored [n, k] (with the
+    per-channel scales on axis 0), s8 hidden activations."""
+    from paper_2301_01333_b200.graph import Graph
+    from paper_2301_01333_b200.workloads import Workload, f32_to_bf16_bits
+    rng = np.random.default_rng(seed)
+    g = Graph(name="mlp_variant")
+    feeds = {}
+    if kind == "int8":
+        x = g.input("u8", (batch, dims[0]), scale=0.02, zero_point=5)
+        feeds[x] = rng.integers(0, 256, size=(batch, dims[0])).astype(np.uint8)
+    elif kind == "bf16":
+        x = g.input("bf16", (batch, dims[0]))
+        feeds[x] = f32_to_bf16_bits(rng.standard_normal((batch, dims[0]), dtype=np.float32))
+    else:
+        x = g.input("f32", (batch, dims[0]))
+        feeds[x] = rng.standard_normal((batch, dims[0]), dtype=np.float32)
+    h = x
+    nl = len(dims) - 1
+    for l in range(nl):
+        k, n = dims[l], dims[l + 1]
+        wshape = (n, k) if transposed else (k, n)
+        if kind == "int8":
+            kw = {}
+            if per_channel:
+                kw = dict(channel_scales=(0.005 * rng.uniform(0.5, 1.5, size=n)).astype(np.float32),
+                          channel_axis=0 if transposed else 1)
+            w = g.input("s8", wshape, scale=0.005, is_constant=True, **kw)
+            feeds[w] = rng.integers(-127, 128, size=wshape).astype(np.int8)
+        else:
+            w = g.input(kind, wshape, is_constant=True)
+            wv = (rng.standard_normal(wshape) * np.sqrt(1.0 / k)).astype(np.float32)
+            feeds[w] = f32_to_bf16_bits(wv) if kind == "bf16" else wv
+        z = g.op("matmul", (h, w), g.tensor("s32" if kind == "int8" else "f32", (batch, n)), transpose_b=transposed)
+        if kind == "int8":
+            z = g.op("dequantize", (z,), g.tensor("f32", (batch, n)))
+        if bias:
+            b = g.input("f32", (n,), is_constant=True)
+            feeds[b] = rng.uniform(-0.1, 0.1, size=(n,)).astype(np.float32)
+            z = g.op("add", (z, b), g.tensor("f32", (batch, n)))
+        if l < nl - 1:
+            z = g.op(act, (z,), g.tensor("f32", (batch, n)))
+            if kind == "int8":
+                h = g.op("quantize", (z,), g.tensor(hidden, (batch, n), scale=0.05, zero_point=3 if hidden == "u8" else 0))
+            elif kind == "bf16":
+                h = g.op("typecast", (z,), g.tensor("bf16", (batch, n)))
+            else:
+                h = z
+        else:
+            h = g.op("typecast", (z,), g.tensor("bf16", (batch, n))) if kind == "bf16" else z
+    g.mark_output(h)
+    return Workload(g.name, g, feeds).finish()
+
+
+@pytest.mark.parametrize("kind,batch,dims,kw", [
+    ("int8", 64, (300, 256, 64, 32), dict(transposed=True, hidden="s8", per_channel=True)),
+    ("int8", 3000, (512, 1024, 1024, 32), dict(transposed=True, per_channel=True)),
+    ("int8", 3000, (512, 1024, 1024, 32), dict(hidden="s8", bias=False)),
+    ("bf16", 96, (256, 512, 128), dict(bias=False, act="gelu_tanh")),
+    ("bf16", 5000, (1024, 1024, 1024), dict(transposed=True, act="gelu_tanh")),
+    ("f32", 32, (100, 256, 64), dict(act="sigmoid")),
+    ("f32", 600, (64, 512, 128), dict(bias=False, transposed=True))])
+@pytest.mark.parametrize("opts", [{}, {"no_chain_fusion": True}])
+def test_mlp_graph_variants(B, kind, batch, dims, kw, opts):
+    w = _mlp_variant(kind, batch, dims, **kw)
+    got, _ = run_gpu(B, w, **opts)
+    ref = oracle(w)
+    if kind == "int8":
+        assert np.array_equal(got, ref)
+    elif kind == "bf16":
+        assert np.abs(bf16_to_f64(got) - ref).max() <= 2e-2
+    else:
+        assert np.abs(got.astype(np.float64) - ref).max() <= 5e-3 * np.abs(ref).max()
+
+
 def test_ffn_bf16_chain_kernel_with_split_reduction(B):
     w = W.ffn_bf16(tokens=96, d_model=512, d_ff=256)
     got, plan = run_gpu(B, w)
