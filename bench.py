@@ -39,6 +39,7 @@ DTYPE = {"c1": "tf32", "c2": "u8xs8->s32", "c3": "bf16", "c4": "u8xu8->s32", "c5
 # c5 runs for about a second so that the clocks settle under the power cap (the regime the "sustained" peak
 # was measured in) and the clock sampler sees the timed region
 DEFAULT_STEPS = {"c1": 2000, "c2": 2000, "c3": 500, "c4": 100, "c5": 8000}
+GRAPH_STEPS = {"c1": 256, "c2": 256, "c3": 256, "c4": 50, "c5": 50}     # executes captured into one CUDA graph
 # DRAM bytes per launch of the dominant kernel from the ncu capture summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum; c5: one launch per step, the 64 MiB hidden tensor is written back)
 TRAFFIC_BYTES_PER_LAUNCH = {"c5": 135.4e6, "c3": None, "c4": 84.8e6}
@@ -233,6 +234,28 @@ def run_sweep(B, device, peaks, only=""):
     return out
 
 
+def run_graph_replay(reps, n_rep, steps, device):
+    """The same rotation of executes captured once into a CUDA graph and replayed (no per-call host work at all):
+    microseconds per subgraph.  gc_execute after its first call only enqueues kernels, so it can be captured."""
+    import torch
+    s = torch.cuda.Stream(device)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=s):
+        for i in range(steps):
+            reps[i % n_rep].c.execute(reps[i % n_rep].ins, reps[i % n_rep].outs, s.cuda_stream)
+    for _ in range(2):
+        g.replay()
+    torch.cuda.synchronize(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(3):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize(device)
+    del g
+    return e0.elapsed_time(e1) * 1e3 / (3 * steps)
+
+
 def run_e2e(w, rep, steps, warmup, device):
     """gc_execute_host with pinned host buffers: H2D of the non-constant inputs, execute, D2H, sync."""
     import torch
@@ -411,6 +434,8 @@ def main():
         # warm: the same buffers every call, so weights and small activations stay in L2
         warm_steps = max(20, steps // 4)
         res["us_per_subgraph_warm"] = max_over_ranks(run_timed(reps[:1], 1, warm_steps, local, barrier)) * 1e3 / warm_steps
+        if not args.only:
+            res["us_per_subgraph_graph"] = run_graph_replay(reps, n_rep, min(steps, GRAPH_STEPS[name]), local)
         if name in ("c1", "c2") and not args.only:
             # coarse-grain fusion ablation (Section VII, Fig. 8): the whole chain in one persistent launch, one
             # launch per layer (fine-grain fusion only), and the CUDA-core kernels

@@ -160,7 +160,11 @@ gc_status_t gc_set_workspace(gc_compiled_t* c, void* workspace_dev, size_t bytes
 /* Execute (Section VII: "the compiled code only needs to be called once" per subgraph).  Enqueues
  * all work on cuda_stream (a cudaStream_t, may be NULL for the default stream) and returns.  On
  * the first call, or when a constant input arrives at a new address, the constant weights are
- * prepacked on the same stream first and cached in the workspace (Section V). */
+ * prepacked on the same stream first and cached in the workspace (Section V).  A call that does
+ * not prepack (same pointers as an earlier call) only enqueues kernel launches with parameters
+ * that do not depend on how often the object has run (the kernels' synchronisation counters keep
+ * their epochs on the device), so it may be recorded by stream capture and replayed as a CUDA
+ * graph; the first call must come before the capture. */
 gc_status_t gc_execute(gc_compiled_t* c, void* cuda_stream, const void* const* in_dev, int32_t n_in,
                        void* const* out_dev, int32_t n_out);
 

@@ -221,7 +221,6 @@ struct LayerPlan {
   std::vector<int> pair_sched;   // [clusters][pair_pitch] tile lists: (layer << 24) | tile, -1 terminated
   int pair_pitch = 0, pair_clusters = 0;
   size_t pair_sched_off = 0, pair_ready_off = 0;
-  unsigned long long pair_execs = 0;   // launches since the counters were cleared
   bool need_comp = false;        // tcgen05 path with a non-zero activation zero point
   size_t comp_off = 0;           // workspace offset of a_zp * colsum(W), s32 per output column
   // cached tensor maps
@@ -265,7 +264,6 @@ struct gc_compiled {
   uint32_t chain_w_smem = 0;
   int chain_a_stages = 0, chain_a_stage_bytes = 0, chain_a_rows = 0;
   std::vector<uint32_t> chain_w_off;         // per layer: offset of its weight slice in shared memory
-  unsigned long long chain_arrivals = 0;     // value of the grid-barrier counter after the launches so far
   std::vector<CUtensorMap> chain_tmaps;      // host copy of the tensor-map array
   const void* chain_a0_ptr = nullptr;        // first-layer A pointer the array was built for
   bool chain_tmaps_valid = false;
@@ -872,7 +870,7 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
       A.pair_sched_off = ws;
       ws = align_up(ws + A.pair_sched.size() * sizeof(int), 256);
       A.pair_ready_off = ws;
-      ws = align_up(ws + static_cast<size_t>(m_pairs) * sizeof(unsigned long long), 256);
+      ws = align_up(ws + static_cast<size_t>(m_pairs + 2) * sizeof(unsigned long long), 256);   // + epoch, finished CTAs
       c->launches -= 1;
       snprintf(line, sizeof(line), "  layers %zu+%zu: one launch, %d clusters, tile schedule over both (longest list %ld of %.1f k-blocks ideal)\n",
                l, l + 1, C, worst, target);
@@ -910,7 +908,6 @@ extern "C" gc_status_t gc_set_workspace(gc_compiled_t* c, void* ws, size_t bytes
   c->ws = ws;
   c->prepacked = false;
   c->status_cleared = false;
-  c->chain_arrivals = 0;                     // the header (status word + barrier counter) is cleared again
   c->chain_tmaps_valid = false;
   for (auto& L : c->layers) {
     L.tmA_ptr = nullptr;
@@ -964,8 +961,7 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
         CUDA_TRY(cudaMemcpyAsync(ws + L.pair_sched_off, L.pair_sched.data(), L.pair_sched.size() * sizeof(int),
                                  cudaMemcpyHostToDevice, st));
         const int m_pairs = (L.m_tiles + 1) / 2;
-        CUDA_TRY(cudaMemsetAsync(ws + L.pair_ready_off, 0, static_cast<size_t>(m_pairs) * sizeof(unsigned long long), st));
-        L.pair_execs = 0;
+        CUDA_TRY(cudaMemsetAsync(ws + L.pair_ready_off, 0, static_cast<size_t>(m_pairs + 2) * sizeof(unsigned long long), st));
       }
     }
     c.prepacked = true;
@@ -978,7 +974,7 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
     cp.a_stage_bytes = c.chain_a_stage_bytes;
     cp.status = status;
     cp.barrier = reinterpret_cast<unsigned long long*>(ws + 64);
-    cp.barrier_base = c.chain_arrivals;
+    cp.n_barriers = c.chain_barriers;
     cp.early_weights = need ? 0 : 1;
     cp.ks = c.chain_ks;
     const LayerPlan& L0 = c.layers[0];
@@ -1041,7 +1037,6 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
     }
     memcpy(cp.tmaps, c.chain_tmaps.data(), sizeof(cp.tmaps));
     CUDA_TRY(launch_mlp_chain(c.chain_kind, cp, c.chain_grid, st));
-    c.chain_arrivals += static_cast<unsigned long long>(c.chain_barriers) * c.chain_grid;
     return GC_OK;
   }
   GemmTcParams pair_first = {};
@@ -1116,10 +1111,10 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
         pp.sched_pitch = F.pair_pitch;
         pp.ready = reinterpret_cast<unsigned long long*>(ws + F.pair_ready_off);
         // every epilogue warp of both CTAs adds one per first-layer tile of the row block
-        pp.ready_target = (F.pair_execs + 1) * static_cast<unsigned long long>(F.n_tiles) * 16ull;
+        pp.m_pairs = (F.m_tiles + 1) / 2;
+        pp.ready_per_launch = static_cast<unsigned long long>(F.n_tiles) * 16ull;
         pp.status = status;
         CUDA_TRY(launch_gemm_tc2_fused(L.kind, F.a_dtype == GC_S8, pp, 2 * F.pair_clusters, st));
-        ++F.pair_execs;
         continue;
       }
       if (L.cta2)

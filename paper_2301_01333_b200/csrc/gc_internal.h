@@ -92,8 +92,13 @@ struct GemmPairParams {
   const int* sched;               // [clusters][sched_pitch]: (layer << 24) | tile, a negative entry ends a list;
   int sched_pitch;                // null: one layer whose implicit_tiles tiles the clusters take round robin
   int implicit_tiles;
-  unsigned long long* ready;      // per 256-row block: completed stores of the first layer (only grows); null for one layer
-  unsigned long long ready_target;   // the value a block's counter reaches in this launch
+  unsigned long long* ready;      // per 256-row block: completed stores of the first layer (only grows); null for one
+                                  // layer.  Two more words follow the counters: [m_pairs] = launches completed so far
+                                  // (the epoch: bumped by the last CTA to finish), [m_pairs + 1] = CTAs finished in
+                                  // this launch.  Keeping the epoch on the device (not in the launch parameters)
+                                  // is what makes a captured launch replayable.
+  int m_pairs;
+  unsigned long long ready_per_launch;   // arrivals a row block's counter receives per launch
   uint32_t* status;
   alignas(64) CUtensorMap tm[6];  // A, Wt, D of the first layer, then of the second
 };
@@ -126,7 +131,9 @@ struct ChainParams {
   int pack_rows;           // its rows (0: the first layer is fed by TMA like the others)
   int64_t pack_src_pitch;  // bytes
   unsigned long long* barrier;              // grid-barrier counter (only grows)
-  unsigned long long barrier_base;          // its value before this launch
+                                            // its value at the start of a launch is derived from the counter itself on
+                                            // the device, so that a captured launch can be replayed
+  int n_barriers;                           // grid barriers one launch passes
   int ks;                                   // CTAs per cluster = parts the reduction axis of every layer is split into
   int early_weights;                        // 1: the prepacked weights were written by an earlier call, so their loads
                                             // need not wait for the kernel that precedes this one on the stream

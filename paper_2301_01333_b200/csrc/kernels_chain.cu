@@ -199,7 +199,16 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
   }
 
   bool failed = false;
-  unsigned long long bar_count = p.barrier_base;                  // counter value before this launch
+  // Counter value before this launch (only thread 0 uses it).  Every completed launch has added
+  // (n_barriers + 1) * gridDim.x: one per CTA and barrier, plus one per CTA on the way out.  CTAs that are ahead of
+  // this one may already have arrived at the first barrier, but fewer than gridDim.x of them (this CTA has not), so
+  // rounding the value down to a multiple of the per-launch total recovers the start value.  Deriving it on the
+  // device instead of passing it as a launch parameter is what lets a captured launch be replayed.
+  unsigned long long bar_count = 0;
+  if (threadIdx.x == 0) {
+    const unsigned long long per_launch = static_cast<unsigned long long>(p.n_barriers + 1) * gridDim.x;
+    bar_count = ld_acquire_u64(p.barrier) / per_launch * per_launch;
+  }
   int stage = 0;                 // ring position, shared by construction between producer and MMA thread
   uint32_t phase = 0;
   uint32_t tphase = 0;           // parity of the accumulator-ready barrier (one completion per active layer)
@@ -455,6 +464,9 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
     tc_fence_after();
     tmem_dealloc(tmem_base, CH_NACC * CH_BLOCK_N);
   }
+  // one more count per CTA on the way out (nobody waits for it): it keeps the counter a multiple of the per-launch
+  // total between launches, which the start-value computation above relies on
+  if (threadIdx.x == 0) asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p.barrier), "l"(1ULL) : "memory");
   // no CTA leaves while another one of its cluster may still write into its shared memory
   if (KS > 1) cluster_sync_all();
 }

@@ -126,6 +126,9 @@ __global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_co
       int stage = 0;
       uint32_t phase = 0;
       const uint32_t leader_full = leader ? bar_full : mapa_shared(bar_full, 0);
+      // the value a row block's counter reaches in this launch: completed launches are counted on the device
+      const unsigned long long ready_target =
+          p.ready ? (f2_ld_acquire(p.ready + p.m_pairs) + 1ULL) * p.ready_per_launch : 0ULL;
       for (int i = 0; i < list_len && !failed; ++i) {
         const int e = entry(i);
         if (e < 0) break;
@@ -137,7 +140,7 @@ __global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_co
           // the 256 hidden rows this tile reads: wait until every store of that row block has completed
           const uint64_t t0 = globaltimer_ns();
           uint32_t spins = 0;
-          while (f2_ld_acquire(p.ready + m_pair) < p.ready_target) {
+          while (f2_ld_acquire(p.ready + m_pair) < ready_target) {
             if ((++spins & 255u) == 0 && globaltimer_ns() - t0 > 2000000000ull) {
               report(p.status, DEV_TIMEOUT_PRODUCER);
               failed = true;
@@ -300,6 +303,15 @@ __global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_co
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc2(tmem_base, F2_TMEM_COLS);
+  }
+  // the last CTA to get here closes the launch (see GemmPairParams::ready)
+  if (p.ready && threadIdx.x == 0) {
+    const unsigned long long prev = atomicAdd(p.ready + p.m_pairs + 1, 1ULL);
+    if (prev + 1 == gridDim.x) {
+      atomicExch(p.ready + p.m_pairs + 1, 0ULL);
+      __threadfence();
+      atomicAdd(p.ready + p.m_pairs, 1ULL);
+    }
   }
   if (failed) {
     const uint64_t t0 = globaltimer_ns();

@@ -588,6 +588,59 @@ def test_repeated_runs_are_bitwise_identical(B):
         assert np.array_equal(res[0], res[1]) and np.array_equal(res[0], res[2])
 
 
+@pytest.mark.parametrize("which", ["chain", "two_layers_one_launch", "attention"])
+def test_captured_executes_replay_correctly(B, which):
+    # gc_execute after the first call is a pure sequence of kernel launches: captured into a CUDA graph and replayed,
+    # it must give the same results, also for the kernels that synchronise through counters in global memory
+    # (their epochs live on the device, not in the launch parameters), and with new input contents per replay
+    import torch
+    if which == "chain":
+        w = W.mlp_int8(batch=128, dims=(479, 1024, 512, 32), final="none", per_channel=True, x_zp=3, act_zp=2)
+    elif which == "two_layers_one_launch":
+        w = W.ffn_bf16(tokens=4900, d_model=1024, d_ff=1024)
+    else:
+        w = W.mha_int8(batch=2, heads=4, seq=384, head_dim=64)
+    c = B.CompiledPartition(w.graph, 0)
+    ins = B.device_inputs(w)
+    outs = B.device_outputs(w.graph)
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        c.execute(ins, outs, s.cuda_stream)                 # first call: constant preprocessing, outside the graph
+    s.synchronize()
+    first = B.output_to_numpy(w.graph, w.graph.outputs[0], outs[0]).copy()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=s):
+        for _ in range(3):
+            c.execute(ins, outs, s.cuda_stream)
+    for _ in range(2):
+        outs[0].zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(B.output_to_numpy(w.graph, w.graph.outputs[0], outs[0]), first)
+    # new activations in the same buffer, one more replay, then an ordinary call again
+    x_pos = 0
+    x_id = w.graph.inputs[x_pos]
+    new_x = np.roll(w.feeds[x_id], 1, axis=0).copy()
+    ins[x_pos].copy_(torch.from_numpy(np.ascontiguousarray(new_x).view(np.uint8).reshape(-1)))
+    g.replay()
+    torch.cuda.synchronize()
+    replayed = B.output_to_numpy(w.graph, w.graph.outputs[0], outs[0]).copy()
+    c.execute(ins, outs)
+    c.query_status()
+    torch.cuda.synchronize()
+    assert np.array_equal(B.output_to_numpy(w.graph, w.graph.outputs[0], outs[0]), replayed)
+    assert not np.array_equal(replayed, first)
+    w.feeds[x_id] = new_x
+    ref = oracle(w)
+    if which == "chain":
+        assert np.array_equal(replayed, ref)
+    elif which == "attention":
+        check_int8_attention(replayed, ref)
+    else:
+        assert np.abs(bf16_to_f64(replayed) - ref).max() <= 2e-2
+    c.close()
+
+
 def test_host_buffer_entry_point_matches_device_entry_point(B):
     import torch
     w = W.mlp_int8()
