@@ -259,7 +259,7 @@ struct gc_compiled {
   std::string desc;
   // fused small-batch chain (one persistent kernel for all layers)
   bool chain_fused = false;
-  int chain_kind = 0, chain_grid = 0, chain_barriers = 0, chain_ks = 1;
+  int chain_kind = 0, chain_grid = 0, chain_barriers = 0, chain_ks = 1, chain_slices = 0;
   size_t chain_tmap_off = 0;                 // workspace offset of the tensor-map array
   uint32_t chain_w_smem = 0;
   int chain_a_stages = 0, chain_a_stage_bytes = 0, chain_a_rows = 0;
@@ -723,11 +723,12 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
     int kind = -1, max_ctas = 0, max_nkb = 1, a_rows = 8;
     for (size_t l = 0; l < c->layers.size() && ok; ++l) {
       LayerPlan& L = c->layers[l];
-      ok = L.M <= 128;
+      ok = L.M <= 512;
       const int lk = is_int8(L.a_dtype) ? 0 : (L.a_dtype == GC_BF16 ? 1 : 2);
       if (kind < 0) kind = lk;
       ok = ok && lk == kind;
-      a_rows = ((L.M + 7) / 8 * 8) > a_rows ? ((L.M + 7) / 8 * 8) : a_rows;
+      const int rows = L.M < 128 ? (L.M + 7) / 8 * 8 : 128;       // rows of one row tile
+      a_rows = rows > a_rows ? rows : a_rows;
       if (L.use_tc) {
         const int ctas = (L.N + 31) / 32;
         max_ctas = ctas > max_ctas ? ctas : max_ctas;
@@ -739,7 +740,9 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
     // A-operand ring: round_up(M, 8) rows per stage and one stage per k-block a CTA handles in the deepest
     // layer, so every layer fetches its whole A operand in one burst.
     const int a_stage_bytes = a_rows * 128;
+    const int row_tiles = c->layers.empty() ? 1 : (c->layers[0].M + 127) / 128;   // all layers of a chain share M
     int ks = max_nkb >= 8 ? 4 : (max_nkb >= 4 ? 2 : 1);
+    while (ks > 1 && max_ctas * ks * row_tiles > c->num_sms) ks >>= 1;   // row tiles come before splitting the reduction
     int a_stages = 0;
     uint32_t w_smem = 0;
     ok = ok && max_ctas > 0;
@@ -752,13 +755,13 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
       }
       a_stages = (max_nkb + ks - 1) / ks;
       const size_t smem = mlp_chain_smem_bytes(w_smem, a_stages, a_stage_bytes);
-      bool fits = a_stages <= 32 && max_ctas * ks <= c->num_sms && smem <= static_cast<size_t>(prop.sharedMemPerBlockOptin);
+      bool fits = a_stages <= 32 && max_ctas * ks * row_tiles <= c->num_sms && smem <= static_cast<size_t>(prop.sharedMemPerBlockOptin);
       // all clusters must be resident together (the layers are separated by a grid-wide barrier)
       if (fits && ks > 1 && cuda_device != GC_DEVICE_PLAN_ONLY) {
         int cur = -1;
         cudaGetDevice(&cur);
         if (cur != cuda_device) cudaSetDevice(cuda_device);     // the occupancy query answers for the current device
-        fits = mlp_chain_max_clusters(kind, ks, smem) >= max_ctas;
+        fits = mlp_chain_max_clusters(kind, ks, smem) >= max_ctas * row_tiles;
         if (cur >= 0 && cur != cuda_device) cudaSetDevice(cur);
       }
       if (fits) break;
@@ -770,15 +773,16 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
       c->chain_a_rows = a_rows;
       c->chain_fused = true;
       c->chain_kind = kind;
-      c->chain_grid = max_ctas * ks;
+      c->chain_grid = max_ctas * ks * row_tiles;
       c->chain_ks = ks;
+      c->chain_slices = max_ctas;
       c->chain_w_smem = w_smem;
       c->chain_barriers = static_cast<int>(c->layers.size()) - 1;   // one grid barrier between consecutive layers
       c->chain_tmap_off = ws;
       ws = align_up(ws + 2 * CHAIN_MAX_LAYERS * sizeof(CUtensorMap), 1024);
       c->launches = 1;
       snprintf(line, sizeof(line), "  fused chain: one persistent kernel, %d CTAs in clusters of %d (split reduction axis), %u KB of resident weight slices per CTA, %d grid barriers\n",
-               max_ctas * ks, ks, w_smem / 1024, c->chain_barriers);
+               max_ctas * ks * row_tiles, ks, w_smem / 1024, c->chain_barriers);
       c->desc += line;
     }
   }
@@ -977,6 +981,7 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
     cp.n_barriers = c.chain_barriers;
     cp.early_weights = need ? 0 : 1;
     cp.ks = c.chain_ks;
+    cp.slices = c.chain_slices;
     const LayerPlan& L0 = c.layers[0];
     const void* a0 = in[L0.a_input];
     if (L0.need_pack) {

@@ -135,6 +135,7 @@ struct ChainParams {
                                             // the device, so that a captured launch can be replayed
   int n_barriers;                           // grid barriers one launch passes
   int ks;                                   // CTAs per cluster = parts the reduction axis of every layer is split into
+  int slices;                               // 32-column slices per row tile: grid = row tiles x slices x ks
   int early_weights;                        // 1: the prepacked weights were written by an earlier call, so their loads
                                             // need not wait for the kernel that precedes this one on the stream
   uint32_t* status;

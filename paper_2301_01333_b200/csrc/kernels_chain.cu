@@ -2,7 +2,7 @@
 // Section V: the outer loops of consecutive fused ops merged so that activations stay in the fastest cache
 // and the per-op synchronisation overhead disappears; Section VII: 2.0x on the int8 MLP-1).
 //
-// Shape of the problem: M <= 128 rows (one MMA row tile), L layers with N_l output columns.  CTA c owns
+// Shape of the problem: M <= 512 rows (up to four independent 128-row MMA tiles), L layers with N_l output columns.  CTA c owns
 // output columns [32 c, 32 c + 32) of every tensor-core layer that has that many columns:
 //   * at kernel start it TMA-loads its 32-row slice of EVERY layer's prepacked weight into shared memory
 //     (HBM latency is paid once, not once per layer);
@@ -137,7 +137,10 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
   const uint32_t bar_wfull = bar_a0 + 8;                          // [CHAIN_MAX_LAYERS]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int ksr = KS > 1 ? static_cast<int>(cluster_ctarank()) : 0;   // my part of the reduction axis
-  const int cta = blockIdx.x / KS;                                // my 32-column slice
+  // CTA index -> (row tile, 32-column slice, part of the reduction axis): batches above 128 rows are cut into row
+  // tiles that run as independent CTAs (rows of a matmul are independent); only the grid barrier joins them
+  const int cta = (blockIdx.x / KS) % p.slices;                   // my 32-column slice
+  const int row0 = (blockIdx.x / KS) / p.slices * 128;            // first row of my row tile
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < CH_STAGES; ++s) {
@@ -223,7 +226,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
     const int lo = kb_lo(L), hi = kb_hi(L);
     for (int kb = lo; kb < hi; ++kb) {
       mbar_arrive_expect_tx(bar_full + 8 * stage, CH_A_STAGE_BYTES);
-      tma_load_2d(smem_u32(sA) + stage * CH_A_STAGE_BYTES, p.tmaps + L.a_tm, kb * K_ELEMS, 0, bar_full + 8 * stage);
+      tma_load_2d(smem_u32(sA) + stage * CH_A_STAGE_BYTES, p.tmaps + L.a_tm, kb * K_ELEMS, row0, bar_full + 8 * stage);
       if (++stage == CH_STAGES) {
         stage = 0;
         phase ^= 1;
@@ -293,7 +296,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
             const int r = q * 32 + lane;
             const int a_rows = CH_A_STAGE_BYTES / 128;
             const int64_t kbytes = static_cast<int64_t>(L.K) * ESZ;
-            const uint8_t* src_row = static_cast<const uint8_t*>(p.pack_src) + static_cast<int64_t>(r) * p.pack_src_pitch;
+            const uint8_t* src_row = static_cast<const uint8_t*>(p.pack_src) + static_cast<int64_t>(row0 + r) * p.pack_src_pitch;
             if (r < a_rows) {
               for (int i = 0; i < my_nkb; ++i) {
                 uint8_t* dst = sA + i * CH_A_STAGE_BYTES + (r >> 3) * 1024 + (r & 7) * 128;
@@ -301,7 +304,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
                 for (int c = 0; c < 8; ++c) {
                   const int64_t off = static_cast<int64_t>(lo + i) * 128 + c * 16;     // byte offset inside the row
                   int64_t nv = kbytes - off;                                             // valid bytes of this chunk
-                  nv = r < L.M ? (nv > 16 ? 16 : nv) : 0;
+                  nv = row0 + r < L.M ? (nv > 16 ? 16 : nv) : 0;
                   uint32_t o[4] = {0u, 0u, 0u, 0u};
                   if (nv > 0) {
                     const uintptr_t a = reinterpret_cast<uintptr_t>(src_row + off);
@@ -362,7 +365,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
             tc_fence_before();
             const int n0 = cta * CH_BLOCK_N;
             if (KS == 1) {
-              const int row = q * 32 + lane;
+              const int row = row0 + q * 32 + lane;
               if (row < L.M) {
                 char* dst_row = static_cast<char*>(L.out) + static_cast<int64_t>(row) * L.out_pitch * L.out_elem;
                 if (n0 < L.N) epi_store16(r, dst_row, n0, L.epi);
@@ -405,7 +408,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
                       }
                     }
                   }
-                  const int grow = ksr * rows_per + frow;
+                  const int grow = row0 + ksr * rows_per + frow;
                   if (grow < L.M) {
                     char* dst_row = static_cast<char*>(L.out) + static_cast<int64_t>(grow) * L.out_pitch * L.out_elem;
                     epi_store16_cols(a, dst_row, fcol, L.epi, fk);
