@@ -143,7 +143,7 @@ struct ChainParams {
   // kept in global memory cost a fetch of several hundred clocks on every load instruction.
   alignas(64) CUtensorMap tmaps[2 * CHAIN_MAX_LAYERS];
 };
-size_t mlp_chain_smem_bytes(size_t w_smem_bytes, int a_stages, int a_stage_bytes);
+size_t mlp_chain_smem_bytes(size_t w_smem_bytes, int a_stages, int a_stage_bytes, int ks);
 cudaError_t launch_mlp_chain(int kind, const ChainParams& p, int grid, cudaStream_t s);
 // clusters of `ks` CTAs of the chain kernel that can be resident together on the current device (0 on error)
 int mlp_chain_max_clusters(int kind, int ks, size_t smem);

@@ -128,7 +128,8 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
   // partial sums from the cluster: [KS sources][128 / KS rows][32 columns] s32 / fp32, 16-byte chunks XOR-swizzled
   uint8_t* sRed = sW + (p.w_smem_bytes < 16384u ? 16384u : p.w_smem_bytes);
   uint8_t* sSend = sRed + CH_RED_BYTES;                           // my own partial sums, staged for the bulk copies
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sSend + CH_RED_BYTES);
+  // (neither buffer exists when the reduction axis is not split)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sRed + (KS > 1 ? 2 * CH_RED_BYTES : 0));
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * CH_MAX_STAGES + 3 + CHAIN_MAX_LAYERS);
   const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * CH_MAX_STAGES;
   const uint32_t bar_tfull = bar_empty + 8 * CH_MAX_STAGES;       // [1]
@@ -474,13 +475,13 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
   if (KS > 1) cluster_sync_all();
 }
 
-size_t mlp_chain_smem_bytes(size_t w_smem_bytes, int a_stages, int a_stage_bytes) {
+size_t mlp_chain_smem_bytes(size_t w_smem_bytes, int a_stages, int a_stage_bytes, int ks) {
   return ((static_cast<size_t>(a_stages) * a_stage_bytes + 1023) & ~size_t(1023)) +
-         (w_smem_bytes < 16384 ? size_t(16384) : w_smem_bytes) + 2 * CH_RED_BYTES + 1024 + 1024;
+         (w_smem_bytes < 16384 ? size_t(16384) : w_smem_bytes) + (ks > 1 ? 2 * CH_RED_BYTES : 0) + 1024 + 1024;
 }
 
 cudaError_t launch_mlp_chain(int kind, const ChainParams& p, int grid, cudaStream_t s) {
-  const size_t smem = mlp_chain_smem_bytes(p.w_smem_bytes, p.a_stages, p.a_stage_bytes);
+  const size_t smem = mlp_chain_smem_bytes(p.w_smem_bytes, p.a_stages, p.a_stage_bytes, p.ks);
   void* kern = kind == KIND_I8 ? reinterpret_cast<void*>(mlp_chain_kernel<KIND_I8>)
                : kind == KIND_BF16 ? reinterpret_cast<void*>(mlp_chain_kernel<KIND_BF16>)
                                    : reinterpret_cast<void*>(mlp_chain_kernel<KIND_TF32>);

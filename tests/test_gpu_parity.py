@@ -169,7 +169,7 @@ def test_int8_matmul_nonzero_zero_point_on_tensor_cores_exact(B, m, k, n, zp):
 
 @pytest.mark.parametrize("batch,dims,ks", [(64, (600, 256, 64), 2), (77, (700, 128, 32), 2), (33, (131, 64, 16), 1),
                                            (128, (1030, 512, 256, 32), 4), (1, (479, 1024, 16), 4),
-                                           (256, (479, 1024, 1024, 512, 256, 1), 2), (512, (100, 1024, 32), 1),
+                                           (256, (479, 1024, 1024, 512, 256, 1), 2), (512, (100, 304, 32), 1), (512, (100, 512, 32), 2),
                                            (300, (13, 512, 256, 128), 2), (130, (70, 64, 32), 1)])
 def test_mlp_int8_chain_kernel_cluster_sizes_and_entry_reorder(B, batch, dims, ks):
     # the fused chain kernel with the reduction axis split over 1, 2 and 4 CTAs, inputs whose rows start at every
