@@ -211,6 +211,14 @@ gc_status_t gc_matmul_s32_noalloc(void* cuda_stream, const void* a_dev, const vo
                                   int32_t m, int32_t k, int32_t n, int32_t a_zero_point);
 size_t gc_noalloc_scratch_bytes(void);
 
+/* No counterpart in the paper: a self-test of the error path of the kernels' bounded waits.  Every wait inside
+ * the kernels (on an mbarrier, on a counter in global memory) gives up after a time limit, records a code in the
+ * status word and lets the kernel return, so that the context stays usable and gc_query_status can report
+ * GC_ERR_TIMEOUT.  This call launches one small kernel whose wait can never be satisfied (a barrier nobody arrives
+ * on), limited to limit_us microseconds (at most 100 000), and which then writes its code to *status_dev
+ * (a 4-byte device word the caller has zeroed).  Asynchronous on cuda_stream. */
+gc_status_t gc_selftest_bounded_wait(void* cuda_stream, void* status_dev, uint32_t limit_us);
+
 const char* gc_last_error(void);
 const char* gc_version(void);
 

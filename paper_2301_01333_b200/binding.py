@@ -33,7 +33,7 @@ EXPORTS = [
     "gc_partition_create", "gc_partition_destroy", "gc_compile", "gc_compiled_destroy", "gc_workspace_bytes",
     "gc_set_workspace", "gc_execute", "gc_host_staging_bytes", "gc_set_host_staging", "gc_execute_host",
     "gc_query_status", "gc_launches_per_execute", "gc_plan_description", "gc_last_error", "gc_version",
-    "gc_matmul_s32_noalloc", "gc_noalloc_scratch_bytes",
+    "gc_matmul_s32_noalloc", "gc_noalloc_scratch_bytes", "gc_selftest_bounded_wait",
 ]
 
 
@@ -94,6 +94,8 @@ def load_library() -> C.CDLL:
     lib.gc_matmul_s32_noalloc.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32]
     lib.gc_matmul_s32_noalloc.restype = i32
     lib.gc_noalloc_scratch_bytes.restype = sz
+    lib.gc_selftest_bounded_wait.argtypes = [vp, vp, C.c_uint32]
+    lib.gc_selftest_bounded_wait.restype = i32
     for name in ("gc_partition_create", "gc_compile", "gc_workspace_bytes", "gc_set_workspace", "gc_execute",
                  "gc_host_staging_bytes", "gc_set_host_staging", "gc_execute_host", "gc_query_status",
                  "gc_launches_per_execute"):
@@ -236,6 +238,11 @@ def gc_matmul_s32_noalloc(stream: int, a_ptr: int, w_ptr: int, out_ptr: int, m: 
     that cannot allocate: the scratch is a fixed 1 MiB array inside the library, shared by all calls."""
     _check(load_library().gc_matmul_s32_noalloc(C.c_void_p(stream), C.c_void_p(a_ptr), C.c_void_p(w_ptr),
                                                 C.c_void_p(out_ptr), m, k, n, a_zero_point))
+
+
+def gc_selftest_bounded_wait(stream: int, status_ptr: int, limit_us: int) -> None:
+    """Launch the kernel whose wait cannot be satisfied; after limit_us it writes a timeout code to *status_ptr."""
+    _check(load_library().gc_selftest_bounded_wait(C.c_void_p(stream), C.c_void_p(status_ptr), limit_us))
 
 
 class CompiledPartition:

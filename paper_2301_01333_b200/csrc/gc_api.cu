@@ -1280,6 +1280,15 @@ extern "C" gc_status_t gc_execute_host(gc_compiled_t* c, void* cuda_stream, cons
   return GC_OK;
 }
 
+extern "C" gc_status_t gc_selftest_bounded_wait(void* cuda_stream, void* status_dev, uint32_t limit_us) {
+  if (!status_dev) return fail(GC_ERR_INVALID_ARG, "null argument");
+  if (reinterpret_cast<uintptr_t>(status_dev) % 4) return fail(GC_ERR_ALIGNMENT, "status word must be 4-byte aligned");
+  if (limit_us > 100000u) limit_us = 100000u;
+  CUDA_TRY(launch_bounded_wait_selftest(static_cast<uint32_t*>(status_dev), static_cast<uint64_t>(limit_us) * 1000ull,
+                                        static_cast<cudaStream_t>(cuda_stream)));
+  return GC_OK;
+}
+
 extern "C" gc_status_t gc_query_status(gc_compiled_t* c, void* cuda_stream) {
   if (!c) return fail(GC_ERR_INVALID_ARG, "null argument");
   if (!c->ws) return fail(GC_ERR_STATE, "gc_set_workspace has not been called");

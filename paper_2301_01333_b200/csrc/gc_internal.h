@@ -158,6 +158,8 @@ cudaError_t launch_prepack_weight(const void* W, void* Wt, int K, int N, int Kp,
 // comp[n] = a_zp * sum_k Wt[n][k] for a prepacked s8 weight (zero padded to Kp)
 cudaError_t launch_weight_compensation(const void* Wt, int N, int Kp, int a_zp, int* comp, cudaStream_t s);
 cudaError_t launch_gemm_simt(const GemmSimtParams& p, cudaStream_t s);
+// one small kernel that waits on a barrier nobody arrives on, gives up after limit_ns and records a timeout code
+cudaError_t launch_bounded_wait_selftest(uint32_t* status, uint64_t limit_ns, cudaStream_t s);
 cudaError_t launch_sdpa_simt(const SdpaParams& p, cudaStream_t s);
 
 // kind: 0 = i8 (u8/s8 x s8 -> s32), 1 = bf16, 2 = tf32.  a_signed only matters for kind 0.

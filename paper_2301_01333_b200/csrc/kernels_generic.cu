@@ -7,6 +7,7 @@
 
 #include "epilogue.cuh"
 #include "gc_internal.h"
+#include "ptx.cuh"
 
 namespace gc {
 
@@ -90,6 +91,30 @@ cudaError_t launch_prepack_weight(const void* W, void* Wt, int K, int N, int Kp,
   else
     prepack_weight_kernel<uint8_t, false><<<grid, block, 0, s>>>(static_cast<const uint8_t*>(W),
                                                                 static_cast<uint8_t*>(Wt), K, N, Kp, transposed);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Self-test of the bounded-wait error path: a wait on a barrier that nobody arrives on, limited in time.
+// ------------------------------------------------------------------------------------------------
+__global__ void bounded_wait_selftest_kernel(uint32_t* status, uint64_t limit_ns) {
+  __shared__ uint64_t bar;
+  const uint32_t b = smem_u32(&bar);
+  if (threadIdx.x == 0) {
+    mbar_init(b, 1);
+    fence_mbar_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const uint64_t t0 = globaltimer_ns();
+    bool done = false;
+    while (!done && globaltimer_ns() - t0 < limit_ns) done = mbar_try_wait(b, 0, 1000u);
+    if (!done) report(status, DEV_TIMEOUT_OTHER);
+  }
+}
+
+cudaError_t launch_bounded_wait_selftest(uint32_t* status, uint64_t limit_ns, cudaStream_t s) {
+  bounded_wait_selftest_kernel<<<1, 32, 0, s>>>(status, limit_ns);
   return cudaGetLastError();
 }
 

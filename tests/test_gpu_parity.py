@@ -643,6 +643,24 @@ def test_captured_executes_replay_correctly(B, which):
     c.close()
 
 
+def test_bounded_wait_gives_up_records_a_code_and_leaves_the_context_usable(B):
+    # the error path every kernel wait has: a wait that cannot be satisfied ends after its time limit, the kernel
+    # writes its code and returns; the context keeps working
+    import time
+    import torch
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    B.gc_selftest_bounded_wait(torch.cuda.current_stream(0).cuda_stream, status.data_ptr(), 20000)   # 20 ms
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    assert int(status.item()) != 0
+    assert 0.015 <= dt < 1.0
+    w = W.single_matmul("u8", "s8", 128, 128, 64, seed=1)
+    got, _ = run_gpu(B, w)
+    assert np.array_equal(got.astype(np.int64), oracle(w))
+
+
 def test_host_buffer_entry_point_matches_device_entry_point(B):
     import torch
     w = W.mlp_int8()
