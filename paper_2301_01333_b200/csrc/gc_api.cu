@@ -6,6 +6,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -220,7 +221,7 @@ struct LayerPlan {
   bool fused_first = false;
   std::vector<int> pair_sched;   // [clusters][pair_pitch] tile lists: (layer << 24) | tile, -1 terminated
   int pair_pitch = 0, pair_clusters = 0;
-  size_t pair_sched_off = 0, pair_ready_off = 0;
+  size_t pair_sched_off = 0, pair_ready_off = 0, pair_ready_words = 0;
   bool need_comp = false;        // tcgen05 path with a non-zero activation zero point
   size_t comp_off = 0;           // workspace offset of a_zp * colsum(W), s32 per output column
   // cached tensor maps
@@ -807,51 +808,50 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
       const long T0 = static_cast<long>(m_pairs) * A.n_tiles, T1 = static_cast<long>(m_pairs) * B.n_tiles;
       const long w0 = A.nkb, w1 = B.nkb;
       if (T0 + T1 < 2L * C || T0 >= (1L << 24) || T1 >= (1L << 24)) continue;
-      // Schedule (static, built here): first-layer tiles in row-block order, round robin over the clusters that
-      // still have quota; second-layer tiles in row-block order, each to the cluster that is free first, starting
-      // no earlier than its row block is ready.  A row block is ready a while after its last first-layer tile's
-      // main loop ends (epilogue, store completion, counter, the poll: about 24 k-block times measured on this
-      // workload), so first-layer work must not end everywhere at the last moment.  The clusters that will take
-      // one second-layer tile fewer take e extra first-layer tiles instead; e is chosen by simulating the step.
-      const long lat = 24;
+      // Schedule (static, built here).  Every cluster's list holds its first-layer tiles, then its second-layer
+      // tiles, so first-layer work never waits and the waits of the second layer cannot deadlock.  A second-layer
+      // tile reads its A operand (256 hidden rows) in groups of k-blocks, one group per first-layer tile of that row
+      // block, and waits group by group, so it can run right behind the tiles that produce its operand.  A tile
+      // becomes readable a while after its main loop ends (epilogue, store completion, counter, the poll: about 24
+      // k-block times measured on the FFN workload).  Candidates are built two ways and the step is simulated for
+      // each; the shortest one wins:
+      //  * "even": first-layer tiles round robin in row-block order; the clusters that will take one second-layer
+      //    tile fewer take e = 0..4 extra first-layer tiles; second-layer tiles to whichever cluster is free first;
+      //  * "balanced": second-layer quotas differ by at most one, first-layer quotas fill every cluster up to the
+      //    same total work; the first-layer tiles of the slots in which only the clusters with large quotas are
+      //    still busy (the tail) are dealt out column by column over the remaining row blocks, so that each of
+      //    those row blocks becomes readable group by group in the order its consumers read it.
+      const long lat = 24, lat_next = 20;
+      const long kpg = B.kind == 0 ? 2 : (B.kind == 1 ? 4 : 8);   // (i8, bf16, tf32) second-layer k-blocks per first-layer tile
       const int heavy = T1 % C ? C - static_cast<int>(T1 % C) : 0;   // clusters with one second-layer tile fewer
       long best_span = -1;
       std::vector<int> best_sched;
       int best_pitch = 0;
-      for (int e = 0; e <= 4; ++e) {
-        if (e > 0 && heavy == 0) break;
-        // first-layer quotas: heavy clusters (the last ones) get e more than the light ones
-        std::vector<long> n0(C, 0);
-        const long light = C - heavy;
-        long base = (T0 - static_cast<long>(heavy) * e) / C;
-        if (base < 0) break;
-        long rest = T0 - base * C - static_cast<long>(heavy) * e;
-        for (int k = 0; k < C; ++k) n0[k] = base + (k >= light ? e : 0);
-        for (int k = 0; rest > 0; k = (k + 1) % C, --rest) ++n0[k];
-        // first layer: tile index -> (cluster, position); finish time of each tile
-        std::vector<std::vector<int>> list(C);
-        std::vector<long> done0(T0);
-        long next0 = 0;
-        while (next0 < T0)
-          for (int k = 0; k < C && next0 < T0; ++k)
-            if (static_cast<long>(list[k].size()) < n0[k]) {
-              list[k].push_back(static_cast<int>(next0));
-              done0[next0] = static_cast<long>(list[k].size()) * w0;
-              ++next0;
-            }
-        std::vector<long> ready(m_pairs, 0), avail(C);
-        for (long t = 0; t < T0; ++t) {
-          const long mp = t / A.n_tiles;
-          ready[mp] = done0[t] + lat > ready[mp] ? done0[t] + lat : ready[mp];
+      // simulate the second layer over given first-layer lists; quota[k] < 0: no limit
+      auto finish = [&](std::vector<std::vector<int>>& list, std::vector<long> quota) {
+        // when a first-layer tile becomes readable: the last one of a list lat after its main loop; the others
+        // are announced at the end of the epilogue of the tile that follows them (see the kernel)
+        std::vector<long> ready0(T0, 0), avail(C);
+        for (int k = 0; k < C; ++k) {
+          const size_t n = list[k].size();
+          for (size_t i = 0; i < n; ++i)
+            ready0[list[k][i]] = i + 1 == n ? static_cast<long>(i + 1) * w0 + lat : static_cast<long>(i + 2) * w0 + lat_next;
+          avail[k] = static_cast<long>(n) * w0;
         }
-        for (int k = 0; k < C; ++k) avail[k] = n0[k] * w0;
         for (long t = 0; t < T1; ++t) {
-          int bestk = 0;
-          for (int k = 1; k < C; ++k)
-            if (avail[k] < avail[bestk]) bestk = k;
+          int bestk = -1;
+          for (int k = 0; k < C; ++k)
+            if (quota[k] != 0 && (bestk < 0 || avail[k] < avail[bestk])) bestk = k;
+          if (bestk < 0) return;
           const long mp = t / B.n_tiles;
-          const long start = avail[bestk] > ready[mp] ? avail[bestk] : ready[mp];
-          avail[bestk] = start + w1;
+          long tt = avail[bestk];
+          for (long j = 0; j < A.n_tiles; ++j) {
+            const long r = ready0[mp * A.n_tiles + j];
+            tt = (tt > r ? tt : r) + kpg;
+          }
+          tt += w1 - kpg * A.n_tiles > 0 ? w1 - kpg * A.n_tiles : 0;
+          avail[bestk] = tt;
+          if (quota[bestk] > 0) --quota[bestk];
           list[bestk].push_back((1 << 24) | static_cast<int>(t));
         }
         long span = 0;
@@ -867,6 +867,60 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
           for (int k = 0; k < C; ++k)
             for (size_t i = 0; i < list[k].size(); ++i) best_sched[static_cast<size_t>(k) * best_pitch + i] = list[k][i];
         }
+      };
+      for (int e = 0; e <= 4; ++e) {                                // "even"
+        if (e > 0 && heavy == 0) break;
+        std::vector<long> n0(C, 0);
+        const long light = C - heavy;
+        long base = (T0 - static_cast<long>(heavy) * e) / C;
+        if (base < 0) break;
+        long rest = T0 - base * C - static_cast<long>(heavy) * e;
+        for (int k = 0; k < C; ++k) n0[k] = base + (k >= light ? e : 0);
+        for (int k = 0; rest > 0; k = (k + 1) % C, --rest) ++n0[k];
+        std::vector<std::vector<int>> list(C);
+        long next0 = 0;
+        while (next0 < T0)
+          for (int k = 0; k < C && next0 < T0; ++k)
+            if (static_cast<long>(list[k].size()) < n0[k]) list[k].push_back(static_cast<int>(next0++));
+        finish(list, std::vector<long>(C, -1));
+      }
+      {                                                             // "balanced"
+        const double target = static_cast<double>(T0 * w0 + T1 * w1) / C;
+        std::vector<long> b1(C), a0(C);
+        long sum = 0;
+        for (int k = 0; k < C; ++k) {
+          b1[k] = T1 / C + (k < T1 % C ? 1 : 0);
+          const double room = (target - static_cast<double>(b1[k] * w1)) / static_cast<double>(w0);
+          a0[k] = room > 0 ? static_cast<long>(room + 0.5) : 0;
+          sum += a0[k];
+        }
+        while (sum != T0) {                                         // rounding: take from the fullest / give to the emptiest
+          int pick = -1;
+          for (int k = 0; k < C; ++k) {
+            if (sum > T0 && a0[k] == 0) continue;
+            if (pick < 0) { pick = k; continue; }
+            const long lk = a0[k] * w0 + b1[k] * w1, lp = a0[pick] * w0 + b1[pick] * w1;
+            if (sum > T0 ? lk > lp : lk < lp) pick = k;
+          }
+          if (sum > T0) { --a0[pick]; --sum; } else { ++a0[pick]; ++sum; }
+        }
+        long amin = a0[0];
+        for (int k = 1; k < C; ++k) amin = a0[k] < amin ? a0[k] : amin;
+        std::vector<std::vector<int>> list(C);
+        const long n_body = amin * C;
+        for (long t = 0; t < n_body; ++t) list[t % C].push_back(static_cast<int>(t));
+        // the tail: column by column (j-major) over the remaining tiles, slot by slot over the clusters with quota left
+        std::vector<int> tail;
+        for (long j = 0; j < A.n_tiles; ++j)
+          for (long mp = 0; mp < m_pairs; ++mp)
+            if (mp * A.n_tiles + j >= n_body) tail.push_back(static_cast<int>(mp * A.n_tiles + j));
+        long amax = amin;
+        for (int k = 0; k < C; ++k) amax = a0[k] > amax ? a0[k] : amax;
+        size_t idx = 0;
+        for (long slot = amin; slot < amax && idx < tail.size(); ++slot)
+          for (int k = 0; k < C && idx < tail.size(); ++k)
+            if (static_cast<long>(list[k].size()) == slot && slot < a0[k]) list[k].push_back(tail[idx++]);
+        if (idx == tail.size()) finish(list, b1);
       }
       if (best_span < 0) continue;
       A.pair_pitch = best_pitch;
@@ -878,7 +932,9 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
       A.pair_sched_off = ws;
       ws = align_up(ws + A.pair_sched.size() * sizeof(int), 256);
       A.pair_ready_off = ws;
-      ws = align_up(ws + static_cast<size_t>(m_pairs + 2) * sizeof(unsigned long long), 256);   // + epoch, finished CTAs
+      // epoch, finished CTAs, then one counter per first-layer tile
+      A.pair_ready_words = 2 + static_cast<size_t>(T0);
+      ws = align_up(ws + A.pair_ready_words * sizeof(unsigned long long), 256);
       c->launches -= 1;
       snprintf(line, sizeof(line), "  layers %zu+%zu: one launch, %d clusters, tile schedule over both (longest list %ld of %.1f k-blocks ideal)\n",
                l, l + 1, C, worst, target);
@@ -968,8 +1024,7 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
       if (L.fused_first) {
         CUDA_TRY(cudaMemcpyAsync(ws + L.pair_sched_off, L.pair_sched.data(), L.pair_sched.size() * sizeof(int),
                                  cudaMemcpyHostToDevice, st));
-        const int m_pairs = (L.m_tiles + 1) / 2;
-        CUDA_TRY(cudaMemsetAsync(ws + L.pair_ready_off, 0, static_cast<size_t>(m_pairs + 2) * sizeof(unsigned long long), st));
+        CUDA_TRY(cudaMemsetAsync(ws + L.pair_ready_off, 0, L.pair_ready_words * sizeof(unsigned long long), st));
       }
     }
     c.prepacked = true;
@@ -1119,9 +1174,6 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
         pp.sched = reinterpret_cast<const int*>(ws + F.pair_sched_off);
         pp.sched_pitch = F.pair_pitch;
         pp.ready = reinterpret_cast<unsigned long long*>(ws + F.pair_ready_off);
-        // every epilogue warp of both CTAs adds one per first-layer tile of the row block
-        pp.m_pairs = (F.m_tiles + 1) / 2;
-        pp.ready_per_launch = static_cast<unsigned long long>(F.n_tiles) * 16ull;
         pp.status = status;
         CUDA_TRY(launch_gemm_tc2_fused(L.kind, F.a_dtype == GC_S8, pp, 2 * F.pair_clusters, st));
         continue;

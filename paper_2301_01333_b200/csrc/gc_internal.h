@@ -92,13 +92,11 @@ struct GemmPairParams {
   const int* sched;               // [clusters][sched_pitch]: (layer << 24) | tile, a negative entry ends a list;
   int sched_pitch;                // null: one layer whose implicit_tiles tiles the clusters take round robin
   int implicit_tiles;
-  unsigned long long* ready;      // per 256-row block: completed stores of the first layer (only grows); null for one
-                                  // layer.  Two more words follow the counters: [m_pairs] = launches completed so far
-                                  // (the epoch: bumped by the last CTA to finish), [m_pairs + 1] = CTAs finished in
-                                  // this launch.  Keeping the epoch on the device (not in the launch parameters)
-                                  // is what makes a captured launch replayable.
-  int m_pairs;
-  unsigned long long ready_per_launch;   // arrivals a row block's counter receives per launch
+  unsigned long long* ready;      // null for one layer.  [0] = launches completed so far (the epoch: bumped by the
+                                  // last CTA to finish; keeping it on the device, not in the launch parameters, is
+                                  // what makes a captured launch replayable), [1] = CTAs finished in this launch,
+                                  // [2 + tile] = one counter per first-layer tile: epilogue warps whose stores of the
+                                  // tile have completed (16 per launch; only grows)
   uint32_t* status;
   alignas(64) CUtensorMap tm[6];  // A, Wt, D of the first layer, then of the second
 };

@@ -25,9 +25,14 @@
 //   * the hidden tensor is read back soon after it was written, while it is still in L2.
 // Dependency: a tile of the second matmul reads 256 rows of the hidden tensor, which the n_tiles tiles of that
 // row block of the first matmul write (TMA stores of 2 CTAs x 8 epilogue warps each).  Every epilogue warp, once its
-// stores of a first-matmul tile have COMPLETED, adds one to the row block's counter in global memory (releasing);
-// the producer thread of a second-matmul tile polls the counter (acquiring, bounded) before it issues the loads of
-// its A operand.  The counters only grow; the host passes the value they reach in this launch.  The schedule puts
+// stores of a first-matmul tile have COMPLETED, adds one to that tile's counter in global memory (one releasing
+// reduction: a release costs 1300-2000 clocks here, so there is exactly one per warp and tile, and for all tiles
+// but the last first-matmul tile of a list it is deferred by one tile so that the wait for the stores is free).
+// The producer warp of a second-matmul tile reads the counters of the row block's tiles (acquiring, one per lane)
+// before it issues the loads of its A operand; for the tiles that are not complete yet it polls (bounded) right
+// before the group of k-blocks that covers that tile's 256 hidden columns, so the tile runs right behind its
+// producers.  The counters only grow; the value they reach in this launch follows from an epoch word kept on the
+// device.  The schedule puts
 // every first-matmul tile before every second-matmul tile in each cluster's list and all clusters are resident
 // (one CTA per SM), so the waits cannot deadlock.  Without a schedule (one layer) the clusters take the tiles
 // round robin.
@@ -45,7 +50,7 @@ constexpr int F2_B_ROWS = 128;           // Wt rows each CTA loads
 constexpr int F2_STAGES = 5;
 constexpr int F2_STAGE_BYTES = (F2_BLOCK_M + F2_B_ROWS) * 128;
 constexpr int F2_EPI_WARPS = 8;
-constexpr int F2_THREADS = 64 + 32 * F2_EPI_WARPS;
+constexpr int F2_THREADS = 64 + 32 * F2_EPI_WARPS + 32;   // producer, MMA issuer, epilogue warps, announcer
 constexpr int F2_STAGING_BYTES = F2_EPI_WARPS * 4096;
 constexpr int F2_BIAS_BYTES = F2_EPI_WARPS * F2_BLOCK_N * 4;
 constexpr int F2_TMEM_COLS = 512;
@@ -64,6 +69,7 @@ template <int KIND, int OUT>
 __global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_constant__ GemmPairParams p) {
   constexpr int A_BYTES = F2_BLOCK_M * 128;
   constexpr int K_ELEMS = KIND == KIND_I8 ? 128 : (KIND == KIND_BF16 ? 64 : 32);
+  constexpr int K_PER_TILE = F2_BLOCK_N / K_ELEMS;                // k-blocks of a second layer per first-layer tile
   constexpr int OUT_BYTES = out_bytes(OUT);
   constexpr int BOX_COLS = 128 / OUT_BYTES;
   constexpr int NUM_BOXES = F2_BLOCK_N / BOX_COLS;
@@ -73,12 +79,13 @@ __global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_co
   uint8_t* staging = smem + F2_STAGES * F2_STAGE_BYTES;
   float* bias_smem = reinterpret_cast<float*>(staging + F2_STAGING_BYTES);
   uint64_t* bars = reinterpret_cast<uint64_t*>(staging + F2_STAGING_BYTES + F2_BIAS_BYTES);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * F2_STAGES + 4);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * F2_STAGES + 6);
   const uint32_t smem_base = smem_u32(smem);
   const uint32_t bar_full = smem_u32(bars);                       // [STAGES]  (used in the leader)
   const uint32_t bar_empty = bar_full + 8 * F2_STAGES;            // [STAGES]
   const uint32_t bar_tfull = bar_empty + 8 * F2_STAGES;           // [2]
   const uint32_t bar_tempty = bar_tfull + 16;                     // [2]       (used in the leader)
+  const uint32_t bar_ann = bar_tempty + 16;                       // [2]  stores of a first-layer tile completed (per CTA)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
@@ -92,6 +99,7 @@ __global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_co
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_tfull + 8 * a, 1);
       mbar_init(bar_tempty + 8 * a, 2 * F2_EPI_WARPS);
+      mbar_init(bar_ann + 8 * a, F2_EPI_WARPS);
     }
     fence_mbar_init();
     for (int i = 0; i < 6; ++i) tma_prefetch_desc(&p.tm[i]);
@@ -122,37 +130,51 @@ __global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_co
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
-    if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      const uint32_t leader_full = leader ? bar_full : mapa_shared(bar_full, 0);
-      // the value a row block's counter reaches in this launch: completed launches are counted on the device
-      const unsigned long long ready_target =
-          p.ready ? (f2_ld_acquire(p.ready + p.m_pairs) + 1ULL) * p.ready_per_launch : 0ULL;
-      for (int i = 0; i < list_len && !failed; ++i) {
-        const int e = entry(i);
-        if (e < 0) break;
-        const int l = e >> 24, tile = e & 0xFFFFFF;
-        const int n_tiles = p.L[l].n_tiles, nkb = p.L[l].num_k_blocks;
-        const int m_pair = tile / n_tiles, n_blk = tile % n_tiles;
-        const int m_blk = m_pair * 2 + static_cast<int>(rank);
-        if (l == 1) {
-          // the 256 hidden rows this tile reads: wait until every store of that row block has completed
-          const uint64_t t0 = globaltimer_ns();
-          uint32_t spins = 0;
-          while (f2_ld_acquire(p.ready + m_pair) < ready_target) {
-            if ((++spins & 255u) == 0 && globaltimer_ns() - t0 > 2000000000ull) {
-              report(p.status, DEV_TIMEOUT_PRODUCER);
-              failed = true;
-              break;
-            }
-          }
-          if (failed) break;
-          asm volatile("fence.proxy.async.global;" ::: "memory");   // acquire (generic) before the TMA loads (async proxy)
-        }
+    // Lane 0 issues the loads; the whole warp walks the tile list so that, for a second-layer tile, 32 lanes can read
+    // the counters of the row block's first-layer tiles in one round trip.
+    int stage = 0;
+    uint32_t phase = 0;
+    const uint32_t leader_full = leader ? bar_full : mapa_shared(bar_full, 0);
+    // the value a tile's counter reaches in this launch: completed launches are counted on the device;
+    // 2 = one announcement by each of the two CTAs
+    const unsigned long long tile_target = p.ready ? (f2_ld_acquire(p.ready) + 1ULL) * 2ULL : 0ULL;
+    for (int i = 0; i < list_len; ++i) {
+      const int e = entry(i);
+      if (e < 0) break;
+      const int l = e >> 24, tile = e & 0xFFFFFF;
+      const int n_tiles = p.L[l].n_tiles, nkb = p.L[l].num_k_blocks;
+      const int m_pair = tile / n_tiles, n_blk = tile % n_tiles;
+      const int m_blk = m_pair * 2 + static_cast<int>(rank);
+      // The 256 hidden rows a second-layer tile reads are written by the first-layer tiles of its row block, 256
+      // hidden columns (K_PER_TILE k-blocks) each.  known: bit j set = tile j's stores have completed.
+      uint32_t known = 0xFFFFFFFFu;
+      const unsigned long long* tile_ready = nullptr;
+      if (l == 1) {
+        tile_ready = p.ready + 2 + static_cast<int64_t>(m_pair) * p.L[0].n_tiles;
+        const bool ok = lane >= p.L[0].n_tiles || f2_ld_acquire(tile_ready + lane) >= tile_target;
+        known = __ballot_sync(0xFFFFFFFFu, ok);
+      }
+      if (lane == 0) {
+        if (l == 1) asm volatile("fence.proxy.async.global;" ::: "memory");   // acquire (generic) before the TMA loads (async proxy)
         const CUtensorMap* tmA = &p.tm[3 * l];
         const CUtensorMap* tmB = &p.tm[3 * l + 1];
         for (int kb = 0; kb < nkb; ++kb) {
+          if (l == 1 && kb % K_PER_TILE == 0) {
+            const int j = kb / K_PER_TILE;
+            if (j < p.L[0].n_tiles && (j >= 32 || !((known >> j) & 1u))) {
+              const uint64_t t0 = globaltimer_ns();
+              uint32_t spins = 0;
+              while (f2_ld_acquire(tile_ready + j) < tile_target) {
+                if ((++spins & 255u) == 0 && globaltimer_ns() - t0 > 2000000000ull) {
+                  report(p.status, DEV_TIMEOUT_PRODUCER);
+                  failed = true;
+                  break;
+                }
+              }
+              if (failed) break;
+              asm volatile("fence.proxy.async.global;" ::: "memory");
+            }
+          }
           if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1)) {
             report(p.status, DEV_TIMEOUT_PRODUCER);
             failed = true;
@@ -169,6 +191,8 @@ __global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_co
           }
         }
       }
+      failed = __shfl_sync(0xFFFFFFFFu, failed ? 1 : 0, 0) != 0;
+      if (failed) break;
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader only)
@@ -213,7 +237,7 @@ __global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_co
         if (acc == 0) acc_phase ^= 1;
       }
     }
-  } else {
+  } else if (warp < 2 + F2_EPI_WARPS) {
     // ------------------------------------------------------------------ epilogue warps (both CTAs)
     const int ew = warp - 2;
     const int q = warp & 3;
@@ -225,6 +249,22 @@ __global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_co
     float* my_bias = bias_smem + ew * F2_BLOCK_N;
     const uint32_t row_off = (lane >> 3) * 1024 + (lane & 7) * 128;
     const uint32_t leader_tempty = leader ? bar_tempty : mapa_shared(bar_tempty, 0);
+    // A first-layer tile is announced to the other clusters once the stores of all 8 epilogue warps have COMPLETED.
+    // Each warp tells the announcer warp (an mbarrier arrival, cheap) when its own stores of the tile have; the
+    // announcer then performs the one releasing reduction per CTA and tile (a release at GPU scope costs
+    // 1300-2000 clocks here: far too much for the path of every epilogue warp).  Waiting for the stores right after
+    // a tile would put their latency on that path too, so a tile that is followed by another first-layer tile is
+    // reported at the end of that next tile, when all but the newest BOXES_PER_WARP bulk groups have long completed.
+    // The last first-layer tile of the list is reported at once: what follows it may wait for other clusters.
+    // Two barriers alternate: a warp is never two first-layer tiles ahead of another one at this point.
+    constexpr int BOXES_PER_WARP = NUM_BOXES / 2;
+    bool pending = false;
+    int n_first = 0;                                               // first-layer tiles reported so far
+    auto report_stores = [&]() {
+      asm volatile("fence.proxy.async.global;" ::: "memory");
+      mbar_arrive(bar_ann + 8 * (n_first & 1));
+      ++n_first;
+    };
     for (int i = 0; i < list_len; ++i) {
       const int e = entry(i);
       if (e < 0) break;
@@ -247,7 +287,7 @@ __global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_co
         __syncwarp();
         epi.bias = my_bias - n_blk * F2_BLOCK_N;                   // indexed by absolute column below
       }
-      if (!mbar_wait(bar_tfull + 8 * acc, acc_phase)) {
+      if (!mbar_wait_prompt(bar_tfull + 8 * acc, acc_phase)) {
         report(p.status, DEV_TIMEOUT_EPILOGUE);
         failed = true;
         break;
@@ -255,9 +295,6 @@ __global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_co
       tc_fence_after();
       const uint32_t t_row = tmem_base + acc * F2_BLOCK_N + (static_cast<uint32_t>(q * 32) << 16);
       for (int box = half; box < NUM_BOXES; box += 2) {
-        // the previous store out of this warp's staging buffer must have read it completely
-        if (lane == 0) tma_store_wait_read<0>();
-        __syncwarp();
 #pragma unroll 1
         for (int sub = 0; sub < BOX_COLS / 32; ++sub) {
           uint32_t r[32];
@@ -266,6 +303,12 @@ __global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_co
           constexpr int NW = 32 * OUT_BYTES / 4;
           uint32_t w[NW];
           epi_chunk32<KIND, OUT>(r, w, n_blk * F2_BLOCK_N + box * BOX_COLS + sub * 32, N, epi);
+          if (sub == 0) {
+            // the previous store out of this warp's staging buffer must have read it completely (checked only
+            // now, with the first chunk's values already in registers)
+            if (lane == 0) tma_store_wait_read<0>();
+            __syncwarp();
+          }
           const int c0 = sub * (NW / 4);
 #pragma unroll
           for (int j = 0; j < NW / 4; ++j)
@@ -282,22 +325,46 @@ __global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_co
       tc_fence_before();
       __syncwarp();
       if (lane == 0) {
+        if (pending) {
+          tma_store_wait_all<BOXES_PER_WARP>();                   // everything but this tile's own stores
+          report_stores();
+          pending = false;
+        }
         if (leader) mbar_arrive(bar_tempty + 8 * acc);
-        else mbar_arrive_cluster(leader_tempty + 8 * acc);
+        else mbar_arrive_cluster_nomem(leader_tempty + 8 * acc);
         if (l == 0 && p.ready) {
           // my part of the hidden row block is in memory once my stores have completed (not merely been read)
-          tma_store_wait_all<0>();
-          asm volatile("fence.proxy.async.global;" ::: "memory");
-          asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p.ready + m_pair), "l"(1ULL) : "memory");
+          const int e2 = i + 1 < list_len ? entry(i + 1) : -1;
+          if (e2 >= 0 && (e2 >> 24) == 0) {
+            pending = true;
+          } else {
+            tma_store_wait_all<0>();
+            report_stores();
+          }
         }
       }
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1;
     }
     if (lane == 0) tma_store_wait_all<0>();
+  } else if (p.ready && lane == 0) {
+    // ------------------------------------------------------------------ announcer (both CTAs)
+    int n_first = 0;
+    for (int i = 0; i < list_len; ++i) {
+      const int e = entry(i);
+      if (e < 0) break;
+      if ((e >> 24) != 0) continue;
+      if (!mbar_wait(bar_ann + 8 * (n_first & 1), (n_first >> 1) & 1)) {
+        report(p.status, DEV_TIMEOUT_OTHER);
+        break;
+      }
+      ++n_first;
+      asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p.ready + 2 + (e & 0xFFFFFF)), "l"(1ULL) : "memory");
+    }
   }
 
   // ---------------------------------------------------------------------- teardown
+  __syncwarp();                                                   // single-lane roles: reconverge before the aligned barrier
   tc_fence_before();
   cluster_sync_all();                                             // the peer no longer reads this CTA's smem
   if (warp == 1) {
@@ -306,11 +373,11 @@ __global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_co
   }
   // the last CTA to get here closes the launch (see GemmPairParams::ready)
   if (p.ready && threadIdx.x == 0) {
-    const unsigned long long prev = atomicAdd(p.ready + p.m_pairs + 1, 1ULL);
+    const unsigned long long prev = atomicAdd(p.ready + 1, 1ULL);
     if (prev + 1 == gridDim.x) {
-      atomicExch(p.ready + p.m_pairs + 1, 0ULL);
+      atomicExch(p.ready + 1, 0ULL);
       __threadfence();
-      atomicAdd(p.ready + p.m_pairs, 1ULL);
+      atomicAdd(p.ready, 1ULL);
     }
   }
   if (failed) {
