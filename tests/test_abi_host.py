@@ -141,3 +141,23 @@ def test_per_channel_scales_and_zero_points_plan_on_tensor_cores_and_bad_uses_ar
     with pytest.raises(B.GcError) as e:
         B.gc_partition_create(w.graph)
     assert e.value.status == B.GC_ERR_INVALID_ARG
+
+
+def test_tile_schedules_of_the_two_layer_launch_over_a_range_of_shapes():
+    # host logic only: the scheduler simulates the step and must never produce a list much longer than a perfect split
+    # of the work when there is plenty of it, and must not fuse when a layer is too small for CTA pairs
+    import re
+    for tokens, d_model, d_ff, fused in [(8192, 1024, 4096, True), (16384, 1024, 4096, True), (8192, 2048, 8192, True),
+                                         (9500, 512, 1008, True), (4900, 1024, 1024, True), (8192, 1024, 1024, True),
+                                         (2048, 1024, 4096, False), (6400, 512, 1008, False)]:
+        c = plan(W.ffn_bf16(tokens=tokens, d_model=d_model, d_ff=d_ff).graph)
+        m = re.search(r"one launch, (\d+) clusters, .*longest list (\d+) of ([\d.]+) k-blocks ideal", c.plan)
+        assert (m is not None) == fused, (tokens, d_model, d_ff, c.plan)
+        if not fused:
+            assert c.launches == 2
+            continue
+        assert c.launches == 1
+        longest, ideal = int(m.group(2)), float(m.group(3))
+        assert longest >= ideal
+        if ideal >= 200:
+            assert longest <= 1.03 * ideal, (tokens, d_model, d_ff, longest, ideal)

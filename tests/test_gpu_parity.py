@@ -202,6 +202,22 @@ def test_two_large_layers_in_one_launch_bf16(B):
     assert np.array_equal(sep, got[0])                   # same tiles, same arithmetic: identical bits
 
 
+def test_two_large_layers_in_one_launch_ragged_hidden_width(B):
+    # hidden width 1008: the fourth 256-column tile of the first layer is clipped and the second layer's last group of
+    # k-blocks is partly padding; 75 row tiles: the last pair is half empty.  bf16 (4 k-blocks per first-layer tile)
+    # and tf32 (8 per tile).
+    w = W.ffn_bf16(tokens=9500, d_model=512, d_ff=1008)
+    got, plan = run_gpu(B, w, n_runs=2)
+    assert "one launch" in plan
+    assert np.array_equal(got[0], got[1])
+    assert np.abs(bf16_to_f64(got[0]) - oracle(w)).max() <= 2e-2
+    w = W.mlp_f32(batch=9500, dims=(256, 1008, 512), seed=4)
+    got, plan = run_gpu(B, w)
+    assert "one launch" in plan
+    ref = oracle(w)
+    assert np.abs(got.astype(np.float64) - ref).max() <= 5e-3 * np.abs(ref).max()
+
+
 def test_two_large_layers_in_one_launch_int8_bit_exact(B):
     w = W.mlp_int8(batch=4900, dims=(1024, 1024, 1024, 16), final="none", per_channel=True, x_zp=9, act_zp=4)
     got, plan = run_gpu(B, w)
