@@ -203,6 +203,43 @@ def sweep_cases():
     return cases
 
 
+def run_plain_gemm(B, device, peaks):
+    """A plain 8192^3 bf16 GEMM through the same library, timed the way the measured cuBLAS peaks were (best of 10
+    single calls; back-to-back calls for about 3 s), next to those peaks: how the GEMM kernel alone compares."""
+    import torch
+    w = W.plain_gemm_bf16()
+    r = Replica(B, w, 0, device)
+    stream = torch.cuda.current_stream(device).cuda_stream
+    for _ in range(3):
+        r.step(stream)
+    torch.cuda.synchronize(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    best = 1e30
+    for _ in range(10):
+        e0.record()
+        r.step(stream)
+        e1.record()
+        torch.cuda.synchronize(device)
+        best = min(best, e0.elapsed_time(e1))
+    time.sleep(2.0)
+    n = int(3000.0 / best)
+    e0.record()
+    for _ in range(n):
+        r.step(stream)
+    e1.record()
+    torch.cuda.synchronize(device)
+    sustained = e0.elapsed_time(e1) / n
+    r.c.query_status()
+    out = {"graph": w.name, "kernel": r.c.plan.strip().splitlines()[-1].strip(), "burst_us": best * 1e3,
+           "burst_tflops": w.ops / (best * 1e-3) / 1e12, "sustained_us": sustained * 1e3, "sustained_calls": n,
+           "sustained_tflops": w.ops / (sustained * 1e-3) / 1e12,
+           "measured_library_peak_tflops": {"burst": peaks.get("bf16_tflops"), "sustained": peaks.get("bf16_tflops_sustained")}}
+    out["frac_of_burst_peak"] = out["burst_tflops"] / peaks["bf16_tflops"]
+    out["frac_of_sustained_peak"] = out["sustained_tflops"] / peaks["bf16_tflops_sustained"]
+    r.c.close()
+    return out
+
+
 def run_sweep(B, device, peaks, only=""):
     """One line per shape: cold time (rotating replicas above the L2 size), kernels chosen, HBM-roofline time."""
     import torch
@@ -348,6 +385,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the headline run, time every shape of the evaluation's workload table (1 GPU)")
+    ap.add_argument("--gemm", action="store_true",
+                    help="instead of the benchmark: one plain 8192^3 bf16 GEMM, timed like the measured library peaks")
     ap.add_argument("--sweep-filter", default="", help="with --sweep: only the cases whose name contains this text")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -384,6 +423,13 @@ def main():
         return float(t.item())
 
     peaks, peak_src = load_peaks()
+    if args.gemm:
+        if rank == 0:
+            print(json.dumps({"plain_gemm": run_plain_gemm(B, local, peaks), "data": "synthetic"}))
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
     if args.sweep:
         if rank == 0:
             print(json.dumps({"sweep": run_sweep(B, local, peaks, args.sweep_filter), "unit": "us per subgraph, cold L2", "data": "synthetic"}))

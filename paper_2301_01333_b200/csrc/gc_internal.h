@@ -92,6 +92,7 @@ struct GemmPairParams {
   const int* sched;               // [clusters][sched_pitch]: (layer << 24) | tile, a negative entry ends a list;
   int sched_pitch;                // null: one layer whose implicit_tiles tiles the clusters take round robin
   int implicit_tiles;
+  int m_pairs, raster_rows;       // one layer: 256-row blocks in all, and how many of them form a group of the tile order
   unsigned long long* ready;      // null for one layer.  [0] = launches completed so far (the epoch: bumped by the
                                   // last CTA to finish; keeping it on the device, not in the launch parameters, is
                                   // what makes a captured launch replayable), [1] = CTAs finished in this launch,

@@ -126,6 +126,22 @@ __global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_co
     const int t = cluster_id + i * num_clusters;
     return t < p.implicit_tiles ? t : -1;
   };
+  // tile number -> (256-row block, 256-column tile).  Scheduled launches number the tiles row block by row block.
+  // Without a schedule, row blocks are taken in groups of p.raster_rows and a group is walked column by column, so
+  // that the clusters working at the same time share a few row blocks of A and a few column tiles of the weights
+  // (both stay in L2) instead of sweeping the whole weight matrix once per round.
+  auto decode = [&](int tile, int n_tiles, int& m_pair, int& n_blk) {
+    if (sched || p.raster_rows <= 1) {
+      m_pair = tile / n_tiles;
+      n_blk = tile % n_tiles;
+      return;
+    }
+    const int per_group = p.raster_rows * n_tiles;
+    const int g = tile / per_group, r = tile - g * per_group;
+    const int rows = min(p.raster_rows, p.m_pairs - g * p.raster_rows);   // the last group may be shorter
+    n_blk = r / rows;
+    m_pair = g * p.raster_rows + r - n_blk * rows;
+  };
   bool failed = false;
 
   if (warp == 0) {
@@ -143,7 +159,8 @@ __global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_co
       if (e < 0) break;
       const int l = e >> 24, tile = e & 0xFFFFFF;
       const int n_tiles = p.L[l].n_tiles, nkb = p.L[l].num_k_blocks;
-      const int m_pair = tile / n_tiles, n_blk = tile % n_tiles;
+      int m_pair, n_blk;
+      decode(tile, n_tiles, m_pair, n_blk);
       const int m_blk = m_pair * 2 + static_cast<int>(rank);
       // The 256 hidden rows a second-layer tile reads are written by the first-layer tiles of its row block, 256
       // hidden columns (K_PER_TILE k-blocks) each.  known: bit j set = tile j's stores have completed.
@@ -270,7 +287,8 @@ __global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_co
       if (e < 0) break;
       const int l = e >> 24, tile = e & 0xFFFFFF;
       const int n_tiles = p.L[l].n_tiles, N = p.L[l].N;
-      const int m_pair = tile / n_tiles, n_blk = tile % n_tiles;
+      int m_pair, n_blk;
+      decode(tile, n_tiles, m_pair, n_blk);
       const int m_blk = m_pair * 2 + static_cast<int>(rank);
       const CUtensorMap* tmD = &p.tm[3 * l + 2];
       // Copy this tile's bias slice into shared memory while the accumulator is still being produced: a
@@ -438,6 +456,8 @@ cudaError_t launch_gemm_tc2(int kind, int a_signed, const CUtensorMap& tmA, cons
   p.L[0].n_tiles = g.n_tiles;
   p.L[0].epi = g.epi;
   p.implicit_tiles = ((g.m_tiles + 1) / 2) * g.n_tiles;
+  p.m_pairs = (g.m_tiles + 1) / 2;
+  p.raster_rows = 8;
   p.status = g.status;
   p.tm[0] = tmA;
   p.tm[1] = tmB;

@@ -161,6 +161,21 @@ def ffn_bf16(tokens: int = 8192, d_model: int = 1024, d_ff: int = 4096, seed: in
     return Workload(g.name, g, feeds).finish()
 
 
+def plain_gemm_bf16(m: int = 8192, k: int = 8192, n: int = 8192, seed: int = 0) -> Workload:
+    """One bf16 matmul with a bf16 result and nothing fused: the shape library GEMM peaks are quoted on."""
+    rng = np.random.default_rng(seed)
+    g = Graph(name=f"gemm_bf16_{m}x{k}x{n}")
+    feeds = {}
+    x = g.input("bf16", (m, k), name="x")
+    feeds[x] = f32_to_bf16_bits(rng.standard_normal((m, k), dtype=np.float32))
+    w = g.input("bf16", (k, n), is_constant=True, name="w")
+    feeds[w] = f32_to_bf16_bits(rng.standard_normal((k, n), dtype=np.float32) * np.float32(0.02))
+    z = g.op("matmul", (x, w), g.tensor("f32", (m, n)))
+    y = g.op("typecast", (z,), g.tensor("bf16", (m, n)))
+    g.mark_output(y)
+    return Workload(g.name, g, feeds).finish()
+
+
 # ------------------------------------------------------------------------------------------------
 # Scaled-dot-product attention blocks
 # ------------------------------------------------------------------------------------------------
