@@ -127,6 +127,9 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 26);
   // per slot and 32-key chunk: 1 = every key of the chunk is masked out, 2 = the chunk has an unmasked key, 0 = neither
   uint32_t* sChunk = tmem_slot + 4;                                       // [2 slots][16]
+  // per slot and group of 32 columns (g): bits 0-7 = key blocks up to the last one whose chunk g is not fully masked,
+  // bit 8 = the group has a chunk with an unmasked key
+  uint32_t* sTail = sChunk + 32;                                          // [2 slots][4]
   const uint32_t b0 = smem_u32(bars);
   const uint32_t bar_kv_full = b0, bar_kv_empty = b0 + 16, bar_kv_ready = b0 + 32;   // [2] each
   const uint32_t bar_s_full = b0 + 48, bar_s_free = b0 + 72, bar_p_full = b0 + 96;   // [3] each
@@ -429,6 +432,7 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         failed = true;
         break;
       }
+      uint32_t tail = 0;                                        // see sTail: this warp covers group (warp - 2) of every block
 #pragma unroll
       for (int i = 0; i < 3; ++i) {                             // a warp covers one aligned 32-key chunk per step
         const int j = t + 128 * i;
@@ -441,8 +445,11 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           // bit 2: all 32 keys of the chunk carry the same mask value, so the largest score is the largest accumulator
           const bool uniform = __all_sync(0xffffffffu, __float_as_uint(mv) == __shfl_sync(0xffffffffu, __float_as_uint(mv), 0));
           if (lane == 0) sChunk[s * 16 + (j >> 5)] = (all_masked ? 1u : (any_valid ? 2u : 0u)) | (uniform ? 4u : 0u);
+          if (!all_masked) tail = (tail & 0x100u) | static_cast<uint32_t>(i + 1);
+          if (any_valid && !all_masked) tail |= 0x100u;
         }
       }
+      if (INT8 && lane == 0) sTail[s * 4 + (warp - 2)] = tail;
       if (INT8 && !p.q_signed) {
         uint4* q4 = reinterpret_cast<uint4*>(slot_q(s));
         for (int i = t; i < L::q_bytes() / 16; i += 128) {
@@ -507,11 +514,10 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       // keeps the two passes free of per-chunk branches: they simply run over fewer blocks.
       int nbp = NB;                                             // my chunks of key blocks nbp .. NB-1 are skipped
       if constexpr (INT8) {
-        const uint32_t* fl = sChunk + s * 16;
-        bool any_valid = false;
-        for (int i = 0; i < NB * 4; ++i) any_valid = any_valid || (fl[i] & 3u) == 2u;
-        if (any_valid)
-          while (nbp > 0 && (fl[(nbp - 1) * 4 + g] & 3u) == 1u) --nbp;
+        const uint4 tl = *reinterpret_cast<const uint4*>(sTail + s * 4);   // prepared with the mask row
+        const bool any_valid = ((tl.x | tl.y | tl.z | tl.w) & 0x100u) != 0;
+        const uint32_t mine = g == 0 ? tl.x : (g == 1 ? tl.y : (g == 2 ? tl.z : tl.w));
+        if (any_valid) nbp = static_cast<int>(mine & 0xFFu);
       }
 
       // ---------------- pass A: one 32-column chunk per key block, transformed in place
