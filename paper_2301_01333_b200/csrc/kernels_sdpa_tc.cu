@@ -57,7 +57,7 @@ struct SdpaSmem {
   __host__ __device__ static constexpr int slot_bytes(int S) { return q_bytes() + 2 * kv_bytes(S); }
   __host__ __device__ static constexpr int total(int S, int slots, int nsb, int stage_out) {
     return slots * slot_bytes(S) + nsb * p_bytes(S) + (stage_out ? OUT_STAGING_BYTES : 0) + slots * S * 4 /*mask*/ +
-           24 * 128 * 4 /*row statistics*/ + 384 /*barriers, TMEM address, chunk flags*/;
+           24 * 128 * 4 /*row statistics*/ + 448 /*barriers, TMEM address, chunk flags*/;
   }
 };
 
@@ -130,10 +130,12 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   // per slot and group of 32 columns (g): bits 0-7 = key blocks up to the last one whose chunk g is not fully masked,
   // bit 8 = the group has a chunk with an unmasked key
   uint32_t* sTail = sChunk + 32;                                          // [2 slots][4]
+  // one barrier per TMEM lane quarter: the four softmax warps that share its rows exchange their row statistics
+  const uint32_t bar_xchg = smem_u32(sTail + 8);                          // [4]
   const uint32_t b0 = smem_u32(bars);
   const uint32_t bar_kv_full = b0, bar_kv_empty = b0 + 16, bar_kv_ready = b0 + 32;   // [2] each
   const uint32_t bar_s_full = b0 + 48, bar_s_free = b0 + 72, bar_p_full = b0 + 96;   // [3] each
-  const uint32_t bar_o_full = b0 + 120, bar_o_free = b0 + 136, bar_xchg = b0 + 152;  // [2], [2], [1]
+  const uint32_t bar_o_full = b0 + 120, bar_o_free = b0 + 136;                       // [2], [2]
   const uint32_t bar_st_ready = b0 + 160, bar_st_free = b0 + 176;                    // [2], [2]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -155,7 +157,7 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       mbar_init(bar_s_free + 8 * i, SDPA_SOFTMAX_WARPS);
       mbar_init(bar_p_full + 8 * i, SDPA_SOFTMAX_WARPS);
     }
-    mbar_init(bar_xchg, SDPA_SOFTMAX_WARPS);
+    for (int i = 0; i < 4; ++i) mbar_init(bar_xchg + 8 * i, SDPA_SOFTMAX_WARPS / 4);
     fence_mbar_init();
     tma_prefetch_desc(&tmQ);
     tma_prefetch_desc(&tmK);
@@ -493,8 +495,8 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 
     auto xchg_sync = [&]() -> bool {
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_xchg);
-      const bool ok = mbar_wait(bar_xchg, xphase);
+      if (lane == 0) mbar_arrive(bar_xchg + 8 * q);
+      const bool ok = mbar_wait(bar_xchg + 8 * q, xphase);
       xphase ^= 1;
       return ok;
     };
