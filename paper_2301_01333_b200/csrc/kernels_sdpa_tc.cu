@@ -130,8 +130,7 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   // per slot and group of 32 columns (g): bits 0-7 = key blocks up to the last one whose chunk g is not fully masked,
   // bit 8 = the group has a chunk with an unmasked key
   uint32_t* sTail = sChunk + 32;                                          // [2 slots][4]
-  // one barrier per TMEM lane quarter: the four softmax warps that share its rows exchange their row statistics
-  const uint32_t bar_xchg = smem_u32(sTail + 8);                          // [4]
+  const uint32_t bar_xchg = smem_u32(sTail + 8);                          // the softmax warps exchange row statistics
   const uint32_t b0 = smem_u32(bars);
   const uint32_t bar_kv_full = b0, bar_kv_empty = b0 + 16, bar_kv_ready = b0 + 32;   // [2] each
   const uint32_t bar_s_full = b0 + 48, bar_s_free = b0 + 72, bar_p_full = b0 + 96;   // [3] each
@@ -157,7 +156,7 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       mbar_init(bar_s_free + 8 * i, SDPA_SOFTMAX_WARPS);
       mbar_init(bar_p_full + 8 * i, SDPA_SOFTMAX_WARPS);
     }
-    for (int i = 0; i < 4; ++i) mbar_init(bar_xchg + 8 * i, SDPA_SOFTMAX_WARPS / 4);
+    mbar_init(bar_xchg, SDPA_SOFTMAX_WARPS);
     fence_mbar_init();
     tma_prefetch_desc(&tmQ);
     tma_prefetch_desc(&tmK);
@@ -495,8 +494,8 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 
     auto xchg_sync = [&]() -> bool {
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_xchg + 8 * q);
-      const bool ok = mbar_wait(bar_xchg + 8 * q, xphase);
+      if (lane == 0) mbar_arrive(bar_xchg);
+      const bool ok = mbar_wait(bar_xchg, xphase);
       xphase ^= 1;
       return ok;
     };

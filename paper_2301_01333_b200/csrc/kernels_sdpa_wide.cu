@@ -126,13 +126,17 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   uint64_t* bars = reinterpret_cast<uint64_t*>(sStat + 24 * 128);
   const uint32_t b0 = smem_u32(bars);
   const uint32_t bar_q_full = b0, bar_q_empty = b0 + 8, bar_q_ready = b0 + 16;
-  const uint32_t bar_o_full = b0 + 24, bar_o_free = b0 + 32, bar_xchg = b0 + 40;
+  const uint32_t bar_o_full = b0 + 24, bar_o_free = b0 + 32;
   const uint32_t bar_st_ready = b0 + 48, bar_st_free = b0 + 64;                      // [2] each
   const uint32_t bar_s_full = b0 + 80, bar_s_free = b0 + 112, bar_p_full = b0 + 144, bar_p_free = b0 + 176;   // [4] each
   const uint32_t bar_kv_full = b0 + 208, bar_kv_empty = b0 + 208 + 8 * W_MAX_STAGES;   // [16] each -> ends at 464
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 60);                      // byte 480
   // per mask buffer and 32-key chunk: 1 = every key masked out, 2 = has an unmasked key, 0 = neither
   uint32_t* sChunk = tmem_slot + 4;                                                  // [2][16], bytes 496..624
+  // per mask buffer and group of 32 columns (g): bits 0-7 = key blocks up to the last one whose chunk g is not fully
+  // masked, bit 8 = the group has a chunk with an unmasked key
+  uint32_t* sTail = sChunk + 32;                                                     // [2][4], bytes 624..656
+  const uint32_t bar_xchg = smem_u32(sTail + 8);                                     // bytes 656..664: row statistics exchange
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int q_tiles = S / W_BLOCK_Q;
@@ -426,6 +430,7 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         failed = true;
         break;
       }
+      uint32_t tail = 0;                                        // see sTail: this warp covers group (warp - 2) of every block
 #pragma unroll
       for (int i = 0; i < 4; ++i) {                             // a warp covers one aligned 32-key chunk per step
         const int j = t + 128 * i;
@@ -438,8 +443,11 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           // bit 2: all 32 keys of the chunk carry the same mask value, so the largest score is the largest accumulator
           const bool uniform = __all_sync(0xffffffffu, __float_as_uint(mv) == __shfl_sync(0xffffffffu, __float_as_uint(mv), 0));
           if (lane == 0) sChunk[(n & 1) * 16 + (j >> 5)] = (all_masked ? 1u : (any_valid ? 2u : 0u)) | (uniform ? 4u : 0u);
+          if (!all_masked) tail = (tail & 0x100u) | static_cast<uint32_t>(i + 1);
+          if (any_valid && !all_masked) tail |= 0x100u;
         }
       }
+      if (INT8 && lane == 0) sTail[(n & 1) * 4 + (warp - 2)] = tail;
       if (INT8 && !p.q_signed) {
         uint4* q4 = reinterpret_cast<uint4*>(sQ);
         for (int i = t; i < L::TILE_BYTES / 16; i += 128) {
@@ -493,11 +501,10 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       if (!mbar_wait(bar_q_ready, upar)) { failed = true; break; }
       int nbp = NB;                                             // my chunks of key blocks nbp .. NB-1 are skipped
       if constexpr (INT8) {
-        const uint32_t* fl = sChunk + (n & 1) * 16;
-        bool any_valid = false;
-        for (int i = 0; i < NB * 4; ++i) any_valid = any_valid || (fl[i] & 3u) == 2u;
-        if (any_valid)
-          while (nbp > 0 && (fl[(nbp - 1) * 4 + g] & 3u) == 1u) --nbp;
+        const uint4 tl = *reinterpret_cast<const uint4*>(sTail + (n & 1) * 4);   // prepared with the mask row
+        const bool any_valid = ((tl.x | tl.y | tl.z | tl.w) & 0x100u) != 0;
+        const uint32_t mine = g == 0 ? tl.x : (g == 1 ? tl.y : (g == 2 ? tl.z : tl.w));
+        if (any_valid) nbp = static_cast<int>(mine & 0xFFu);
       }
 
       // ---------------- pass A: scale + mask, running row max [int8: exp2 and running sum, written back]
