@@ -113,6 +113,21 @@ def test_cta_pair_gemm_bf16_with_epilogue(B):
     assert np.abs(bf16_to_f64(got) - oracle(w)).max() <= 2e-2
 
 
+def test_cta_pair_gemm_bf16_grouped_tile_order_sampled_rows(B):
+    # a plain GEMM large enough for the grouped tile order of the CTA-pair kernel: 20 row blocks of 256 = two full
+    # groups of eight and a short one, 16 column tiles; every row block is sampled, the last one is ragged
+    w = W.plain_gemm_bf16(5000, 1024, 4096, seed=5)
+    got, plan = run_gpu(B, w)
+    assert "cta_pair" in plan
+    rows = np.unique(np.concatenate([np.arange(0, 5000, 19), [127, 128, 255, 256, 2047, 2048, 4095, 4096, 4863, 4864, 4999]]))
+    sub = W.plain_gemm_bf16(len(rows), 1024, 4096, seed=5)
+    for a, b in zip(sub.graph.inputs, w.graph.inputs):
+        sub.feeds[a] = w.feeds[b][rows] if a == sub.graph.inputs[0] else w.feeds[b]
+    ref = oracle(sub)
+    assert np.abs(bf16_to_f64(got)[rows] - ref).max() <= 2e-2
+    assert np.isfinite(bf16_to_f64(got)).all()
+
+
 def test_batched_matmul_int8_exact(B):
     w = W.single_matmul("u8", "u8", 24, 16, 24, seed=3, transpose_b=True, a_zp=128, batch=(2, 3))
     w.graph.tensors[w.graph.inputs[1]].zero_point = 128
