@@ -469,8 +469,9 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
     tmem_dealloc(tmem_base, CH_NACC * CH_BLOCK_N);
   }
   // one more count per CTA on the way out (nobody waits for it): it keeps the counter a multiple of the per-launch
-  // total between launches, which the start-value computation above relies on
-  if (threadIdx.x == 0) asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p.barrier), "l"(1ULL) : "memory");
+  // total between launches, which the start-value computation above relies on.  Relaxed: the next launch reads the
+  // counter only after this one has completed, and a release here would hold the CTA back for over a thousand clocks.
+  if (threadIdx.x == 0) asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(p.barrier), "l"(1ULL) : "memory");
   // no CTA leaves while another one of its cluster may still write into its shared memory
   if (KS > 1) cluster_sync_all();
 }
