@@ -229,7 +229,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1;
     }
-    if (TMA_STORE && lane == 0) tma_store_wait_all<0>();
+    if (TMA_STORE && lane == 0) tma_store_wait_read<0>();   // (reads of the staging buffers, not completion: the stores complete with the kernel)
   }
 
   // ---------------------------------------------------------------------- teardown

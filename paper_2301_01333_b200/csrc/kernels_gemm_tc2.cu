@@ -364,7 +364,7 @@ __global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_co
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1;
     }
-    if (lane == 0) tma_store_wait_all<0>();
+    if (lane == 0) tma_store_wait_read<0>();   // (reads of the staging buffers, not completion: the stores complete with the kernel)
   } else if (p.ready && lane == 0) {
     // ------------------------------------------------------------------ announcer (both CTAs)
     int n_first = 0;

@@ -473,7 +473,7 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       report(p.status, DEV_TIMEOUT_OTHER);
       failed = true;
     }
-    if (lane == 0) tma_store_wait_all<0>();
+    if (lane == 0) tma_store_wait_read<0>();   // (reads of the staging buffers, not completion: the stores complete with the kernel)
   } else {
     // ------------------------------------------------------------------ softmax warps
     // Four threads share a query row (TMEM lane): warp w covers lane quarter (w % 4) and, of every 128-key
