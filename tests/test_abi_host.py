@@ -161,3 +161,21 @@ def test_tile_schedules_of_the_two_layer_launch_over_a_range_of_shapes():
         assert longest >= ideal
         if ideal >= 200:
             assert longest <= 1.03 * ideal, (tokens, d_model, d_ff, longest, ideal)
+
+
+def test_reference_arm_of_the_bench_prints_the_contract_line_without_a_gpu():
+    # `bench.py --impl reference` times the oracle on the host cores: no GPU, one JSON line with the contract's keys
+    import json
+    import subprocess
+    import sys
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1", "--warmup", "1",
+                        "--workload", "c1"], capture_output=True, text=True, timeout=600, cwd=ROOT)
+    assert r.returncode == 0, r.stderr[-2000:]
+    line = json.loads(r.stdout.strip().splitlines()[-1])
+    for key in ("impl", "metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
+                "vs_baseline", "dtype", "data", "config", "cpu_baseline", "e2e"):
+        assert key in line, key
+    assert line["impl"] == "reference" and line["steps"] == 1 and line["value"] > 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
+    assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
+    assert line["config"]["workload"] == "c1"
