@@ -125,7 +125,11 @@ typedef struct {
   int32_t streaming_attention; /* 1: attention always runs on the streaming tcgen05 kernel (K/V and P rings),
                              also for the shapes (head dimension 64, up to 384 keys) that by default use the
                              kernel with resident K/V (ablation) */
-  int32_t reserved[5];
+  int32_t exact_max_softmax;   /* 1: the softmax always subtracts the row maximum.  By default an 8-bit attention
+                             block without a mask whose scores are bounded at compile time (|score| * log2(e) <= 60,
+                             from the operand ranges and the folded scales) skips it: the "fast softmax" of
+                             Section VII, equal in exact arithmetic (ablation) */
+  int32_t reserved[4];
 } gc_compile_options_t;
 
 typedef struct gc_partition gc_partition_t;

@@ -642,8 +642,13 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
     c->sdpa.use_tc = tc;
     c->sdpa.wide = tc && wide;
     c->launches = 1;
-    snprintf(line, sizeof(line), "pattern=attention %s B=%d H=%d S=%d D=%d kernel=%s\n", s.is_int8 ? "int8" : "bf16", s.B,
-             s.H, s.S, s.D, tc ? (wide ? "tcgen05.streaming" : "tcgen05") : "cuda-core");
+    // The paper's max-free softmax, where it is safe: 8-bit operands bound every score at compile time; with
+    // |score| log2(e) <= 60 neither an exponential nor a row sum can leave fp32's range, and without a mask no row
+    // can be pushed out of it at run time.  skip_thr = 2 bound + 151 (see match_sdpa).
+    s.max_free = tc && !wide && s.is_int8 && c->sdpa.mask_input < 0 && !c->opt.exact_max_softmax && s.skip_thr > 0.f &&
+                 (static_cast<double>(s.skip_thr) - 151.0) * 0.5 <= 60.0;
+    snprintf(line, sizeof(line), "pattern=attention %s B=%d H=%d S=%d D=%d kernel=%s%s\n", s.is_int8 ? "int8" : "bf16", s.B,
+             s.H, s.S, s.D, tc ? (wide ? "tcgen05.streaming" : "tcgen05") : "cuda-core", s.max_free ? " softmax=max-free" : "");
     c->desc = line;
   } else {
     gc_status_t st = match_mlp(*p, *c);

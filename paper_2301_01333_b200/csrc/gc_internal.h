@@ -78,6 +78,8 @@ struct SdpaParams {
   float skip_thr;      // int8: a 32-key chunk whose mask values times log2(e) are all <= -skip_thr contributes exactly
                        // zero to the softmax of any row that has an unmasked key (bound derived from the largest
                        // possible integer score); 0 disables the skipping of such chunks
+  int max_free;        // int8, no mask, scores bounded at compile time: exponentials without a row maximum (Section VII's
+                       // "fast softmax"); only the kernel for 64-wide heads with resident K/V implements it
   uint32_t* status;
 };
 

@@ -219,7 +219,7 @@ def mha_bf16(batch: int = 32, heads: int = 12, seq: int = 128, head_dim: int = 6
 def mha_int8(batch: int = 64, heads: int = 16, seq: int = 384, head_dim: int = 64, seed: int = 0,
              s_qkv: float = 0.03, zp_qkv: int = 128, s_out: float = 0.02, zp_out: int = 128,
              valid_lo: int | None = None, valid_hi: int | None = None,
-             all_value: int | None = None) -> Workload:
+             all_value: int | None = None, with_mask: bool = True) -> Workload:
     """int8 attention block (config 4 at the defaults): u8 Q, K, V (zero point 128), exact s32
     Q.K^T, dequantize, x 1/sqrt(d), + mask, softmax, probabilities quantised to u8 (scale
     1/255), exact s32 P.V, dequantize, requantize to u8."""
@@ -235,17 +235,19 @@ def mha_int8(batch: int = 64, heads: int = 16, seq: int = 384, head_dim: int = 6
             feeds[t] = rng.integers(0, 256, size=shp, dtype=np.int64).astype(np.uint8)
         else:
             feeds[t] = np.full(shp, all_value, dtype=np.uint8)
-    mask = g.input("f32", (batch, 1, 1, seq), name="mask")
     lo = seq // 2 if valid_lo is None else valid_lo
     hi = seq if valid_hi is None else valid_hi
     valid = rng.integers(lo, hi + 1, size=(batch,))
-    feeds[mask] = _mask_from_valid(valid, seq)
+    if with_mask:
+        mask = g.input("f32", (batch, 1, 1, seq), name="mask")
+        feeds[mask] = _mask_from_valid(valid, seq)
     sshape = (batch, heads, seq, seq)
     s_p = float(np.float32(1.0 / 255.0))
     a = g.op("matmul", (q, k), g.tensor("s32", sshape), transpose_b=True)
     s = g.op("dequantize", (a,), g.tensor("f32", sshape))
     s = g.op("mul", (s,), g.tensor("f32", sshape), scalar=float(1.0 / np.sqrt(head_dim)))
-    s = g.op("add", (s, mask), g.tensor("f32", sshape))
+    if with_mask:
+        s = g.op("add", (s, mask), g.tensor("f32", sshape))
     p = g.op("softmax", (s,), g.tensor("f32", sshape), axis=-1)
     pq = g.op("quantize", (p,), g.tensor("u8", sshape, scale=s_p, zero_point=0))
     a2 = g.op("matmul", (pq, v), g.tensor("s32", shp))

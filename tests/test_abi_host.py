@@ -179,3 +179,14 @@ def test_reference_arm_of_the_bench_prints_the_contract_line_without_a_gpu():
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
     assert line["config"]["workload"] == "c1"
+
+
+def test_max_free_softmax_is_planned_only_under_a_compile_time_score_bound():
+    # Section VII's fast softmax: 8-bit operands, no mask, |score| log2(e) <= 60 from the ranges and the folded scales
+    ok = plan(W.mha_int8(batch=2, heads=2, seq=384, s_qkv=0.01, with_mask=False).graph)
+    assert "softmax=max-free" in ok.plan
+    assert "max-free" not in plan(W.mha_int8(batch=2, heads=2, seq=384, s_qkv=0.01, with_mask=False).graph, exact_max_softmax=True).plan
+    assert "max-free" not in plan(W.mha_int8(batch=2, heads=2, seq=384, s_qkv=0.03, with_mask=False).graph).plan
+    assert "max-free" not in plan(W.mha_int8(batch=2, heads=2, seq=384, s_qkv=0.01).graph).plan          # masked
+    assert "max-free" not in plan(W.mha_int8(batch=2, heads=2, seq=512, s_qkv=0.01, with_mask=False).graph).plan   # streaming kernel
+    assert "max-free" not in plan(W.mha_bf16(batch=2, heads=2, seq=128).graph).plan

@@ -492,6 +492,26 @@ def test_mha_int8_reduced(B, b, h, s, d, generic):
     check_int8_attention(got, oracle(w))
 
 
+@pytest.mark.parametrize("s", [128, 384])
+def test_mha_int8_max_free_softmax(B, s):
+    # 8-bit attention without a mask and with scales small enough that every score is bounded at compile time
+    # (|score| log2(e) <= 60): the planner picks the max-free softmax (Section VII); same results as with the row
+    # maximum (the option switches it off), both within the int8 bar of the oracle
+    w = W.mha_int8(batch=2, heads=3, seq=s, head_dim=64, s_qkv=0.012, with_mask=False, seed=7)
+    got, plan = run_gpu(B, w)
+    assert "softmax=max-free" in plan
+    ref = oracle(w)
+    check_int8_attention(got, ref)
+    exact, plan2 = run_gpu(B, w, exact_max_softmax=True)
+    assert "max-free" not in plan2
+    check_int8_attention(exact, ref)
+    assert (np.abs(got.astype(np.int64) - exact.astype(np.int64)) <= 1).all()
+    # larger scales or a mask: the bound does not hold, the row maximum stays
+    for kw in (dict(s_qkv=0.03, with_mask=False), dict(s_qkv=0.012, with_mask=True)):
+        w2 = W.mha_int8(batch=1, heads=1, seq=s, head_dim=64, **kw)
+        assert "max-free" not in B.CompiledPartition(w2.graph, 0).plan
+
+
 def test_mha_int8_masked_chunk_skipping_edge_cases(B):
     # the tcgen05 kernel leaves out 32-key chunks whose keys are all masked; rows must not notice.  Batches:
     # everything masked (no skipping allowed: the mask then cancels in the softmax), one valid key, a valid
