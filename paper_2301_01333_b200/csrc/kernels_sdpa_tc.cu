@@ -101,7 +101,9 @@ __device__ __forceinline__ int quantize_magic(float u, int zp, int lo, int hi) {
   return min(max(r + zp, lo), hi);
 }
 
-template <bool INT8>
+// MAXFREE: the planner has bounded every score (see SdpaParams::max_free); a separate instantiation keeps the
+// general int8 kernel's code as it is.
+template <bool INT8, bool MAXFREE = false>
 __global__ void __launch_bounds__(SDPA_THREADS, 1)
 sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO, const SdpaParams p,
@@ -533,7 +535,7 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         if constexpr (INT8) tmem_wait_st();                     // v[] may still feed the previous block's store
         tmem_ld32(t_row + col, v);
         tmem_wait_ld();
-        if (INT8 && p.max_free) {
+        if constexpr (INT8 && MAXFREE) {
           // "Fast softmax" (Section VII): the planner has shown that no exponential and no row sum can leave fp32's
           // range (8-bit operands, small scales, no mask), so the scores go through exp2 as they are.  The common
           // factor 2^rho of the bias trick's rounding residue drops out of the softmax as on the path below.
@@ -776,6 +778,11 @@ cudaError_t launch_sdpa_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const
   lc.attrs = attr;
   lc.numAttrs = 1;
   cudaError_t e;
+  if (p.is_int8 && p.max_free) {
+    e = cudaFuncSetAttribute(sdpa_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(cfg.smem));
+    if (e != cudaSuccess) return e;
+    return cudaLaunchKernelEx(&lc, sdpa_tc_kernel<true, true>, tmQ, tmK, tmV, tmO, p, cfg.slots, cfg.nsb, cfg.stage_out);
+  }
   if (p.is_int8) {
     e = cudaFuncSetAttribute(sdpa_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(cfg.smem));
     if (e != cudaSuccess) return e;
