@@ -103,11 +103,17 @@ __device__ __forceinline__ int quantize_magic(float u, int zp, int lo, int hi) {
 
 // MAXFREE: the planner has bounded every score (see SdpaParams::max_free); a separate instantiation keeps the
 // general int8 kernel's code as it is.
-template <bool INT8, bool MAXFREE = false>
+// S_CT / CFG: sequence length and buffer configuration (100 slots + 10 score buffers + staged outputs) as
+// compile-time constants; S_CT = 0: both at run time.  With them the per-block loops unroll and the buffer
+// bookkeeping folds away: 112 -> 98 µs on the 384-key int8 benchmark shape, 11.8 -> 10.5 µs on the 128-key bf16 one.
+template <bool INT8, bool MAXFREE = false, int S_CT = 0, int CFG = 0>
 __global__ void __launch_bounds__(SDPA_THREADS, 1)
 sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO, const SdpaParams p,
-               const int slots, const int nsb, const int stage_out) {
+               const int slots_rt, const int nsb_rt, const int stage_out_rt) {
+  const int slots = S_CT ? CFG / 100 : slots_rt;
+  const int nsb = S_CT ? (CFG / 10) % 10 : nsb_rt;
+  const int stage_out = S_CT ? CFG % 10 : stage_out_rt;
   using L = SdpaSmem<INT8>;
   constexpr int ROW_BYTES = L::ROW_BYTES;
   constexpr uint32_t SWZ = INT8 ? SWZ_64B : SWZ_128B;
@@ -115,7 +121,7 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   constexpr int P_BLOCK_BYTES = SDPA_BLOCK_Q * 128 * L::ESZ;    // one 128-key block of P
   constexpr uint32_t TMEM_COLS = 512;
 
-  const int S = p.S;
+  const int S = S_CT ? S_CT : p.S;
   const int NB = S / 128;                                       // key blocks
   const int BUF_COLS = S + SDPA_D;                              // TMEM columns per (S, O) buffer
   extern __shared__ uint8_t smem_raw[];
@@ -777,20 +783,29 @@ cudaError_t launch_sdpa_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = attr;
   lc.numAttrs = 1;
-  cudaError_t e;
-  if (p.is_int8 && p.max_free) {
-    e = cudaFuncSetAttribute(sdpa_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(cfg.smem));
+  const int code = cfg.slots * 100 + cfg.nsb * 10 + cfg.stage_out;
+  auto go = [&](auto kern) -> cudaError_t {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(cfg.smem));
     if (e != cudaSuccess) return e;
-    return cudaLaunchKernelEx(&lc, sdpa_tc_kernel<true, true>, tmQ, tmK, tmV, tmO, p, cfg.slots, cfg.nsb, cfg.stage_out);
-  }
-  if (p.is_int8) {
-    e = cudaFuncSetAttribute(sdpa_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(cfg.smem));
-    if (e != cudaSuccess) return e;
-    return cudaLaunchKernelEx(&lc, sdpa_tc_kernel<true>, tmQ, tmK, tmV, tmO, p, cfg.slots, cfg.nsb, cfg.stage_out);
-  }
-  e = cudaFuncSetAttribute(sdpa_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(cfg.smem));
-  if (e != cudaSuccess) return e;
-  return cudaLaunchKernelEx(&lc, sdpa_tc_kernel<false>, tmQ, tmK, tmV, tmO, p, cfg.slots, cfg.nsb, cfg.stage_out);
+    return cudaLaunchKernelEx(&lc, kern, tmQ, tmK, tmV, tmO, p, cfg.slots, cfg.nsb, cfg.stage_out);
+  };
+  // the shapes the resident-K/V kernel takes, each with the configuration sdpa_cfg gives it: compile-time variants
+#define GC_SDPA_CASE(I8, MF, S_, C_) \
+  if (static_cast<bool>(p.is_int8) == I8 && static_cast<bool>(p.max_free) == MF && p.S == S_ && code == C_) \
+    return go(sdpa_tc_kernel<I8, MF, S_, C_>);
+  GC_SDPA_CASE(true, false, 128, 221)
+  GC_SDPA_CASE(true, false, 256, 211)
+  GC_SDPA_CASE(true, false, 384, 211)
+  GC_SDPA_CASE(true, true, 128, 221)
+  GC_SDPA_CASE(true, true, 256, 211)
+  GC_SDPA_CASE(true, true, 384, 211)
+  GC_SDPA_CASE(false, false, 128, 221)
+  GC_SDPA_CASE(false, false, 256, 111)
+  GC_SDPA_CASE(false, false, 384, 110)
+#undef GC_SDPA_CASE
+  if (p.is_int8 && p.max_free) return go(sdpa_tc_kernel<true, true>);
+  if (p.is_int8) return go(sdpa_tc_kernel<true>);
+  return go(sdpa_tc_kernel<false>);
 }
 
 }  // namespace gc
