@@ -65,7 +65,7 @@ struct WideCfg {
 };
 
 template <bool INT8, int D>
-WideCfg wide_cfg_t(int S) {
+constexpr WideCfg wide_cfg_t(int S) {
   using L = WideLayout<INT8, D>;
   const int NB = S / 128;
   const long limit = 227 * 1024;
@@ -105,14 +105,18 @@ __device__ __forceinline__ float w_ex2(float x) {
 // exact (float)a for |a| < 2^22 without a conversion instruction
 __device__ __forceinline__ float w_int_to_float(int a) { return __int_as_float(a + W_MAGIC_I) - W_MAGIC_F; }
 
-template <bool INT8, int D>
+// NB_CT, NP_CT, ST_CT: key blocks and ring sizes as compile-time constants (the launcher instantiates every
+// sequence length the kernel takes); with them the per-block loops unroll and the ring bookkeeping folds away.
+template <bool INT8, int D, int NB_CT, int NP_CT, int ST_CT>
 __global__ void __launch_bounds__(W_THREADS, 1)
 sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                 const __grid_constant__ CUtensorMap tmV, const SdpaParams p, const int np, const int stages) {
+                 const __grid_constant__ CUtensorMap tmV, const SdpaParams p) {
   using L = WideLayout<INT8, D>;
   constexpr uint32_t TMEM_COLS = 512;
-  const int S = p.S;
-  const int NB = S / 128;
+  constexpr int S = NB_CT * 128;
+  constexpr int NB = NB_CT;
+  constexpr int np = NP_CT;
+  constexpr int stages = ST_CT;
   const bool alias = S + D > 512;                               // O takes over the columns of score block 0
   const uint32_t o_col = alias ? 0u : static_cast<uint32_t>(S);
 
@@ -742,27 +746,43 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   }
 }
 
+template <bool INT8, int D, int NB>
+cudaError_t launch_wide_nb(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const SdpaParams& p,
+                           int num_sms, cudaStream_t s) {
+  constexpr WideCfg cfg = wide_cfg_t<INT8, D>(NB * 128);
+  if constexpr (cfg.smem == 0) {
+    return cudaErrorInvalidValue;
+  } else {
+    auto kern = sdpa_wide_kernel<INT8, D, NB, cfg.np, cfg.stages>;
+    const int units = p.B * p.H * (p.S / W_BLOCK_Q);
+    const int grid = units < num_sms ? units : num_sms;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(cfg.smem));
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(grid);
+    lc.blockDim = dim3(W_THREADS);
+    lc.dynamicSmemBytes = cfg.smem;
+    lc.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    return cudaLaunchKernelEx(&lc, kern, tmQ, tmK, tmV, p);
+  }
+}
+
 template <bool INT8, int D>
 cudaError_t launch_wide_t(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const SdpaParams& p,
                           int num_sms, cudaStream_t s) {
-  const WideCfg cfg = wide_cfg_t<INT8, D>(p.S);
-  if (!cfg.smem) return cudaErrorInvalidValue;
-  const int units = p.B * p.H * (p.S / W_BLOCK_Q);
-  const int grid = units < num_sms ? units : num_sms;
-  cudaError_t e = cudaFuncSetAttribute(sdpa_wide_kernel<INT8, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(cfg.smem));
-  if (e != cudaSuccess) return e;
-  cudaLaunchConfig_t lc = {};
-  lc.gridDim = dim3(grid);
-  lc.blockDim = dim3(W_THREADS);
-  lc.dynamicSmemBytes = cfg.smem;
-  lc.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  lc.attrs = attr;
-  lc.numAttrs = 1;
-  return cudaLaunchKernelEx(&lc, sdpa_wide_kernel<INT8, D>, tmQ, tmK, tmV, p, cfg.np, cfg.stages);
+  if (p.S % 128 != 0) return cudaErrorInvalidValue;
+  switch (p.S / 128) {
+    case 1: return launch_wide_nb<INT8, D, 1>(tmQ, tmK, tmV, p, num_sms, s);
+    case 2: return launch_wide_nb<INT8, D, 2>(tmQ, tmK, tmV, p, num_sms, s);
+    case 3: return launch_wide_nb<INT8, D, 3>(tmQ, tmK, tmV, p, num_sms, s);
+    case 4: return launch_wide_nb<INT8, D, 4>(tmQ, tmK, tmV, p, num_sms, s);
+    default: return cudaErrorInvalidValue;
+  }
 }
 
 }  // namespace
