@@ -671,7 +671,7 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           const int c0 = g * 2;                                 // 16-byte chunk index inside the 128-byte row
           *reinterpret_cast<uint4*>(blk + (((c0 + 0) ^ (r & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
           *reinterpret_cast<uint4*>(blk + (((c0 + 1) ^ (r & 7)) * 16)) = make_uint4(w[4], w[5], w[6], w[7]);
-          if (p.P_out) {                                          // optional output: the codes the second MMA consumes
+          if (S_CT == 0 && p.P_out) {                             // optional output (run-time variant only): the codes the second MMA consumes
             const int64_t grow = static_cast<int64_t>(unit / q_tiles) * S + (unit % q_tiles) * SDPA_BLOCK_Q + r;
             uint4* po = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.P_out) + grow * S + col);
             po[0] = make_uint4(w[0], w[1], w[2], w[3]);
@@ -729,7 +729,7 @@ sdpa_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           const int c0 = g * 2;
           *reinterpret_cast<uint4*>(blk + (((c0 + 0) ^ (r & 7)) * 16)) = make_uint4(0u, 0u, 0u, 0u);
           *reinterpret_cast<uint4*>(blk + (((c0 + 1) ^ (r & 7)) * 16)) = make_uint4(0u, 0u, 0u, 0u);
-          if (p.P_out) {
+          if (S_CT == 0 && p.P_out) {
             const int64_t grow = static_cast<int64_t>(unit / q_tiles) * S + (unit % q_tiles) * SDPA_BLOCK_Q + r;
             uint4* po = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.P_out) + grow * S + col);
             po[0] = make_uint4(0u, 0u, 0u, 0u);
@@ -791,7 +791,7 @@ cudaError_t launch_sdpa_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const
   };
   // the shapes the resident-K/V kernel takes, each with the configuration sdpa_cfg gives it: compile-time variants
 #define GC_SDPA_CASE(I8, MF, S_, C_) \
-  if (static_cast<bool>(p.is_int8) == I8 && static_cast<bool>(p.max_free) == MF && p.S == S_ && code == C_) \
+  if (static_cast<bool>(p.is_int8) == I8 && static_cast<bool>(p.max_free) == MF && p.S == S_ && code == C_ && !p.P_out) \
     return go(sdpa_tc_kernel<I8, MF, S_, C_>);
   GC_SDPA_CASE(true, false, 128, 221)
   GC_SDPA_CASE(true, false, 256, 211)
