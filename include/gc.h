@@ -95,7 +95,8 @@ typedef struct {
   float scale;            /* per-tensor quantisation scale; ignored for float dtypes */
   int32_t zero_point;
   int32_t is_constant;    /* 1: same pointer and contents on every execution (weights, biases) */
-  /* Per-channel quantisation (Section VII: "per channel s8 symmetric quantization for weight"): a HOST array
+  /* Per-channel quantisation (the weight scheme of Section VII's int8 evaluation: symmetric s8 weights with one
+   * scale per output channel): a HOST array
    * of dims[channel_axis] scales, copied by gc_partition_create; NULL = the per-tensor `scale` applies.
    * Accepted only on the constant s8 weight of a 2-D MatMul, along its output-channel axis (1 for a [k,n]
    * weight, 0 for a transposed [n,k] one); anything else is GC_ERR_UNSUPPORTED. */
@@ -155,13 +156,15 @@ gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, const gc_co
                        gc_compiled_t** out);
 void gc_compiled_destroy(gc_compiled_t* c);
 
-/* Scratch memory the compiled object needs (inter-layer activations, prepacked weights, padded
- * input copies, a status word).  The caller allocates it on the device (256-byte aligned), hands
- * it over once and keeps it alive until gc_compiled_destroy.  Contents need no initialisation. */
+/* Scratch memory the compiled object needs (Section VI: temporary buffers are sized, and reused
+ * between fused ops whose life spans do not overlap, at compile time; Section V: the preprocessed
+ * constant weights are kept for reuse): inter-layer activations, prepacked weights, padded input
+ * copies, a status word.  The caller allocates it on the device (256-byte aligned), hands it over
+ * once and keeps it alive until gc_compiled_destroy.  Contents need no initialisation. */
 gc_status_t gc_workspace_bytes(const gc_compiled_t* c, size_t* bytes);
 gc_status_t gc_set_workspace(gc_compiled_t* c, void* workspace_dev, size_t bytes);
 
-/* Execute (Section VII: "the compiled code only needs to be called once" per subgraph).  Enqueues
+/* Execute (Section VII: a subgraph costs one call into compiled code, not one per op).  Enqueues
  * all work on cuda_stream (a cudaStream_t, may be NULL for the default stream) and returns.  On
  * the first call, or when a constant input arrives at a new address, the constant weights are
  * prepacked on the same stream first and cached in the workspace (Section V).  A call that does
@@ -180,13 +183,14 @@ gc_status_t gc_set_host_staging(gc_compiled_t* c, void* staging_dev, size_t byte
 gc_status_t gc_execute_host(gc_compiled_t* c, void* cuda_stream, const void* const* in_host,
                             int32_t n_in, void* const* out_host, int32_t n_out);
 
-/* Synchronise the stream and read the device status word: GC_OK, GC_ERR_TIMEOUT (a bounded
- * device-side wait expired) or GC_ERR_CUDA (the stream reported an error). */
+/* No counterpart in the paper (its CPU kernels cannot time out).  Synchronise the stream and read
+ * the device status word: GC_OK, GC_ERR_TIMEOUT (a bounded device-side wait expired) or
+ * GC_ERR_CUDA (the stream reported an error). */
 gc_status_t gc_query_status(gc_compiled_t* c, void* cuda_stream);
 
-/* Introspection: number of kernel launches one gc_execute enqueues after prepacking, and a short
- * text description of the plan (pattern, per-layer kernel and tile).  The string is owned by the
- * compiled object. */
+/* No counterpart in the paper: introspection for tests and benchmarks.  Number of kernel launches
+ * one gc_execute enqueues after prepacking, and a short text description of the plan (pattern,
+ * per-layer kernel and tile).  The string is owned by the compiled object. */
 gc_status_t gc_launches_per_execute(const gc_compiled_t* c, int32_t* n);
 const char* gc_plan_description(const gc_compiled_t* c);
 

@@ -11,7 +11,7 @@ fused kernel must reproduce.
 
 Arithmetic domains
   * 8-bit x 8-bit MatMul: exact integers.  Operands have their zero point subtracted first
-    (asymmetric activations, Section V: "scales A ... then offset by a_z"); the sum is taken in
+    (asymmetric activations: Section V's dequantisation removes the zero point a_z); the sum is taken in
     int64 and checked to fit s32, which is the accumulator type of an int8 matmul.
   * Dequantize / Add / Mul / ReLU / Quantize applied to values that are exactly representable in
     fp32 (integer accumulators, fp32 graph inputs): IEEE fp32, one rounding per op, no fused

@@ -93,6 +93,51 @@ def test_requant_boundary_vectors_golden():
         assert got.tolist() == [r[2] for r in sel]
 
 
+def test_requant_boundary_vectors_signed_golden():
+    """tests/golden/requant_boundaries_s8.txt: the same rule with an s8 result - the range is [-128, 127],
+    both bounds are reachable without saturation, and ties go to even on the negative side too."""
+    rows = []
+    with open(os.path.join(GOLDEN, "requant_boundaries_s8.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                u, zp, q = line.split()
+                rows.append((float(u), int(zp), int(q)))
+    assert len(rows) >= 16 and min(r[2] for r in rows) == -128 and max(r[2] for r in rows) == 127
+    for zp in sorted({r[1] for r in rows}):
+        sel = [r for r in rows if r[1] == zp]
+        g = Graph()
+        x = g.input("f32", (len(sel),))
+        g.mark_output(g.op("quantize", (x,), g.tensor("s8", (len(sel),), scale=1.0, zero_point=zp)))
+        got = interp.run(g, {x: np.array([r[0] for r in sel], dtype=np.float32)})[g.outputs[0]]
+        assert got.tolist() == [r[2] for r in sel]
+
+
+def test_bf16_rounding_ties_to_even_and_no_double_rounding_golden():
+    """tests/golden/bf16_rounding.txt: exact ties between two bf16 neighbours (lower neighbour even, and odd), both
+    signs, and fp64 values just above a tie, which a detour through fp32 would round the other way."""
+    vals, bits = [], []
+    with open(os.path.join(GOLDEN, "bf16_rounding.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                sign, exps, b = line.split()
+                v = math.fsum(2.0 ** int(t) for t in exps.split(","))
+                vals.append(-v if sign == "-" else v)
+                bits.append(int(b, 16))
+    assert len(vals) >= 10
+    got = interp._round_to_bf16(np.array(vals, dtype=np.float64))
+    assert got.dtype == np.float32
+    assert (got.view(np.uint32) & 0xFFFF == 0).all()                    # bf16 values
+    assert (got.view(np.uint32) >> 16).tolist() == bits
+    # the faithful TypeCast goes through the same routine
+    g = Graph()
+    x = g.input("f32", (2,))
+    g.mark_output(g.op("typecast", (x,), g.tensor("bf16", (2,))))
+    out = interp.run(g, {x: np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8], dtype=np.float32)}, faithful=True)[g.outputs[0]]
+    assert (out.view(np.uint32) >> 16).tolist() == [0x3F80, 0x3F82]
+
+
 def test_requant_reciprocal_constants():
     # the reciprocal is formed in fp32; for the workloads' scales it is exactly these values
     assert np.float32(1.0) / np.float32(0.05) == np.float32(20.0)
