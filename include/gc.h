@@ -43,7 +43,13 @@
  *     be 16-byte aligned (GC_ERR_ALIGNMENT otherwise).
  *   - in_*[i] corresponds to input_ids[i] given at gc_partition_create, out_*[i] to output_ids[i].
  *   - gc_execute is asynchronous on the given stream.  One compiled object must not be executed
- *     concurrently on two streams (it owns one workspace).
+ *     concurrently on two streams (it owns one workspace).  Plans that run as ONE persistent kernel
+ *     whose CTAs wait for one another (the small-batch chain, two large layers in one launch; the
+ *     plan description names them) size their grid to what the device can hold resident at once,
+ *     queried at gc_compile: work of another object, or of anything else, that occupies SMs at the
+ *     same time can keep part of such a grid from starting.  Run these objects one at a time per
+ *     GPU (one stream, or ordered streams); if they are overlapped anyway the bounded waits expire
+ *     and gc_query_status reports GC_ERR_TIMEOUT - nothing hangs.
  *   - Device-side waits are bounded: if one expires the kernel records an error in a status word
  *     and returns; gc_query_status reports it as GC_ERR_TIMEOUT.  Nothing traps.
  */
@@ -185,8 +191,17 @@ gc_status_t gc_execute_host(gc_compiled_t* c, void* cuda_stream, const void* con
 
 /* No counterpart in the paper (its CPU kernels cannot time out).  Synchronise the stream and read
  * the device status word: GC_OK, GC_ERR_TIMEOUT (a bounded device-side wait expired) or
- * GC_ERR_CUDA (the stream reported an error). */
+ * GC_ERR_CUDA (the stream reported an error).  A kernel that gave up leaves its synchronisation
+ * counters mid-count, and the outputs of that execute (and of any later one issued before this
+ * call) are undefined; when this call reports GC_ERR_TIMEOUT it has also zeroed the status word
+ * and those counters, so the object can be executed again afterwards.  The cached prepacked
+ * constants are kept. */
 gc_status_t gc_query_status(gc_compiled_t* c, void* cuda_stream);
+
+/* Constants are preprocessed once per address (Section V) and the result is cached; a caller that
+ * rewrites a constant IN PLACE (same address, new contents) calls this to drop the cache: the next
+ * execute preprocesses every constant again.  Host only; must not race with an execute. */
+gc_status_t gc_invalidate_constants(gc_compiled_t* c);
 
 /* No counterpart in the paper: introspection for tests and benchmarks.  Number of kernel launches
  * one gc_execute enqueues after prepacking, and a short text description of the plan (pattern,
@@ -206,6 +221,8 @@ const char* gc_plan_description(const gc_compiled_t* c);
  *
  *   - Limit: n * round_up(k, 128) <= gc_noalloc_scratch_bytes() (1 MiB); larger problems are rejected
  *     with GC_ERR_UNSUPPORTED and a message - use gc_compile / gc_execute with a workspace instead.
+ *     Also rejected: a_zero_point outside 0..255 (GC_ERR_INVALID_ARG), k > 65536 (the exact sum could
+ *     leave s32) and m * n beyond what one launch covers (about 1.7e10), both GC_ERR_UNSUPPORTED.
  *   - The array costs every GPU that loads this library 1 MiB of device memory until the process exits.
  *   - All calls share the array.  Calls that can overlap on the GPU (different streams, or host threads
  *     racing on one stream) corrupt each other's scratch: keep them on one stream or serialise them.

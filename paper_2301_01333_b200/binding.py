@@ -33,7 +33,7 @@ EXPORTS = [
     "gc_partition_create", "gc_partition_destroy", "gc_compile", "gc_compiled_destroy", "gc_workspace_bytes",
     "gc_set_workspace", "gc_execute", "gc_host_staging_bytes", "gc_set_host_staging", "gc_execute_host",
     "gc_query_status", "gc_launches_per_execute", "gc_plan_description", "gc_last_error", "gc_version",
-    "gc_matmul_s32_noalloc", "gc_noalloc_scratch_bytes", "gc_selftest_bounded_wait",
+    "gc_matmul_s32_noalloc", "gc_noalloc_scratch_bytes", "gc_selftest_bounded_wait", "gc_invalidate_constants",
 ]
 
 
@@ -94,6 +94,8 @@ def load_library() -> C.CDLL:
     lib.gc_matmul_s32_noalloc.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32]
     lib.gc_matmul_s32_noalloc.restype = i32
     lib.gc_noalloc_scratch_bytes.restype = sz
+    lib.gc_invalidate_constants.argtypes = [vp]
+    lib.gc_invalidate_constants.restype = i32
     lib.gc_selftest_bounded_wait.argtypes = [vp, vp, C.c_uint32]
     lib.gc_selftest_bounded_wait.restype = i32
     for name in ("gc_partition_create", "gc_compile", "gc_workspace_bytes", "gc_set_workspace", "gc_execute",
@@ -219,6 +221,10 @@ def gc_query_status(c, stream: int = 0) -> None:
     _check(load_library().gc_query_status(c, C.c_void_p(stream)))
 
 
+def gc_invalidate_constants(c) -> None:
+    _check(load_library().gc_invalidate_constants(c))
+
+
 def gc_launches_per_execute(c) -> int:
     n = C.c_int32()
     _check(load_library().gc_launches_per_execute(c, C.byref(n)))
@@ -308,6 +314,9 @@ class CompiledPartition:
         if stream is None:
             stream = torch.cuda.current_stream(self.device).cuda_stream
         gc_query_status(self._comp, stream)
+
+    def invalidate_constants(self) -> None:
+        gc_invalidate_constants(self._comp)
 
     # -- host execution ---------------------------------------------------------------------------
     def execute_host(self, in_arrays: List[np.ndarray], out_arrays: List[np.ndarray], stream: Optional[int] = None):

@@ -767,7 +767,7 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
       // 256-1 at batch 512, 42 against 33 microseconds).
       if (row_tiles > 1 && ks == 1 && a_stages > 4) fits = false;
       // all clusters must be resident together (the layers are separated by a grid-wide barrier)
-      if (fits && ks > 1 && cuda_device != GC_DEVICE_PLAN_ONLY) {
+      if (fits && cuda_device != GC_DEVICE_PLAN_ONLY) {
         int cur = -1;
         cudaGetDevice(&cur);
         if (cur != cuda_device) cudaSetDevice(cuda_device);     // the occupancy query answers for the current device
@@ -808,7 +808,18 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
       const bool kinds_ok = A.use_tc && B.use_tc && A.cta2 && B.cta2 && A.kind == B.kind && A.M == B.M && !B.need_pack &&
                             out_kind(A) == out_kind(B) && out_kind(A) == A.kind;   // i8 -> 8-bit, bf16 -> bf16, tf32 -> f32
       if (!kinds_ok) continue;
-      const int C = c->num_sms / 2;
+      // Second-layer tiles wait on counters that first-layer tiles of OTHER clusters advance, so every cluster of the
+      // launch must be resident at once: no more clusters than the device can hold of this kernel.
+      int C = c->num_sms / 2;
+      if (cuda_device != GC_DEVICE_PLAN_ONLY) {
+        int cur = -1;
+        cudaGetDevice(&cur);
+        if (cur != cuda_device) cudaSetDevice(cuda_device);
+        const int resident = gemm_tc2_max_clusters(A.kind, A.epi.out_dtype);
+        if (cur >= 0 && cur != cuda_device) cudaSetDevice(cur);
+        if (resident < C) C = resident;
+      }
+      if (C < 1) continue;
       const int m_pairs = (A.m_tiles + 1) / 2;
       const long T0 = static_cast<long>(m_pairs) * A.n_tiles, T1 = static_cast<long>(m_pairs) * B.n_tiles;
       const long w0 = A.nkb, w1 = B.nkb;
@@ -1269,6 +1280,16 @@ static gc_status_t run_sdpa(gc_compiled& c, cudaStream_t st, const void* const* 
   return GC_OK;
 }
 
+// Zero the status word, the chain kernel's grid-barrier counter (both in the first 256 bytes of the workspace) and
+// the counters of every fused two-layer launch.
+static gc_status_t reset_device_state(gc_compiled& c, cudaStream_t st) {
+  CUDA_TRY(cudaMemsetAsync(c.ws, 0, 256, st));
+  for (auto& L : c.layers)
+    if (L.fused_first)
+      CUDA_TRY(cudaMemsetAsync(static_cast<char*>(c.ws) + L.pair_ready_off, 0, L.pair_ready_words * sizeof(unsigned long long), st));
+  return GC_OK;
+}
+
 extern "C" gc_status_t gc_execute(gc_compiled_t* c, void* cuda_stream, const void* const* in_dev, int32_t n_in,
                                   void* const* out_dev, int32_t n_out) {
   if (!c || !in_dev || !out_dev) return fail(GC_ERR_INVALID_ARG, "null argument");
@@ -1322,6 +1343,9 @@ extern "C" gc_status_t gc_execute_host(gc_compiled_t* c, void* cuda_stream, cons
     din[i] = sg + c->in_stage_off[i];
     if (!c->in_constant[i] || c->host_const_seen[i] != in_host[i]) {
       CUDA_TRY(cudaMemcpyAsync(sg + c->in_stage_off[i], in_host[i], c->in_bytes[i], cudaMemcpyHostToDevice, st));
+      // A constant that arrives at a new host address lands at the same staging address: forget the device
+      // pointer recorded at the last prepack, so that the execute below preprocesses the new contents.
+      if (c->in_constant[i] && c->host_const_seen[i] != nullptr) c->const_ptrs[i] = nullptr;
       c->host_const_seen[i] = in_host[i];
     }
   }
@@ -1353,6 +1377,23 @@ extern "C" gc_status_t gc_query_status(gc_compiled_t* c, void* cuda_stream) {
   uint32_t word = 0;
   CUDA_TRY(cudaMemcpyAsync(&word, c->ws, sizeof(word), cudaMemcpyDeviceToHost, st));
   CUDA_TRY(cudaStreamSynchronize(st));
-  if (word != 0) return fail(GC_ERR_TIMEOUT, "a bounded device-side wait expired (code 0x%x)", word);
+  if (word != 0) {
+    // The kernels that gave up left their synchronisation counters (grid-barrier count, the fused two-layer
+    // launch's epoch and per-tile counters) mid-count.  The stream is idle here: zero them together with the status
+    // word, so that the next execute starts from a clean state; the cached prepacked weights stay valid.
+    gc_status_t r = reset_device_state(*c, st);
+    if (r != GC_OK) return r;
+    CUDA_TRY(cudaStreamSynchronize(st));
+    return fail(GC_ERR_TIMEOUT, "a bounded device-side wait expired (code 0x%x); the object's device state has been reset",
+                word);
+  }
+  return GC_OK;
+}
+
+extern "C" gc_status_t gc_invalidate_constants(gc_compiled_t* c) {
+  if (!c) return fail(GC_ERR_INVALID_ARG, "null argument");
+  c->prepacked = false;
+  std::fill(c->const_ptrs.begin(), c->const_ptrs.end(), nullptr);
+  std::fill(c->host_const_seen.begin(), c->host_const_seen.end(), nullptr);
   return GC_OK;
 }

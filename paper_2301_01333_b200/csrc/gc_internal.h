@@ -149,6 +149,10 @@ cudaError_t launch_mlp_chain(int kind, const ChainParams& p, int grid, cudaStrea
 // clusters of `ks` CTAs of the chain kernel that can be resident together on the current device (0 on error)
 int mlp_chain_max_clusters(int kind, int ks, size_t smem);
 
+// Raise a kernel's dynamic shared-memory limit to at least `smem` bytes on the current device.  The driver call is made
+// once per (kernel, device) and size, not on every launch.
+cudaError_t ensure_dynamic_smem(const void* kern, size_t smem);
+
 // ---- launchers (each enqueues exactly one kernel on the stream and returns cudaGetLastError) ----
 cudaError_t launch_pack_rows(const void* src, void* dst, int rows, int64_t src_pitch_bytes, int64_t dst_pitch_bytes,
                              cudaStream_t s);
@@ -175,6 +179,8 @@ cudaError_t launch_gemm_tc(int kind, int block_n, int a_signed, const CUtensorMa
 // CTA-pair variant (cta_group::2): 256 x 256 tiles per cluster of two CTAs; tmB must have a 128-row box.
 // `grid` must be even.
 size_t gemm_tc2_smem_bytes();
+// clusters of two CTAs of the CTA-pair kernel that can be resident together on the current device (0 on error)
+int gemm_tc2_max_clusters(int kind, int out_dtype);
 cudaError_t launch_gemm_tc2(int kind, int a_signed, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmD,
                             const GemmTcParams& p, int grid, bool pdl, cudaStream_t s);
 

@@ -55,6 +55,13 @@ extern "C" gc_status_t gc_matmul_s32_noalloc(void* cuda_stream, const void* a_de
   if (!a_dev || !w_dev || !out_dev) return gc_set_error(GC_ERR_INVALID_ARG, "gc_matmul_s32_noalloc: null pointer");
   if (m <= 0 || k <= 0 || n <= 0) return gc_set_error(GC_ERR_SHAPE, "gc_matmul_s32_noalloc: non-positive dimension");
   if (reinterpret_cast<uintptr_t>(out_dev) % 4) return gc_set_error(GC_ERR_ALIGNMENT, "gc_matmul_s32_noalloc: output must be 4-byte aligned");
+  if (a_zero_point < 0 || a_zero_point > 255)
+    return gc_set_error(GC_ERR_INVALID_ARG, "gc_matmul_s32_noalloc: the zero point of a u8 operand lies in 0..255");
+  // |a - zp| <= 255 and |w| <= 128: the exact sum stays inside s32 for k up to 65536
+  if (k > 65536) return gc_set_error(GC_ERR_UNSUPPORTED, "gc_matmul_s32_noalloc: k above 65536 could overflow the s32 result");
+  // one warp per output element, eight warps per block, at most 2^31 - 1 blocks
+  if (static_cast<int64_t>(m) * n > 8LL * 0x7FFFFFFFLL)
+    return gc_set_error(GC_ERR_UNSUPPORTED, "gc_matmul_s32_noalloc: m * n exceeds what one launch covers");
   const int64_t kp = (static_cast<int64_t>(k) + 127) / 128 * 128;   // reduction axis padded to 128 bytes
   if (kp * n > static_cast<int64_t>(GC_NOALLOC_SCRATCH_BYTES))
     return gc_set_error(GC_ERR_UNSUPPORTED,

@@ -486,7 +486,7 @@ cudaError_t launch_mlp_chain(int kind, const ChainParams& p, int grid, cudaStrea
   void* kern = kind == KIND_I8 ? reinterpret_cast<void*>(mlp_chain_kernel<KIND_I8>)
                : kind == KIND_BF16 ? reinterpret_cast<void*>(mlp_chain_kernel<KIND_BF16>)
                                    : reinterpret_cast<void*>(mlp_chain_kernel<KIND_TF32>);
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  cudaError_t e = ensure_dynamic_smem(kern, smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
@@ -515,7 +515,7 @@ int mlp_chain_max_clusters(int kind, int ks, size_t smem) {
   void* kern = kind == KIND_I8 ? reinterpret_cast<void*>(mlp_chain_kernel<KIND_I8>)
                : kind == KIND_BF16 ? reinterpret_cast<void*>(mlp_chain_kernel<KIND_BF16>)
                                    : reinterpret_cast<void*>(mlp_chain_kernel<KIND_TF32>);
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) return 0;
+  if (ensure_dynamic_smem(kern, smem) != cudaSuccess) return 0;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(ks));
   cfg.blockDim = dim3(CH_THREADS);

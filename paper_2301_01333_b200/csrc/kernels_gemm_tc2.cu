@@ -409,7 +409,7 @@ template <int KIND, int OUT>
 cudaError_t launch_fused_t(const GemmPairParams& p, int grid, bool pdl, cudaStream_t s) {
   const size_t smem = fused_smem_bytes();
   auto kern = gemm_tc2_kernel<KIND, OUT>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
@@ -431,6 +431,30 @@ cudaError_t launch_fused_t(const GemmPairParams& p, int grid, bool pdl, cudaStre
 }  // namespace
 
 size_t gemm_tc2_smem_bytes() { return fused_smem_bytes(); }
+
+int gemm_tc2_max_clusters(int kind, int out_dtype) {
+  const void* kern = nullptr;
+  if (kind == KIND_BF16 && out_dtype == GC_BF16) kern = reinterpret_cast<const void*>(gemm_tc2_kernel<KIND_BF16, OUT_BF16>);
+  else if (kind == KIND_I8 && (out_dtype == GC_U8 || out_dtype == GC_S8)) kern = reinterpret_cast<const void*>(gemm_tc2_kernel<KIND_I8, OUT_Q8>);
+  else if (kind == KIND_TF32 && out_dtype == GC_F32) kern = reinterpret_cast<const void*>(gemm_tc2_kernel<KIND_TF32, OUT_F32>);
+  if (!kern) return 0;
+  const size_t smem = fused_smem_bytes();
+  if (ensure_dynamic_smem(kern, smem) != cudaSuccess) return 0;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2);
+  cfg.blockDim = dim3(F2_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) return 0;
+  return n;
+}
 
 // kind: 0 = i8, 1 = bf16, 2 = tf32; both layers share the MMA kind and the output element type.
 cudaError_t launch_gemm_tc2_fused(int kind, int a_signed, const GemmPairParams& p_in, int grid, cudaStream_t s) {

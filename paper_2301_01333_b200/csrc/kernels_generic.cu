@@ -4,6 +4,9 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <map>
+#include <mutex>
+#include <utility>
 
 #include "epilogue.cuh"
 #include "gc_internal.h"
@@ -188,10 +191,25 @@ __global__ void gemm_simt_kernel(const GemmSimtParams p) {
   }
 }
 
+cudaError_t ensure_dynamic_smem(const void* kern, size_t smem) {
+  static std::mutex mu;
+  static std::map<std::pair<const void*, int>, size_t> done;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  std::lock_guard<std::mutex> lock(mu);
+  size_t& have = done[std::make_pair(kern, dev)];
+  if (have >= smem && have != 0) return cudaSuccess;
+  e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e == cudaSuccess) have = smem;
+  return e;
+}
+
 cudaError_t launch_gemm_simt(const GemmSimtParams& p, cudaStream_t s) {
   const int64_t warps = static_cast<int64_t>(p.M) * p.N * p.batch;
   const int block = 256;
   const int64_t grid = (warps * 32 + block - 1) / block;
+  if (grid > 0x7FFFFFFFLL) return cudaErrorInvalidValue;          // one warp per output element: beyond the x-dimension limit
   gemm_simt_kernel<<<static_cast<unsigned>(std::max<int64_t>(grid, 1)), block, 0, s>>>(p);
   return cudaGetLastError();
 }
@@ -283,8 +301,7 @@ cudaError_t launch_sdpa_simt(const SdpaParams& p, cudaStream_t s) {
   const int64_t rows = static_cast<int64_t>(p.B) * p.H * p.S;
   const size_t smem = static_cast<size_t>(SDPA_SIMT_WARPS) * p.S * sizeof(float);
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(sdpa_simt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(smem));
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(sdpa_simt_kernel), smem);
     if (e != cudaSuccess) return e;
   }
   const int64_t grid = (rows + SDPA_SIMT_WARPS - 1) / SDPA_SIMT_WARPS;

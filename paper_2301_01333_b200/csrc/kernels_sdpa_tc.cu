@@ -785,7 +785,7 @@ cudaError_t launch_sdpa_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const
   lc.numAttrs = 1;
   const int code = cfg.slots * 100 + cfg.nsb * 10 + cfg.stage_out;
   auto go = [&](auto kern) -> cudaError_t {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(cfg.smem));
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), cfg.smem);
     if (e != cudaSuccess) return e;
     return cudaLaunchKernelEx(&lc, kern, tmQ, tmK, tmV, tmO, p, cfg.slots, cfg.nsb, cfg.stage_out);
   };

@@ -756,7 +756,7 @@ cudaError_t launch_wide_nb(const CUtensorMap& tmQ, const CUtensorMap& tmK, const
     auto kern = sdpa_wide_kernel<INT8, D, NB, cfg.np, cfg.stages>;
     const int units = p.B * p.H * (p.S / W_BLOCK_Q);
     const int grid = units < num_sms ? units : num_sms;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(cfg.smem));
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), cfg.smem);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(grid);

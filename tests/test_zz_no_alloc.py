@@ -7,6 +7,7 @@ different shape right after the first to show that what the first call left behi
 import numpy as np
 import pytest
 
+from oracle import interp
 from paper_2301_01333_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
@@ -43,8 +44,18 @@ def test_noalloc_matmul_matches_regular_entry_point_twice_in_a_row():
         torch.cuda.synchronize()
         got = out.cpu().numpy().reshape(m, n)
         assert np.array_equal(got, expect)          # integer path: bit-exact, the tolerance the other tests use
+        # and directly against the oracle's definition of the same matmul
+        assert np.array_equal(got.astype(np.int64), interp.run(w.graph, w.feeds)[w.graph.outputs[0]])
 
     # beyond the built-in scratch: refused with a clear message, nothing launched
     with pytest.raises(B.GcError) as e:
         B.gc_matmul_s32_noalloc(stream, a_dev.data_ptr(), w_dev.data_ptr(), out.data_ptr(), 8, 4096, 1024, 0)
     assert e.value.status == B.GC_ERR_UNSUPPORTED and "1 MiB" in str(e.value)
+    # a zero point no u8 operand can have, and a reduction long enough to leave s32: refused as well
+    for bad_zp in (-1, 256):
+        with pytest.raises(B.GcError) as e:
+            B.gc_matmul_s32_noalloc(stream, a_dev.data_ptr(), w_dev.data_ptr(), out.data_ptr(), 8, 64, 16, bad_zp)
+        assert e.value.status == B.GC_ERR_INVALID_ARG
+    with pytest.raises(B.GcError) as e:
+        B.gc_matmul_s32_noalloc(stream, a_dev.data_ptr(), w_dev.data_ptr(), out.data_ptr(), 8, 70000, 8, 0)
+    assert e.value.status == B.GC_ERR_UNSUPPORTED
