@@ -121,10 +121,13 @@ class Replica:
         self.c.execute(self.ins, self.outs, stream)
 
 
-def time_config(B, name, steps, warmup, device, **opts):
-    """Builds the rotating replicas of one config (total footprint above the L2 size) and warms them up."""
+def time_config(B, name, steps, warmup, device, shard=None, **opts):
+    """Builds the rotating replicas of one config (total footprint above the L2 size) and warms them up.
+    shard = (first, count): this rank's units of the config's one batch instead of the whole batch."""
     import torch
     w = W.CONFIGS[name]()
+    if shard is not None:
+        w = W.shard_config(name, w, shard[0], shard[1])
     stream = torch.cuda.current_stream(device).cuda_stream
     first = Replica(B, w, 0, device, **opts)
     n_rep = int(min(64, max(2, -(-int(1.25 * L2_BYTES) // first.bytes))))
@@ -316,6 +319,45 @@ def run_e2e(w, rep, steps, warmup, device):
     return dt / steps, h2d, d2h
 
 
+def parity_check(B, name, w, rep):
+    """Outside the timed region: the output one timed replica last produced against the oracle on the same inputs -
+    every output for the small-batch chains, 256 sampled rows for the FFN, one sequence (all heads) for attention -
+    at the tolerances of the parity tests.  Uses the oracle, so it belongs to the CPU-baseline leg."""
+    from oracle import interp
+    make, key, _ = W.CONFIG_UNITS[name]
+    g = w.graph
+    total = g.tensors[g.inputs[0]].dims[0]
+    if name in ("c1", "c2"):
+        idx = np.arange(total)
+    elif name == "c5":
+        idx = np.sort(np.random.default_rng(1).choice(total, size=min(256, total), replace=False))
+    else:
+        idx = np.array([total // 2])
+    sub = make(**{key: len(idx)})
+    for a, b in zip(sub.graph.inputs, g.inputs):
+        src = w.feeds[b]
+        sub.feeds[a] = np.ascontiguousarray(src[idx]) if (not g.tensors[b].is_constant and src.shape[0] == total) else src
+    ref = interp.run(sub.graph, sub.feeds)[sub.graph.outputs[0]]
+    got = B.output_to_numpy(g, g.outputs[0], rep.outs[0])[idx]
+    if name == "c4":
+        d = np.abs(got.astype(np.int64) - ref)
+        err, frac = float(d.max()), float((d != 0).mean())
+        ok = err <= 1 and frac <= 1e-3
+        return {"rows": int(len(idx)), "unit": "sequences (all heads)", "max_err": err, "mismatch_frac": frac,
+                "tolerance": "codes within 1, at most 1e-3 of them different", "ok": bool(ok)}
+    if name in ("c3", "c5"):
+        err = float(np.abs(W.bf16_bits_to_f32(got).astype(np.float64) - ref).max())
+        tol = 2e-2
+    elif name == "c1":
+        err = float(np.abs(got - ref).max())
+        tol = 5e-3 * float(np.abs(ref).max())
+    else:
+        err = float(np.abs(got.astype(np.float64) - ref).max())
+        tol = 2e-6
+    return {"rows": int(len(idx)), "unit": "sequences (all heads)" if name == "c3" else "rows", "max_err": err,
+            "tolerance": tol, "ok": bool(err <= tol)}
+
+
 def cpu_sample(name):
     """A bounded sample of the config for the oracle: returns (workload, fraction of the full ops, text)."""
     if name == "c1":
@@ -388,6 +430,9 @@ def main():
     ap.add_argument("--gemm", action="store_true",
                     help="instead of the benchmark: one plain 8192^3 bf16 GEMM, timed like the measured library peaks")
     ap.add_argument("--sweep-filter", default="", help="with --sweep: only the cases whose name contains this text")
+    ap.add_argument("--split", action="store_true",
+                    help="with N ranks: split the config's ONE batch evenly over the ranks (8192/N tokens, 64/N sequences; "
+                         "strong scaling) instead of one full batch per rank")
     args = ap.parse_args()
     if args.impl == "reference":
         if args.steps == 0:
@@ -395,47 +440,37 @@ def main():
         return reference_arm(args)
 
     import torch
-    import torch.distributed as dist
     from paper_2301_01333_b200 import build as gc_build
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2301_01333_b200 import multi
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
-    if local == 0:
-        gc_build.build()
-    if world > 1:
-        dist.barrier()
+    ranks = multi.init_ranks("nccl", f"cuda:{local}")
+    rank, world = ranks.rank, ranks.world
+    multi.build_on_local_root(ranks, gc_build.build)
     from paper_2301_01333_b200 import binding as B
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        multi.barrier(ranks)
 
     def max_over_ranks(x):
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=f"cuda:{local}")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return multi.max_over_ranks(ranks, x, f"cuda:{local}")
 
     peaks, peak_src = load_peaks()
     if args.gemm:
         if rank == 0:
             print(json.dumps({"plain_gemm": run_plain_gemm(B, local, peaks), "data": "synthetic"}))
         if world > 1:
-            dist.barrier()
-            dist.destroy_process_group()
+            barrier()
+            multi.finish(ranks)
         return
     if args.sweep:
         if rank == 0:
             print(json.dumps({"sweep": run_sweep(B, local, peaks, args.sweep_filter), "unit": "us per subgraph, cold L2", "data": "synthetic"}))
         if world > 1:
-            dist.barrier()
-            dist.destroy_process_group()
+            barrier()
+            multi.finish(ranks)
         return
     head = args.workload
     names = [head] if args.only else [head] + [n for n in W.CONFIGS if n != head]
@@ -447,7 +482,11 @@ def main():
     e2e = None
     for name in names:
         steps = args.steps if (args.steps and name == head) else DEFAULT_STEPS[name]
-        w, reps, n_rep = time_config(B, name, steps, args.warmup, local)
+        shard = None
+        if args.split and world > 1:
+            shard = multi.split_units(W.CONFIG_UNITS[name][2], world, rank)
+        w, reps, n_rep = time_config(B, name, steps, args.warmup, local, shard=shard)
+        job_ops = multi.sum_over_ranks(ranks, float(w.ops), f"cuda:{local}")     # what all ranks process per step
         sampler = None
         if name == head and rank == 0:
             sampler = ClockSampler(local)
@@ -468,7 +507,7 @@ def main():
         t_tensor_meas = w.ops / (tensor_meas * 1e12)
         bound = "tensor" if t_tensor_meas > t_hbm_meas else "hbm"
         res = {
-            "graph": w.name, "us_per_subgraph": us, "value": w.ops * world / (us * 1e-6) / 1e12, "unit": UNIT[name],
+            "graph": w.name, "us_per_subgraph": us, "value": job_ops / (us * 1e-6) / 1e12, "unit": UNIT[name],
             "steps": steps, "replicas": n_rep, "launches_per_step": reps[0].c.launches,
             "algorithmic_ops": w.ops, "algorithmic_bytes": w.bytes,
             "achieved_gbs": w.bytes / (us * 1e-6) / 1e9,
@@ -502,11 +541,13 @@ def main():
             res["exp_bound_us"] = t_exp * 1e6
             res["exp_bound_frac"] = t_exp / (us * 1e-6)
             res["scores"] = n_exp
+        if rank == 0 and not args.no_cpu:
+            res["parity_checked"] = parity_check(B, name, w, reps[0])
         if name == head:
             launches_total = steps * reps[0].c.launches
             e2e_s, h2d, d2h = run_e2e(w, reps[0], max(3, min(steps, 50)), args.warmup, local)
             e2e_s = max_over_ranks(e2e_s)
-            e2e = {"value": w.ops * world / e2e_s / 1e12, "unit": UNIT[name], "h2d_bytes_per_step": h2d,
+            e2e = {"value": job_ops / e2e_s / 1e12, "unit": UNIT[name], "h2d_bytes_per_step": h2d,
                    "d2h_bytes_per_step": d2h, "us_per_subgraph": e2e_s * 1e6}
             head_w, head_ms, head_steps, head_reps, head_peak_key = w, ms, steps, n_rep, peak_key
         results[name] = res
@@ -517,7 +558,7 @@ def main():
 
     if rank != 0:
         if world > 1:
-            dist.destroy_process_group()
+            multi.finish(ranks)
         return
     hr = results[head]
     us = hr["us_per_subgraph"]
@@ -554,17 +595,24 @@ def main():
     line = {
         "metric": "fused_subgraph_throughput", "value": hr["value"], "unit": UNIT[head], "n_gpus": world,
         "steps": head_steps, "warmup": max(args.warmup, 3), "ms_per_step": head_ms / head_steps, "us_per_subgraph": us,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": DTYPE[head], "data": "synthetic",
+        "higher_is_better": True, "scaling": "strong" if (args.split and world > 1) else "weak", "vs_baseline": None,
+        "dtype": DTYPE[head], "data": "synthetic",
         "config": {"workload": head, "graph": head_w.name,
                    "l2": f"steps rotate through {head_reps} independent replicas (weights, workspace, inputs, outputs) "
                          f"whose total footprint exceeds the 126 MB L2",
-                   "parallelism": f"replicas x{world} (independent batches per GPU, no collective)"},
+                   "parallelism": (f"one batch split evenly over {world} GPUs (rows / sequences are independent, no collective)"
+                                   if (args.split and world > 1) else
+                                   f"replicas x{world} (independent batches per GPU, no collective)")},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_total, "roofline": roof, "cpu_baseline": cpu,
+        "parity_checked": hr.get("parity_checked"),
         "configs": results,
     }
     print(json.dumps(line))
     if world > 1:
-        dist.destroy_process_group()
+        multi.finish(ranks)
+    bad = [n for n, r in results.items() if r.get("parity_checked") and not r["parity_checked"]["ok"]]
+    if bad:
+        raise SystemExit(f"parity check against the oracle failed for {bad}")
 
 
 if __name__ == "__main__":

@@ -40,8 +40,8 @@ class LogicalTensor:
     zero_point: int = 0
     is_constant: bool = False  # same pointer and contents on every execution (weights, biases)
     name: str = ""
-    # per-channel quantisation of a constant s8 weight (Section VII: "per channel s8 symmetric quantization
-    # for weight"): one scale per index of `channel_axis`, which must be the output-channel axis of the
+    # per-channel quantisation of a constant s8 weight (the symmetric per-output-channel weight scheme of
+    # Section VII's int8 evaluation): one scale per index of `channel_axis`, which must be the output-channel axis of the
     # MatMul that consumes the tensor.  None = the per-tensor `scale` applies.
     channel_scales: Optional[Tuple[float, ...]] = None
     channel_axis: int = -1

@@ -293,3 +293,29 @@ CONFIGS = {
     "c4": lambda: mha_int8(),
     "c5": lambda: ffn_bf16(),
 }
+
+# The independent units a config shards over when several GPUs split ONE batch (rows of an MLP chain, sequences of
+# an attention block; Section V's outer parallel loop over the batch and Section VII's independent (batch, head)
+# units): builder keyword that sets the unit count, and the full count.
+CONFIG_UNITS = {
+    "c1": (mlp_f32, "batch", 32),
+    "c2": (mlp_int8, "batch", 128),
+    "c3": (mha_bf16, "batch", 32),
+    "c4": (mha_int8, "batch", 64),
+    "c5": (ffn_bf16, "tokens", 8192),
+}
+
+
+def shard_config(name: str, full: Workload, first: int, count: int) -> Workload:
+    """Units [first, first + count) of config `name`: a workload of `count` units whose per-unit inputs are that
+    slice of the full workload's inputs (leading axis) and whose constants are the full workload's."""
+    make, key, total = CONFIG_UNITS[name]
+    shard = make(**{key: count})
+    for a, b in zip(shard.graph.inputs, full.graph.inputs):
+        src = full.feeds[b]
+        if not full.graph.tensors[b].is_constant and src.shape[0] == total:
+            shard.feeds[a] = np.ascontiguousarray(src[first:first + count])
+        else:
+            shard.feeds[a] = src
+    shard.info = dict(shard.info, first=first, count=count, of=total)
+    return shard
