@@ -316,6 +316,25 @@ static gc_status_t make_tmap(CUtensorMap* m, const void* ptr, int dtype, uint64_
   return GC_OK;
 }
 
+// 3-D tensor [slices][rows][inner], dense; box = [1][box_rows][box_inner].  Rows past a slice's end (and columns past
+// `inner`) read as zeros.
+static gc_status_t make_tmap3(CUtensorMap* m, const void* ptr, int dtype, uint64_t inner, uint64_t rows, uint64_t slices,
+                              uint32_t box_inner, uint32_t box_rows, int swizzle_bytes) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return fail(GC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+  const uint64_t esz = static_cast<uint64_t>(dtype_bytes(dtype));
+  CUtensorMapDataType dt = dtype == GC_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8;
+  cuuint64_t gdim[3] = {inner, rows, slices};
+  cuuint64_t gstr[2] = {inner * esz, inner * esz * rows};
+  cuuint32_t box[3] = {box_inner, box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUtensorMapSwizzle sw = swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+  CUresult r = enc(m, dt, 3, const_cast<void*>(ptr), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(GC_ERR_CUDA, "cuTensorMapEncodeTiled (3-D) failed with code %d", (int)r);
+  return GC_OK;
+}
+
 // ------------------------------------------------------------------------------------------------
 // pattern formation
 // ------------------------------------------------------------------------------------------------
@@ -634,6 +653,8 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
       wide = tc = need > 0 && need <= static_cast<size_t>(prop.sharedMemPerBlockOptin);
     }
     if (!s.is_int8 && c->sdpa.p_out_pos >= 0) tc = false;   // the bf16 tcgen05 kernels never form normalised P
+    // the probabilities as a second output: written in 16-byte pieces, which needs whole key blocks
+    if (c->sdpa.p_out_pos >= 0 && s.S % 128 != 0) tc = false;
     if (s.is_int8)
       // Q must be exactly centred (s8 / zero point 0, or u8 / zero point 128); a zero point on K only
       // shifts every score of a row by the same amount, which softmax cancels
@@ -1247,8 +1268,9 @@ static gc_status_t run_sdpa(gc_compiled& c, cudaStream_t st, const void* const* 
     CUtensorMap* maps[3] = {&s.tmQ, &s.tmK, &s.tmV};
     for (int i = 0; i < 3; ++i) {
       if (*cached[i] == ptrs[i]) continue;
-      // a box wider than the head (D = 96) reads zeros past the tensor's edge
-      gc_status_t r = make_tmap(maps[i], ptrs[i], dt, prm.D, rows, static_cast<uint64_t>(prm.D) * esz, box, 128, swz);
+      // a box wider than the head (D = 96) reads zeros past the tensor's edge, and so does a box that reaches past
+      // the end of a head's sequence (sequence lengths that are not a multiple of 128)
+      gc_status_t r = make_tmap3(maps[i], ptrs[i], dt, prm.D, prm.S, static_cast<uint64_t>(prm.B) * prm.H, box, 128, swz);
       if (r != GC_OK) return r;
       *cached[i] = ptrs[i];
     }

@@ -22,6 +22,11 @@
 //
 // Zero points, the conversions by the 1.5 * 2^23 bias trick and the skipping of fully masked 32-key chunks
 // follow the D = 64 kernel.
+//
+// Sequence lengths that are not a multiple of 128 run as the next multiple: Q, K and V are addressed through 3-D
+// tensor maps [batch x head][key][d], so rows past the end of a head's sequence arrive as zeros; the keys past the end
+// carry a mask term of minus infinity (their exponentials, hence their codes, are exactly zero) and the query rows
+// past the end are computed but not stored.
 #include <cuda_bf16.h>
 
 #include "epilogue.cuh"
@@ -84,7 +89,8 @@ constexpr WideCfg wide_cfg_t(int S) {
 }
 
 WideCfg wide_cfg(int S, int D, int is_int8) {
-  if (S % 128 != 0 || S < 128 || S > 512) return {0, 0, 0};
+  if (S < 1 || S > 512) return {0, 0, 0};
+  S = (S + 127) / 128 * 128;                                    // runs as the next multiple of 128 keys
   if (is_int8) {
     if (D == 64) return wide_cfg_t<true, 64>(S);
     if (D == 96) return wide_cfg_t<true, 96>(S);
@@ -145,6 +151,7 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int q_tiles = S / W_BLOCK_Q;
   const int num_units = p.B * p.H * q_tiles;
+  const int s_real = p.S;                                       // S is its next multiple of 128
 
   if (tid == 0) {
     mbar_init(bar_q_full, 1);
@@ -188,12 +195,12 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (threadIdx.x == 0 && static_cast<int>(blockIdx.x) < p.B * p.H * (S / W_BLOCK_Q)) {
     const int unit = blockIdx.x, qt0 = S / W_BLOCK_Q;
-    const int row0 = (unit / qt0) * S;
-    for (int j = 0; j < L::NSUB; ++j) tma_prefetch_2d(&tmQ, j * L::SUB_ELEMS, row0 + (unit % qt0) * W_BLOCK_Q);
+    const int bh0 = unit / qt0;
+    for (int j = 0; j < L::NSUB; ++j) tma_prefetch_3d(&tmQ, j * L::SUB_ELEMS, (unit % qt0) * W_BLOCK_Q, bh0);
     for (int b = 0; b < NB; ++b)
       for (int j = 0; j < L::NSUB; ++j) {
-        tma_prefetch_2d(&tmK, j * L::SUB_ELEMS, row0 + b * 128);
-        tma_prefetch_2d(&tmV, j * L::SUB_ELEMS, row0 + b * 128);
+        tma_prefetch_3d(&tmK, j * L::SUB_ELEMS, b * 128, bh0);
+        tma_prefetch_3d(&tmV, j * L::SUB_ELEMS, b * 128, bh0);
       }
   }
   asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -215,8 +222,8 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (!mbar_wait(bar_q_empty, (nn & 1) ^ 1)) return false;
         mbar_arrive_expect_tx(bar_q_full, static_cast<uint32_t>(L::TILE_BYTES));
         for (int j = 0; j < L::NSUB; ++j)
-          tma_load_2d(smem_u32(sQ) + j * L::SUB_BYTES, &tmQ, j * L::SUB_ELEMS,
-                      (u / q_tiles) * S + (u % q_tiles) * W_BLOCK_Q, bar_q_full);
+          tma_load_3d(smem_u32(sQ) + j * L::SUB_BYTES, &tmQ, j * L::SUB_ELEMS, (u % q_tiles) * W_BLOCK_Q, u / q_tiles,
+                      bar_q_full);
         return true;
       };
       auto load_block = [&](const CUtensorMap* tm, int u, int b) -> bool {   // one 128-key block into the next stage
@@ -225,7 +232,7 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (!mbar_wait(bar_kv_empty + 8 * st, (use & 1) ^ 1)) return false;
         mbar_arrive_expect_tx(bar_kv_full + 8 * st, static_cast<uint32_t>(L::TILE_BYTES));
         for (int j = 0; j < L::NSUB; ++j)
-          tma_load_2d(smem_u32(sKV) + st * L::TILE_BYTES + j * L::SUB_BYTES, tm, j * L::SUB_ELEMS, (u / q_tiles) * S + b * 128,
+          tma_load_3d(smem_u32(sKV) + st * L::TILE_BYTES + j * L::SUB_BYTES, tm, j * L::SUB_ELEMS, b * 128, u / q_tiles,
                       bar_kv_full + 8 * st);
         return true;
       };
@@ -362,7 +369,8 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       if (!mbar_wait(bar_o_full, n0 & 1)) return false;
       tc_fence_after();
       const int bh = unit / q_tiles, qt = unit % q_tiles;
-      const int64_t grow = static_cast<int64_t>(bh) * S + qt * W_BLOCK_Q + r;
+      const bool row_ok = qt * W_BLOCK_Q + r < s_real;           // query rows past the sequence end are not stored
+      const int64_t grow = static_cast<int64_t>(bh) * s_real + qt * W_BLOCK_Q + r;
       uint8_t* dst = static_cast<uint8_t*>(p.O) + grow * OUT_ROW_BYTES;
       const int lo = p.out_dtype == GC_U8 ? 0 : -128, hi = p.out_dtype == GC_U8 ? 255 : 127;
       const int corr = INT8 ? p.zp_v * __float_as_int(total) : 0;   // zero point of V times the row sum of P
@@ -398,8 +406,10 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             w[i] = __byte_perm(__byte_perm(y[0], y[1], 0x0040), __byte_perm(y[2], y[3], 0x0040), 0x5410);
           }
           uint4* d4 = reinterpret_cast<uint4*>(dst + c * 32);
-          d4[0] = make_uint4(w[0], w[1], w[2], w[3]);
-          d4[1] = make_uint4(w[4], w[5], w[6], w[7]);
+          if (row_ok) {
+            d4[0] = make_uint4(w[0], w[1], w[2], w[3]);
+            d4[1] = make_uint4(w[4], w[5], w[6], w[7]);
+          }
         } else {
           uint32_t w[16];
 #pragma unroll
@@ -408,8 +418,10 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             w[i] = *reinterpret_cast<uint32_t*>(&hh);
           }
           uint4* d4 = reinterpret_cast<uint4*>(dst + c * 64);
+          if (row_ok) {
 #pragma unroll
-          for (int i = 0; i < 4; ++i) d4[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+            for (int i = 0; i < 4; ++i) d4[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+          }
         }
       }
       return true;
@@ -427,7 +439,7 @@ sdpa_wide_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int j = t + 128 * i;
-        mreg[i] = (p.mask && j < S) ? __ldg(p.mask + static_cast<int64_t>(b) * S + j) * W_LOG2E : 0.0f;
+        mreg[i] = j >= s_real ? -INFINITY : (p.mask ? __ldg(p.mask + static_cast<int64_t>(b) * s_real + j) * W_LOG2E : 0.0f);
       }
       if (!mbar_wait(bar_q_full, n & 1)) {
         report(p.status, DEV_TIMEOUT_OTHER);
@@ -754,7 +766,7 @@ cudaError_t launch_wide_nb(const CUtensorMap& tmQ, const CUtensorMap& tmK, const
     return cudaErrorInvalidValue;
   } else {
     auto kern = sdpa_wide_kernel<INT8, D, NB, cfg.np, cfg.stages>;
-    const int units = p.B * p.H * (p.S / W_BLOCK_Q);
+    const int units = p.B * p.H * ((p.S + W_BLOCK_Q - 1) / W_BLOCK_Q);
     const int grid = units < num_sms ? units : num_sms;
     cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), cfg.smem);
     if (e != cudaSuccess) return e;
@@ -775,8 +787,7 @@ cudaError_t launch_wide_nb(const CUtensorMap& tmQ, const CUtensorMap& tmK, const
 template <bool INT8, int D>
 cudaError_t launch_wide_t(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const SdpaParams& p,
                           int num_sms, cudaStream_t s) {
-  if (p.S % 128 != 0) return cudaErrorInvalidValue;
-  switch (p.S / 128) {
+  switch ((p.S + 127) / 128) {
     case 1: return launch_wide_nb<INT8, D, 1>(tmQ, tmK, tmV, p, num_sms, s);
     case 2: return launch_wide_nb<INT8, D, 2>(tmQ, tmK, tmV, p, num_sms, s);
     case 3: return launch_wide_nb<INT8, D, 3>(tmQ, tmK, tmV, p, num_sms, s);

@@ -361,7 +361,7 @@ def test_ffn_bf16_full_size_every_output(B):
 def test_mha_bf16(B, b, h, s, d):
     w = W.mha_bf16(batch=b, heads=h, seq=s, head_dim=d)
     got, plan = run_gpu(B, w)
-    assert ("tcgen05" in plan) == (d == 64 and s % 128 == 0)
+    assert ("tcgen05" in plan) == (d == 64)                  # any sequence length up to 512 keys; head width 32 is CUDA-core
     assert np.abs(bf16_to_f64(got) - oracle(w)).max() <= 2e-2
 
 
@@ -374,6 +374,41 @@ WIDE_SHAPES = [(1, 2, 128, 96), (1, 2, 384, 128), (1, 2, 512, 64), (2, 1, 256, 1
 @pytest.mark.parametrize("b,h,s,d", WIDE_SHAPES)
 def test_mha_bf16_streaming_kernel(B, b, h, s, d):
     w = W.mha_bf16(batch=b, heads=h, seq=s, head_dim=d)
+    got, plan = run_gpu(B, w)
+    assert "tcgen05.streaming" in plan
+    assert np.abs(bf16_to_f64(got) - oracle(w)).max() <= 2e-2
+
+
+# sequence lengths that are not a multiple of the 128-key block (a batch padded to 200 or 320 keys, fewer keys than one
+# block, one key short of or past a block): the kernel runs the next multiple, the keys past the end must get weight
+# exactly zero, the query rows past the end must not be stored (the guard bands around the output check that)
+RAGGED_SHAPES = [(1, 1, 200, 64), (2, 2, 320, 64), (1, 2, 72, 64), (2, 3, 127, 96), (1, 2, 129, 128), (3, 20, 200, 64),
+                 (1, 2, 500, 64), (1, 1, 8, 64)]
+
+
+@pytest.mark.parametrize("b,h,s,d", RAGGED_SHAPES)
+@pytest.mark.parametrize("kind", ["bf16", "int8"])
+def test_mha_ragged_sequence_lengths_on_tensor_cores(B, kind, b, h, s, d):
+    w = W.mha_bf16(batch=b, heads=h, seq=s, head_dim=d) if kind == "bf16" else W.mha_int8(batch=b, heads=h, seq=s, head_dim=d)
+    got, plan = run_gpu(B, w)
+    assert "tcgen05.streaming" in plan
+    if kind == "bf16":
+        assert np.abs(bf16_to_f64(got) - oracle(w)).max() <= 2e-2
+    else:
+        check_int8_attention(got, oracle(w))
+
+
+def test_mha_ragged_without_a_mask_and_with_minus_infinity(B):
+    # no mask op at all (the kernel still has to mask the keys past the end), and a user mask that already holds -inf
+    w = _attention_variant("int8", 2, 3, 200, 64, False, True, False)
+    got, plan = run_gpu(B, w)
+    assert "tcgen05.streaming" in plan
+    check_int8_attention(got, oracle(w))
+    w = W.mha_bf16(batch=2, heads=2, seq=300, head_dim=64, seed=4)
+    mid = [t for t in w.graph.inputs if w.graph.tensors[t].name == "mask"][0]
+    m = w.feeds[mid].copy()
+    m[m < 0] = -np.inf
+    w.feeds[mid] = m
     got, plan = run_gpu(B, w)
     assert "tcgen05.streaming" in plan
     assert np.abs(bf16_to_f64(got) - oracle(w)).max() <= 2e-2
