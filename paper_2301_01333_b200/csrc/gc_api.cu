@@ -237,6 +237,7 @@ struct SdpaPlan {
   int p_out_pos = -1;        // graph output position of the probabilities tensor, if it is an output too
   bool use_tc = false;
   bool wide = false;         // streaming kernel (wider heads, 512 keys) instead of the D = 64 kernel
+  bool two_pass = false;     // more than 512 keys: blockwise softmax with the scores computed twice
   CUtensorMap tmQ, tmK, tmV, tmO;
   const void *q_ptr = nullptr, *k_ptr = nullptr, *v_ptr = nullptr, *o_ptr = nullptr;
 };
@@ -652,6 +653,11 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
       const size_t need = sdpa_wide_smem_bytes(s.S, s.D, s.is_int8);
       wide = tc = need > 0 && need <= static_cast<size_t>(prop.sharedMemPerBlockOptin);
     }
+    bool two_pass = false;
+    if (!tc && !c->opt.force_generic && s.S > 512 && c->sdpa.p_out_pos < 0) {
+      const size_t need = sdpa_long_smem_bytes(s.S, s.D, s.is_int8);
+      two_pass = wide = tc = need > 0 && need <= static_cast<size_t>(prop.sharedMemPerBlockOptin);
+    }
     if (!s.is_int8 && c->sdpa.p_out_pos >= 0) tc = false;   // the bf16 tcgen05 kernels never form normalised P
     // the probabilities as a second output: written in 16-byte pieces, which needs whole key blocks
     if (c->sdpa.p_out_pos >= 0 && s.S % 128 != 0) tc = false;
@@ -662,6 +668,7 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
     if (!tc && s.S > 8192) return bail(fail(GC_ERR_UNSUPPORTED, "attention: sequence length %d not supported", s.S));
     c->sdpa.use_tc = tc;
     c->sdpa.wide = tc && wide;
+    c->sdpa.two_pass = tc && two_pass;
     c->launches = 1;
     // The paper's max-free softmax, where it is safe: 8-bit operands bound every score at compile time; with
     // |score| log2(e) <= 60 neither an exponential nor a row sum can leave fp32's range, and without a mask no row
@@ -669,7 +676,8 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
     s.max_free = tc && !wide && s.is_int8 && c->sdpa.mask_input < 0 && !c->opt.exact_max_softmax && s.skip_thr > 0.f &&
                  (static_cast<double>(s.skip_thr) - 151.0) * 0.5 <= 60.0;
     snprintf(line, sizeof(line), "pattern=attention %s B=%d H=%d S=%d D=%d kernel=%s%s\n", s.is_int8 ? "int8" : "bf16", s.B,
-             s.H, s.S, s.D, tc ? (wide ? "tcgen05.streaming" : "tcgen05") : "cuda-core", s.max_free ? " softmax=max-free" : "");
+             s.H, s.S, s.D, tc ? (two_pass ? "tcgen05.two-pass" : (wide ? "tcgen05.streaming" : "tcgen05")) : "cuda-core",
+             s.max_free ? " softmax=max-free" : "");
     c->desc = line;
   } else {
     gc_status_t st = match_mlp(*p, *c);
@@ -1274,7 +1282,10 @@ static gc_status_t run_sdpa(gc_compiled& c, cudaStream_t st, const void* const* 
       if (r != GC_OK) return r;
       *cached[i] = ptrs[i];
     }
-    CUDA_TRY(launch_sdpa_wide(s.tmQ, s.tmK, s.tmV, prm, c.num_sms, st));
+    if (s.two_pass)
+      CUDA_TRY(launch_sdpa_long(s.tmQ, s.tmK, s.tmV, prm, c.num_sms, st));
+    else
+      CUDA_TRY(launch_sdpa_wide(s.tmQ, s.tmK, s.tmV, prm, c.num_sms, st));
     return GC_OK;
   }
   const int swz = prm.is_int8 ? 64 : 128;

@@ -185,6 +185,12 @@ cudaError_t launch_gemm_tc2(int kind, int a_signed, const CUtensorMap& tmA, cons
                             const GemmTcParams& p, int grid, bool pdl, cudaStream_t s);
 
 size_t sdpa_tc_smem_bytes(int S, int is_int8);
+// Attention for rows longer than tensor memory holds (kernels_sdpa_long.cu): head dimension 64 / 96 / 128, any number of
+// keys, scores computed twice around a blockwise softmax.  Takes the 3-D tensor maps of the streaming kernel
+// (sdpa_wide_box).  Dynamic shared memory it needs (0 = shape not supported).
+size_t sdpa_long_smem_bytes(int S, int D, int is_int8);
+cudaError_t launch_sdpa_long(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const SdpaParams& p,
+                             int num_sms, cudaStream_t s);
 // Streaming attention kernel (head dimension 64 / 96 / 128, up to 512 keys): dynamic shared memory it needs
 // (0 = shape not supported), the TMA box (elements per row, swizzle bytes) its Q / K / V tensor maps must use
 // (128 rows per box), and the launcher.

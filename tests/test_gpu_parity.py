@@ -414,6 +414,23 @@ def test_mha_ragged_without_a_mask_and_with_minus_infinity(B):
     assert np.abs(bf16_to_f64(got) - oracle(w)).max() <= 2e-2
 
 
+# rows of more than 512 keys do not fit tensor memory next to the output: blockwise softmax with the scores computed
+# twice; several units per CTA on the larger cases (rings and barrier phases wrap), a ragged length, every head width
+LONG_SHAPES = [(1, 2, 640, 64), (1, 2, 1024, 128), (1, 1, 1000, 96), (1, 40, 640, 64), (1, 40, 768, 128), (1, 1, 2048, 64)]
+
+
+@pytest.mark.parametrize("b,h,s,d", LONG_SHAPES)
+@pytest.mark.parametrize("kind", ["bf16", "int8"])
+def test_mha_more_than_512_keys_on_tensor_cores(B, kind, b, h, s, d):
+    w = W.mha_bf16(batch=b, heads=h, seq=s, head_dim=d) if kind == "bf16" else W.mha_int8(batch=b, heads=h, seq=s, head_dim=d)
+    got, plan = run_gpu(B, w)
+    assert "tcgen05.two-pass" in plan
+    if kind == "bf16":
+        assert np.abs(bf16_to_f64(got) - oracle(w)).max() <= 2e-2
+    else:
+        check_int8_attention(got, oracle(w))
+
+
 @pytest.mark.parametrize("b,h,s,d", WIDE_SHAPES)
 def test_mha_int8_streaming_kernel(B, b, h, s, d):
     w = W.mha_int8(batch=b, heads=h, seq=s, head_dim=d)
