@@ -238,6 +238,7 @@ struct SdpaPlan {
   bool use_tc = false;
   bool wide = false;         // streaming kernel (wider heads, 512 keys) instead of the D = 64 kernel
   bool two_pass = false;     // more than 512 keys: blockwise softmax with the scores computed twice
+  bool small = false;        // bf16, 128 keys, width 64: one unit per CTA, several CTAs per SM
   CUtensorMap tmQ, tmK, tmV, tmO;
   const void *q_ptr = nullptr, *k_ptr = nullptr, *v_ptr = nullptr, *o_ptr = nullptr;
 };
@@ -669,6 +670,7 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
     c->sdpa.use_tc = tc;
     c->sdpa.wide = tc && wide;
     c->sdpa.two_pass = tc && two_pass;
+    c->sdpa.small = tc && !wide && c->sdpa.p_out_pos < 0 && sdpa_small_supported(s.S, s.D, s.is_int8);
     c->launches = 1;
     // The paper's max-free softmax, where it is safe: 8-bit operands bound every score at compile time; with
     // |score| log2(e) <= 60 neither an exponential nor a row sum can leave fp32's range, and without a mask no row
@@ -676,7 +678,7 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
     s.max_free = tc && !wide && s.is_int8 && c->sdpa.mask_input < 0 && !c->opt.exact_max_softmax && s.skip_thr > 0.f &&
                  (static_cast<double>(s.skip_thr) - 151.0) * 0.5 <= 60.0;
     snprintf(line, sizeof(line), "pattern=attention %s B=%d H=%d S=%d D=%d kernel=%s%s\n", s.is_int8 ? "int8" : "bf16", s.B,
-             s.H, s.S, s.D, tc ? (two_pass ? "tcgen05.two-pass" : (wide ? "tcgen05.streaming" : "tcgen05")) : "cuda-core",
+             s.H, s.S, s.D, tc ? (two_pass ? "tcgen05.two-pass" : (wide ? "tcgen05.streaming" : (c->sdpa.small ? "tcgen05.unit-per-cta" : "tcgen05"))) : "cuda-core",
              s.max_free ? " softmax=max-free" : "");
     c->desc = line;
   } else {
@@ -1303,6 +1305,10 @@ static gc_status_t run_sdpa(gc_compiled& c, cudaStream_t st, const void* const* 
     gc_status_t r = make_tmap(&s.tmV, prm.V, dt, prm.D, rows, static_cast<uint64_t>(prm.D) * esz, prm.D, 128, swz);
     if (r != GC_OK) return r;
     s.v_ptr = prm.V;
+  }
+  if (s.small) {
+    CUDA_TRY(launch_sdpa_small(s.tmQ, s.tmK, s.tmV, prm, st));
+    return GC_OK;
   }
   if (s.o_ptr != prm.O) {
     gc_status_t r = make_tmap(&s.tmO, prm.O, dt, prm.D, rows, static_cast<uint64_t>(prm.D) * esz, prm.D, 32, prm.D * esz);

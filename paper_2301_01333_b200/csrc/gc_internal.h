@@ -194,6 +194,10 @@ cudaError_t launch_sdpa_long(const CUtensorMap& tmQ, const CUtensorMap& tmK, con
 // Streaming attention kernel (head dimension 64 / 96 / 128, up to 512 keys): dynamic shared memory it needs
 // (0 = shape not supported), the TMA box (elements per row, swizzle bytes) its Q / K / V tensor maps must use
 // (128 rows per box), and the launcher.
+// One unit per CTA, several CTAs per SM (kernels_sdpa_small.cu): bf16, 128 keys, head width 64.
+bool sdpa_small_supported(int S, int D, int is_int8);
+cudaError_t launch_sdpa_small(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const SdpaParams& p,
+                              cudaStream_t s);
 size_t sdpa_wide_smem_bytes(int S, int D, int is_int8);
 void sdpa_wide_box(int D, int is_int8, int* box_elems, int* swizzle_bytes);
 cudaError_t launch_sdpa_wide(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const SdpaParams& p,

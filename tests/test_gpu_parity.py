@@ -365,6 +365,22 @@ def test_mha_bf16(B, b, h, s, d):
     assert np.abs(bf16_to_f64(got) - oracle(w)).max() <= 2e-2
 
 
+@pytest.mark.parametrize("b,h,valid", [(32, 12, None), (1, 1, None), (50, 12, None), (3, 5, (1, 128)), (2, 4, (0, 40))])
+def test_mha_bf16_one_unit_per_cta(B, b, h, valid):
+    # 128 keys, head width 64: one (batch, head) unit per CTA, three CTAs per SM.  600 units are more than the 444 that
+    # are resident at once (a second wave); padding masks from a single valid key up, and rows whose mask is minus
+    # infinity for most keys
+    kw = {} if valid is None else {"valid_lo": valid[0], "valid_hi": valid[1]}
+    w = W.mha_bf16(batch=b, heads=h, seq=128, head_dim=64, seed=b + h, **kw)
+    if valid == (0, 40):
+        mask = w.feeds[w.graph.inputs[3]]
+        mask[mask < 0] = -np.inf
+        mask[..., :1] = 0.0                                     # every row keeps one key
+    got, plan = run_gpu(B, w)
+    assert "tcgen05.unit-per-cta" in plan
+    assert np.abs(bf16_to_f64(got) - oracle(w)).max() <= 2e-2
+
+
 # the other head dimensions and sequence lengths of the evaluation's workload table, on the streaming kernel;
 # the larger cases give every CTA more than one work unit, so the rings and barrier phases wrap
 WIDE_SHAPES = [(1, 2, 128, 96), (1, 2, 384, 128), (1, 2, 512, 64), (2, 1, 256, 128), (1, 1, 512, 128), (1, 1, 256, 96),
