@@ -40,10 +40,13 @@ DTYPE = {"c1": "tf32", "c2": "u8xs8->s32", "c3": "bf16", "c4": "u8xu8->s32", "c5
 # was measured in) and the clock sampler sees the timed region
 DEFAULT_STEPS = {"c1": 2000, "c2": 2000, "c3": 500, "c4": 100, "c5": 8000}
 GRAPH_STEPS = {"c1": 256, "c2": 256, "c3": 256, "c4": 50, "c5": 50}     # executes captured into one CUDA graph
-# DRAM bytes per launch of the dominant kernel from the ncu capture summarised under profiles/
-# (dram__bytes_read.sum + dram__bytes_write.sum; c5: one launch per step, the 64 MiB hidden tensor is written back)
-TRAFFIC_BYTES_PER_LAUNCH = {"c5": 117.4e6, "c3": None, "c4": 84.8e6}
-DOMINANT_KERNEL = {"c1": "mlp_chain_kernel<tf32>", "c2": "mlp_chain_kernel<i8>", "c3": "sdpa_tc_kernel<bf16>",
+# DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum) from the newest ncu
+# capture of each, which TRAFFIC_SOURCE names; a profiler figure cannot be re-measured inside an untimed run, so the
+# line carries the capture it comes from.  c5: one launch per step, the 64 MiB hidden tensor is written back.
+TRAFFIC_BYTES_PER_LAUNCH = {"c5": 126.65e6, "c3": 18.9e6, "c4": 84.8e6}
+TRAFFIC_SOURCE = {"c5": "profiles/gemm_tc2_bf16_c5_ffn_one_launch.md (capture of the one-launch FFN, 70.0 MB read + 56.7 MB written)",
+                  "c3": "profiles/sdpa_small_c3_attention.md (reads; the 6.3 MB of output were still in the L2 when the launch ended)", "c4": "profiles/sdpa_tc_c3_c4_attention.md"}
+DOMINANT_KERNEL = {"c1": "mlp_chain_kernel<tf32>", "c2": "mlp_chain_kernel<i8>", "c3": "sdpa_small_kernel (bf16, one unit per CTA)",
                    "c4": "sdpa_tc_kernel<int8>", "c5": "gemm_tc2_kernel<bf16, bf16 out> (both FFN GEMMs in one launch)"}
 
 
@@ -568,7 +571,7 @@ def main():
         peak = exp_peak_per_s(sm_max_mhz) / 1e12
         achieved = hr["scores"] / (us * 1e-6) / 1e12
         roof = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "Texp/s", "frac": achieved / peak,
-                "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(head),
+                "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(head), "traffic_source": TRAFFIC_SOURCE.get(head),
                 "peak_source": "derived: 148 SMs x 16 ex2 per clock x 1965 MHz (one exponential per attention score)",
                 "kernel": DOMINANT_KERNEL[head], "launches_per_step": n_launch, "avg_launch_us": us / n_launch,
                 "hbm_frac_measured_peak": hr["roofline_frac_measured_peak"]}
@@ -576,7 +579,7 @@ def main():
         peak = peaks.get(head_peak_key, 1590.0) * KIND_RATIO[head]
         achieved = head_w.ops / (us * 1e-6) / 1e12
         roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s" if "FLOP" in UNIT[head] else "TOP/s",
-                "frac": achieved / peak, "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(head),
+                "frac": achieved / peak, "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(head), "traffic_source": TRAFFIC_SOURCE.get(head),
                 "peak_source": f"{peak_src} cuBLAS {head_peak_key} (timed region {head_ms:.0f} ms) x kind ratio {KIND_RATIO[head]}",
                 "kernel": DOMINANT_KERNEL[head], "launches_per_step": n_launch, "avg_launch_us": us / n_launch,
                 "algorithmic_flops_per_launch": head_w.ops / n_launch,
@@ -585,7 +588,7 @@ def main():
     else:
         achieved = head_w.bytes / (us * 1e-6) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(head), "peak_source": peak_src, "kernel": DOMINANT_KERNEL[head],
+                "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(head), "traffic_source": TRAFFIC_SOURCE.get(head), "peak_source": peak_src, "kernel": DOMINANT_KERNEL[head],
                 "launches_per_step": n_launch, "avg_launch_us": us / n_launch,
                 "algorithmic_bytes_per_launch": head_w.bytes / n_launch}
     cpu = None
