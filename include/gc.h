@@ -189,6 +189,25 @@ gc_status_t gc_set_host_staging(gc_compiled_t* c, void* staging_dev, size_t byte
 gc_status_t gc_execute_host(gc_compiled_t* c, void* cuda_stream, const void* const* in_host,
                             int32_t n_in, void* const* out_host, int32_t n_out);
 
+/* No counterpart in the paper (its tensors live in host memory already): the same computation with
+ * HOST buffers, but asynchronous, so that the copies of consecutive batches overlap each other and
+ * the execution.  The staging area set by gc_set_host_staging holds one slot per multiple of
+ * gc_host_staging_bytes (at most GC_HOST_SLOTS; three keep both copy directions busy when a batch
+ * spends about as long in each copy as in the execution).  The call enqueues, for staging slot
+ * `slot` (0 .. slots - 1): the
+ * host-to-device copies of the non-constant inputs on a copy stream the object owns, the execute
+ * on cuda_stream behind them, and the device-to-host copies of the outputs on a second copy stream
+ * behind the execute; then it returns.  gc_host_wait(c, slot) blocks until that slot's outputs
+ * have arrived in out_host; the host buffers must stay valid and untouched until then, and should
+ * be page-locked (with pageable memory the copies are correct but do not overlap).  A slot that is
+ * still in flight is refused with GC_ERR_STATE; constants are copied once, as in gc_execute_host,
+ * and shared by both slots.  All calls on one object use the same cuda_stream. */
+#define GC_HOST_SLOTS 4
+gc_status_t gc_execute_host_async(gc_compiled_t* c, void* cuda_stream, int32_t slot,
+                                  const void* const* in_host, int32_t n_in, void* const* out_host,
+                                  int32_t n_out);
+gc_status_t gc_host_wait(gc_compiled_t* c, int32_t slot);
+
 /* No counterpart in the paper (its CPU kernels cannot time out).  Synchronise the stream and read
  * the device status word: GC_OK, GC_ERR_TIMEOUT (a bounded device-side wait expired) or
  * GC_ERR_CUDA (the stream reported an error).  A kernel that gave up leaves its synchronisation

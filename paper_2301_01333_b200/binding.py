@@ -32,6 +32,7 @@ NP_DTYPE = {"f32": np.float32, "bf16": np.uint16, "u8": np.uint8, "s8": np.int8,
 EXPORTS = [
     "gc_partition_create", "gc_partition_destroy", "gc_compile", "gc_compiled_destroy", "gc_workspace_bytes",
     "gc_set_workspace", "gc_execute", "gc_host_staging_bytes", "gc_set_host_staging", "gc_execute_host",
+    "gc_execute_host_async", "gc_host_wait",
     "gc_query_status", "gc_launches_per_execute", "gc_plan_description", "gc_last_error", "gc_version",
     "gc_matmul_s32_noalloc", "gc_noalloc_scratch_bytes", "gc_selftest_bounded_wait", "gc_invalidate_constants",
 ]
@@ -85,6 +86,8 @@ def load_library() -> C.CDLL:
     lib.gc_host_staging_bytes.argtypes = [vp, C.POINTER(sz)]
     lib.gc_set_host_staging.argtypes = [vp, vp, sz]
     lib.gc_execute_host.argtypes = [vp, vp, C.POINTER(vp), i32, C.POINTER(vp), i32]
+    lib.gc_execute_host_async.argtypes = [vp, vp, i32, C.POINTER(vp), i32, C.POINTER(vp), i32]
+    lib.gc_host_wait.argtypes = [vp, i32]
     lib.gc_query_status.argtypes = [vp, vp]
     lib.gc_launches_per_execute.argtypes = [vp, C.POINTER(i32)]
     lib.gc_plan_description.argtypes = [vp]
@@ -99,8 +102,8 @@ def load_library() -> C.CDLL:
     lib.gc_selftest_bounded_wait.argtypes = [vp, vp, C.c_uint32]
     lib.gc_selftest_bounded_wait.restype = i32
     for name in ("gc_partition_create", "gc_compile", "gc_workspace_bytes", "gc_set_workspace", "gc_execute",
-                 "gc_host_staging_bytes", "gc_set_host_staging", "gc_execute_host", "gc_query_status",
-                 "gc_launches_per_execute"):
+                 "gc_host_staging_bytes", "gc_set_host_staging", "gc_execute_host", "gc_execute_host_async",
+                 "gc_host_wait", "gc_query_status", "gc_launches_per_execute"):
         getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -217,6 +220,15 @@ def gc_execute_host(c, stream: int, in_ptrs: Sequence[int], out_ptrs: Sequence[i
                                           _ptr_array(out_ptrs), len(out_ptrs)))
 
 
+def gc_execute_host_async(c, stream: int, slot: int, in_ptrs: Sequence[int], out_ptrs: Sequence[int]) -> None:
+    _check(load_library().gc_execute_host_async(c, C.c_void_p(stream), slot, _ptr_array(in_ptrs), len(in_ptrs),
+                                                _ptr_array(out_ptrs), len(out_ptrs)))
+
+
+def gc_host_wait(c, slot: int) -> None:
+    _check(load_library().gc_host_wait(c, slot))
+
+
 def gc_query_status(c, stream: int = 0) -> None:
     _check(load_library().gc_query_status(c, C.c_void_p(stream)))
 
@@ -329,6 +341,28 @@ class CompiledPartition:
         if stream is None:
             stream = torch.cuda.current_stream(self.device).cuda_stream
         gc_execute_host(self._comp, stream, [_host_ptr(a) for a in in_arrays], [_host_ptr(a) for a in out_arrays])
+
+    HOST_SLOTS = 3
+
+    def execute_host_async(self, slot: int, in_arrays: List[np.ndarray], out_arrays: List[np.ndarray],
+                           stream: Optional[int] = None):
+        """Enqueue copies in, execute and copies out for staging slot 0 .. HOST_SLOTS - 1 and return; host_wait(slot)
+        completes it.  Several slots in flight overlap the copies of one batch with the execution and the copies of
+        its neighbours."""
+        import torch
+        n = gc_host_staging_bytes(self._comp)
+        if self._staging is None or self._staging.numel() < self.HOST_SLOTS * n:
+            for s in range(self.HOST_SLOTS):
+                self.host_wait(s)
+            self._staging = torch.empty(max(self.HOST_SLOTS * n, 256), dtype=torch.uint8, device=f"cuda:{self.device}")
+            gc_set_host_staging(self._comp, self._staging.data_ptr(), self._staging.numel())
+        if stream is None:
+            stream = torch.cuda.current_stream(self.device).cuda_stream
+        gc_execute_host_async(self._comp, stream, slot, [_host_ptr(a) for a in in_arrays],
+                              [_host_ptr(a) for a in out_arrays])
+
+    def host_wait(self, slot: int) -> None:
+        gc_host_wait(self._comp, slot)
 
     def close(self) -> None:
         if getattr(self, "_comp", None):

@@ -275,6 +275,12 @@ struct gc_compiled {
   void* staging = nullptr;
   std::vector<size_t> in_stage_off, out_stage_off;
   std::vector<const void*> host_const_seen;
+  // overlapped host execution: up to GC_HOST_SLOTS staging slots, copy streams of their own, one event triple per slot
+  int staging_slots = 0;
+  bool pipe_ready = false;
+  cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
+  cudaEvent_t ev_in[GC_HOST_SLOTS] = {}, ev_exec[GC_HOST_SLOTS] = {}, ev_out[GC_HOST_SLOTS] = {};
+  bool slot_busy[GC_HOST_SLOTS] = {};
 };
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -1004,7 +1010,20 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
   return GC_OK;
 }
 
-extern "C" void gc_compiled_destroy(gc_compiled_t* c) { delete c; }
+extern "C" void gc_compiled_destroy(gc_compiled_t* c) {
+  if (!c) return;
+  if (c->pipe_ready) {
+    for (int s = 0; s < GC_HOST_SLOTS; ++s) {
+      if (c->slot_busy[s]) cudaEventSynchronize(c->ev_out[s]);
+      cudaEventDestroy(c->ev_in[s]);
+      cudaEventDestroy(c->ev_exec[s]);
+      cudaEventDestroy(c->ev_out[s]);
+    }
+    cudaStreamDestroy(c->h2d_stream);
+    cudaStreamDestroy(c->d2h_stream);
+  }
+  delete c;
+}
 
 extern "C" gc_status_t gc_workspace_bytes(const gc_compiled_t* c, size_t* bytes) {
   if (!c || !bytes) return fail(GC_ERR_INVALID_ARG, "null argument");
@@ -1038,7 +1057,10 @@ extern "C" gc_status_t gc_set_host_staging(gc_compiled_t* c, void* p, size_t byt
   if (!c || !p) return fail(GC_ERR_INVALID_ARG, "null argument");
   if (bytes < c->staging_bytes) return fail(GC_ERR_INVALID_ARG, "staging area too small");
   if (reinterpret_cast<uintptr_t>(p) % 256) return fail(GC_ERR_ALIGNMENT, "staging area must be 256-byte aligned");
+  for (int s = 0; s < GC_HOST_SLOTS; ++s)
+    if (c->slot_busy[s]) return fail(GC_ERR_STATE, "a host execute is still in flight: call gc_host_wait first");
   c->staging = p;
+  c->staging_slots = c->staging_bytes ? static_cast<int>(std::min<size_t>(GC_HOST_SLOTS, bytes / c->staging_bytes)) : 1;
   std::fill(c->host_const_seen.begin(), c->host_const_seen.end(), nullptr);
   return GC_OK;
 }
@@ -1368,35 +1390,105 @@ extern "C" gc_status_t gc_execute(gc_compiled_t* c, void* cuda_stream, const voi
   return r;
 }
 
+// Enqueue one host-buffer execute on staging slot `slot`: inputs -> slot (on `in_st`), execute (on `st`), slot -> host
+// (on `out_st`).  With in_st == st == out_st everything is ordered by the stream alone; otherwise the three are chained
+// by the slot's events.  The constants live in slot 0 only (one device address, so the prepack cache stays valid).
+static gc_status_t host_enqueue(gc_compiled_t* c, cudaStream_t st, cudaStream_t in_st, cudaStream_t out_st, int slot,
+                                const void* const* in_host, int32_t n_in, void* const* out_host, int32_t n_out) {
+  char* base0 = static_cast<char*>(c->staging);
+  char* sg = base0 + static_cast<size_t>(slot) * c->staging_bytes;
+  std::vector<const void*> din(n_in);
+  std::vector<void*> dout(n_out);
+  for (int i = 0; i < n_in; ++i)
+    if (!in_host[i]) return fail(GC_ERR_INVALID_ARG, "input %d is null", i);
+  for (int i = 0; i < n_out; ++i)
+    if (!out_host[i]) return fail(GC_ERR_INVALID_ARG, "output %d is null", i);
+  for (int i = 0; i < n_in; ++i) {
+    if (c->in_constant[i]) {
+      din[i] = base0 + c->in_stage_off[i];
+      if (c->host_const_seen[i] != in_host[i]) {
+        CUDA_TRY(cudaMemcpyAsync(base0 + c->in_stage_off[i], in_host[i], c->in_bytes[i], cudaMemcpyHostToDevice, st));
+        // A constant that arrives at a new host address lands at the same staging address: forget the device
+        // pointer recorded at the last prepack, so that the execute below preprocesses the new contents.
+        if (c->host_const_seen[i] != nullptr) c->const_ptrs[i] = nullptr;
+        c->host_const_seen[i] = in_host[i];
+      }
+    } else {
+      din[i] = sg + c->in_stage_off[i];
+      CUDA_TRY(cudaMemcpyAsync(sg + c->in_stage_off[i], in_host[i], c->in_bytes[i], cudaMemcpyHostToDevice, in_st));
+    }
+  }
+  if (in_st != st) {
+    CUDA_TRY(cudaEventRecord(c->ev_in[slot], in_st));
+    CUDA_TRY(cudaStreamWaitEvent(st, c->ev_in[slot], 0));
+  }
+  for (int i = 0; i < n_out; ++i) dout[i] = sg + c->out_stage_off[i];
+  gc_status_t r = gc_execute(c, st, din.data(), n_in, dout.data(), n_out);
+  if (r != GC_OK) return r;
+  if (out_st != st) {
+    CUDA_TRY(cudaEventRecord(c->ev_exec[slot], st));
+    CUDA_TRY(cudaStreamWaitEvent(out_st, c->ev_exec[slot], 0));
+  }
+  for (int i = 0; i < n_out; ++i)
+    CUDA_TRY(cudaMemcpyAsync(out_host[i], sg + c->out_stage_off[i], c->out_bytes[i], cudaMemcpyDeviceToHost, out_st));
+  return GC_OK;
+}
+
 extern "C" gc_status_t gc_execute_host(gc_compiled_t* c, void* cuda_stream, const void* const* in_host, int32_t n_in,
                                        void* const* out_host, int32_t n_out) {
   if (!c || !in_host || !out_host) return fail(GC_ERR_INVALID_ARG, "null argument");
   if (n_in != c->n_in || n_out != c->n_out) return fail(GC_ERR_INVALID_ARG, "wrong number of inputs or outputs");
   if (!c->staging) return fail(GC_ERR_STATE, "gc_set_host_staging has not been called");
+  if (c->slot_busy[0]) return fail(GC_ERR_STATE, "staging slot 0 is in flight: call gc_host_wait first");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  char* sg = static_cast<char*>(c->staging);
-  std::vector<const void*> din(n_in);
-  std::vector<void*> dout(n_out);
-  for (int i = 0; i < n_in; ++i) {
-    if (!in_host[i]) return fail(GC_ERR_INVALID_ARG, "input %d is null", i);
-    din[i] = sg + c->in_stage_off[i];
-    if (!c->in_constant[i] || c->host_const_seen[i] != in_host[i]) {
-      CUDA_TRY(cudaMemcpyAsync(sg + c->in_stage_off[i], in_host[i], c->in_bytes[i], cudaMemcpyHostToDevice, st));
-      // A constant that arrives at a new host address lands at the same staging address: forget the device
-      // pointer recorded at the last prepack, so that the execute below preprocesses the new contents.
-      if (c->in_constant[i] && c->host_const_seen[i] != nullptr) c->const_ptrs[i] = nullptr;
-      c->host_const_seen[i] = in_host[i];
-    }
-  }
-  for (int i = 0; i < n_out; ++i) {
-    if (!out_host[i]) return fail(GC_ERR_INVALID_ARG, "output %d is null", i);
-    dout[i] = sg + c->out_stage_off[i];
-  }
-  gc_status_t r = gc_execute(c, cuda_stream, din.data(), n_in, dout.data(), n_out);
+  gc_status_t r = host_enqueue(c, st, st, st, 0, in_host, n_in, out_host, n_out);
   if (r != GC_OK) return r;
-  for (int i = 0; i < n_out; ++i)
-    CUDA_TRY(cudaMemcpyAsync(out_host[i], sg + c->out_stage_off[i], c->out_bytes[i], cudaMemcpyDeviceToHost, st));
   CUDA_TRY(cudaStreamSynchronize(st));
+  return GC_OK;
+}
+
+extern "C" gc_status_t gc_execute_host_async(gc_compiled_t* c, void* cuda_stream, int32_t slot, const void* const* in_host,
+                                             int32_t n_in, void* const* out_host, int32_t n_out) {
+  if (!c || !in_host || !out_host) return fail(GC_ERR_INVALID_ARG, "null argument");
+  if (n_in != c->n_in || n_out != c->n_out) return fail(GC_ERR_INVALID_ARG, "wrong number of inputs or outputs");
+  if (!c->staging) return fail(GC_ERR_STATE, "gc_set_host_staging has not been called");
+  if (slot < 0 || slot >= c->staging_slots)
+    return fail(GC_ERR_INVALID_ARG, "slot %d: the staging area holds %d slot(s) of gc_host_staging_bytes each", slot,
+                c->staging_slots);
+  if (c->slot_busy[slot]) return fail(GC_ERR_STATE, "slot %d is still in flight: call gc_host_wait first", slot);
+  int cur = -1;
+  CUDA_TRY(cudaGetDevice(&cur));
+  if (cur != c->device) CUDA_TRY(cudaSetDevice(c->device));
+  if (!c->pipe_ready) {
+    CUDA_TRY(cudaStreamCreateWithFlags(&c->h2d_stream, cudaStreamNonBlocking));
+    CUDA_TRY(cudaStreamCreateWithFlags(&c->d2h_stream, cudaStreamNonBlocking));
+    for (int s = 0; s < GC_HOST_SLOTS; ++s) {
+      CUDA_TRY(cudaEventCreateWithFlags(&c->ev_in[s], cudaEventDisableTiming));
+      CUDA_TRY(cudaEventCreateWithFlags(&c->ev_exec[s], cudaEventDisableTiming));
+      CUDA_TRY(cudaEventCreateWithFlags(&c->ev_out[s], cudaEventDisableTiming));
+    }
+    c->pipe_ready = true;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  gc_status_t r = host_enqueue(c, st, c->h2d_stream, c->d2h_stream, slot, in_host, n_in, out_host, n_out);
+  if (r != GC_OK) {
+    // whatever was enqueued before the failure must not outlive the caller's buffers
+    cudaStreamSynchronize(c->h2d_stream);
+    cudaStreamSynchronize(st);
+    cudaStreamSynchronize(c->d2h_stream);
+    return r;
+  }
+  CUDA_TRY(cudaEventRecord(c->ev_out[slot], c->d2h_stream));
+  c->slot_busy[slot] = true;
+  return GC_OK;
+}
+
+extern "C" gc_status_t gc_host_wait(gc_compiled_t* c, int32_t slot) {
+  if (!c) return fail(GC_ERR_INVALID_ARG, "null argument");
+  if (slot < 0 || slot >= GC_HOST_SLOTS) return fail(GC_ERR_INVALID_ARG, "slot %d out of range", slot);
+  if (!c->slot_busy[slot]) return GC_OK;
+  c->slot_busy[slot] = false;
+  CUDA_TRY(cudaEventSynchronize(c->ev_out[slot]));
   return GC_OK;
 }
 

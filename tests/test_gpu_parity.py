@@ -791,6 +791,52 @@ def test_host_buffer_entry_point_matches_device_entry_point(B):
     torch.cuda.synchronize()
 
 
+def test_overlapped_host_entry_point_batches_in_flight(B):
+    # different activations per staging slot, the constants shared; each slot's result must be its own batch's
+    import torch
+    ws = []
+    for s in range(7):
+        w = W.mlp_int8(batch=128, dims=(479, 256, 64, 1), seed=1)      # same weights, own activations
+        x = w.graph.inputs[0]
+        w.feeds[x] = np.random.default_rng(100 + s).integers(0, 256, size=w.feeds[x].shape).astype(np.uint8)
+        ws.append(w)
+    g = ws[0].graph
+    c = B.CompiledPartition(g, 0)
+    ns = c.HOST_SLOTS
+    assert 2 <= ns < len(ws)
+    refs = [interp.run(w.graph, w.feeds)[w.graph.outputs[0]] for w in ws]
+    assert not np.array_equal(refs[0], refs[1])
+    consts = [np.ascontiguousarray(ws[0].feeds[t]) for t in g.inputs[1:]]
+    pinned_in = [torch.empty(ws[0].feeds[g.inputs[0]].nbytes, dtype=torch.uint8).pin_memory() for _ in range(ns)]
+    pinned_out = [torch.empty(g.tensors[g.outputs[0]].nbytes, dtype=torch.uint8).pin_memory() for _ in range(ns)]
+    got = [None] * len(ws)
+
+    def collect(i):
+        c.host_wait(i % ns)
+        got[i] = pinned_out[i % ns].numpy().view(np.float32).reshape(refs[i].shape).copy()
+
+    for i, w in enumerate(ws):
+        if i >= ns:
+            collect(i - ns)
+        pinned_in[i % ns].numpy()[:] = np.ascontiguousarray(w.feeds[g.inputs[0]]).view(np.uint8).reshape(-1)
+        c.execute_host_async(i % ns, [pinned_in[i % ns]] + consts, [pinned_out[i % ns]])
+    # a slot in flight is refused, and so is a slot the staging area does not have
+    with pytest.raises(B.GcError):
+        c.execute_host_async((len(ws) - 1) % ns, [pinned_in[0]] + consts, [pinned_out[0]])
+    with pytest.raises(B.GcError):
+        c.execute_host_async(ns, [pinned_in[0]] + consts, [pinned_out[0]])
+    for i in range(len(ws) - ns, len(ws)):
+        collect(i)
+    for i in range(len(ws)):
+        assert np.abs(got[i] - refs[i]).max() <= 2e-6, i
+    # the synchronous call still works on the same object afterwards
+    out = np.zeros(refs[0].shape, dtype=np.float32)
+    c.execute_host([np.ascontiguousarray(ws[3].feeds[g.inputs[0]])] + consts, [out])
+    assert np.array_equal(out, got[3])
+    c.close()
+    torch.cuda.synchronize()
+
+
 def test_host_buffer_entry_point_picks_up_a_constant_at_a_new_host_address(B):
     # a constant that arrives at a new host address is copied to the same staging address: the weights must be
     # preprocessed again, not only the bias re-read
