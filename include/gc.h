@@ -136,7 +136,11 @@ typedef struct {
                              block without a mask whose scores are bounded at compile time (|score| * log2(e) <= 60,
                              from the operand ranges and the folded scales) skips it: the "fast softmax" of
                              Section VII, equal in exact arithmetic (ablation) */
-  int32_t reserved[4];
+  int32_t grid_wide_chain;     /* 1: a small fp32 MLP chain that would run inside one thread-block cluster
+                             (activations handed over through distributed shared memory) runs on the
+                             grid-wide chain kernel instead (hand-over through the L2 behind a grid barrier;
+                             ablation) */
+  int32_t reserved[3];
 } gc_compile_options_t;
 
 typedef struct gc_partition gc_partition_t;

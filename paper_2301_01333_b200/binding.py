@@ -51,7 +51,7 @@ class gc_op_t(C.Structure):
 
 class gc_compile_options_t(C.Structure):
     _fields_ = [("force_generic", C.c_int32), ("no_chain_fusion", C.c_int32), ("streaming_attention", C.c_int32),
-                ("exact_max_softmax", C.c_int32), ("reserved", C.c_int32 * 4)]
+                ("exact_max_softmax", C.c_int32), ("grid_wide_chain", C.c_int32), ("reserved", C.c_int32 * 3)]
 
 
 class GcError(RuntimeError):
@@ -170,13 +170,15 @@ def gc_partition_destroy(p) -> None:
 
 
 def gc_compile(p, cuda_device: int = 0, force_generic: bool = False, no_chain_fusion: bool = False,
-               streaming_attention: bool = False, exact_max_softmax: bool = False) -> C.c_void_p:
+               streaming_attention: bool = False, exact_max_softmax: bool = False,
+               grid_wide_chain: bool = False) -> C.c_void_p:
     lib = load_library()
     opt = gc_compile_options_t()
     opt.force_generic = int(force_generic)
     opt.no_chain_fusion = int(no_chain_fusion)
     opt.streaming_attention = int(streaming_attention)
     opt.exact_max_softmax = int(exact_max_softmax)
+    opt.grid_wide_chain = int(grid_wide_chain)
     h = C.c_void_p()
     _check(lib.gc_compile(p, cuda_device, C.byref(opt), C.byref(h)))
     return h
@@ -268,14 +270,14 @@ class CompiledPartition:
     """Convenience owner: partition + compiled object + torch-allocated workspace."""
 
     def __init__(self, g: Graph, device: int = 0, force_generic: bool = False, no_chain_fusion: bool = False,
-                 streaming_attention: bool = False, exact_max_softmax: bool = False):
+                 streaming_attention: bool = False, exact_max_softmax: bool = False, grid_wide_chain: bool = False):
         import torch
         self.graph = g
         self.device = device
         self._part = gc_partition_create(g)
         try:
             self._comp = gc_compile(self._part, device, force_generic, no_chain_fusion, streaming_attention,
-                                    exact_max_softmax)
+                                    exact_max_softmax, grid_wide_chain)
         except Exception:
             gc_partition_destroy(self._part)
             self._part = None

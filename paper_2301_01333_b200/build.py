@@ -13,7 +13,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgc_b200.so")
-SOURCES = ["gc_api.cu", "gc_noalloc.cu", "kernels_generic.cu", "kernels_gemm_tc.cu", "kernels_gemm_tc2.cu", "kernels_chain.cu",
+SOURCES = ["gc_api.cu", "gc_noalloc.cu", "kernels_generic.cu", "kernels_gemm_tc.cu", "kernels_gemm_tc2.cu", "kernels_chain.cu", "kernels_chain_cluster.cu",
            "kernels_sdpa_tc.cu", "kernels_sdpa_wide.cu", "kernels_sdpa_long.cu", "kernels_sdpa_small.cu"]
 HEADERS = ["gc_internal.h", "ptx.cuh", "epilogue.cuh", "gemm_epilogue.cuh", os.path.join("..", "..", "include", "gc.h")]
 NVCC_FLAGS = [

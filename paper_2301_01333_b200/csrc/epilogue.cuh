@@ -93,22 +93,10 @@ __device__ __forceinline__ void epi_load_cols16(EpiCols16& k, int n0, const Epil
   }
 }
 
-// Store 16 consecutive outputs of one row (columns n0..n0+15) from 16 raw accumulator words.
-// `dst_row` points at column 0 of the row; n0 is a multiple of 16 and the row pitch keeps 16-byte
-// alignment of (dst_row + n0) for every supported dtype.
-__device__ __forceinline__ void epi_store16_cols(const uint32_t* raw, void* dst_row, int n0, const Epilogue& e,
-                                                 const EpiCols16& k) {
-  if (e.acc_is_int && !e.has_dq) {   // raw s32 accumulators (zero-point compensation is exact in s32)
-    int4* d = reinterpret_cast<int4*>(static_cast<int*>(dst_row) + n0);
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-      d[i] = make_int4(static_cast<int>(raw[4 * i]) - k.c[4 * i], static_cast<int>(raw[4 * i + 1]) - k.c[4 * i + 1],
-                       static_cast<int>(raw[4 * i + 2]) - k.c[4 * i + 2], static_cast<int>(raw[4 * i + 3]) - k.c[4 * i + 3]);
-    return;
-  }
+// The 16 values after dequantisation, bias and activation (fp32, before any conversion to the output type).
+__device__ __forceinline__ void epi_values16(const uint32_t* raw, float (&t)[16], const Epilogue& e, const EpiCols16& k) {
   const bool has_bias = e.bias != nullptr, acc_int = e.acc_is_int != 0;
   const int act = e.act;
-  float t[16];
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
     float x = acc_int ? __fmul_rn(__int2float_rn(static_cast<int>(raw[i]) - k.c[i]), k.dq[i]) : __uint_as_float(raw[i]);
@@ -122,6 +110,23 @@ __device__ __forceinline__ void epi_store16_cols(const uint32_t* raw, void* dst_
 #pragma unroll
     for (int i = 0; i < 16; ++i) t[i] = apply_act(t[i], act);
   }
+}
+
+// Store 16 consecutive outputs of one row (columns n0..n0+15) from 16 raw accumulator words.
+// `dst_row` points at column 0 of the row; n0 is a multiple of 16 and the row pitch keeps 16-byte
+// alignment of (dst_row + n0) for every supported dtype.
+__device__ __forceinline__ void epi_store16_cols(const uint32_t* raw, void* dst_row, int n0, const Epilogue& e,
+                                                 const EpiCols16& k) {
+  if (e.acc_is_int && !e.has_dq) {   // raw s32 accumulators (zero-point compensation is exact in s32)
+    int4* d = reinterpret_cast<int4*>(static_cast<int*>(dst_row) + n0);
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      d[i] = make_int4(static_cast<int>(raw[4 * i]) - k.c[4 * i], static_cast<int>(raw[4 * i + 1]) - k.c[4 * i + 1],
+                       static_cast<int>(raw[4 * i + 2]) - k.c[4 * i + 2], static_cast<int>(raw[4 * i + 3]) - k.c[4 * i + 3]);
+    return;
+  }
+  float t[16];
+  epi_values16(raw, t, e, k);
   if (e.out_dtype == GC_F32) {
     float4* d = reinterpret_cast<float4*>(static_cast<float*>(dst_row) + n0);
 #pragma unroll

@@ -270,6 +270,9 @@ struct gc_compiled {
   std::vector<CUtensorMap> chain_tmaps;      // host copy of the tensor-map array
   const void* chain_a0_ptr = nullptr;        // first-layer A pointer the array was built for
   bool chain_tmaps_valid = false;
+  // the same chain inside one thread-block cluster (small fp32 chains)
+  int chain_cluster = 0;                     // cluster size (0: the grid-wide kernel)
+  std::vector<int> chain_ks_l, chain_rows_per;
   // host staging
   size_t staging_bytes = 0;
   void* staging = nullptr;
@@ -832,6 +835,62 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
                max_ctas * ks * row_tiles, ks, w_smem / 1024, c->chain_barriers);
       c->desc += line;
     }
+    // The smallest fp32 chains fit ONE thread-block cluster: weights of every layer resident in its CTAs, activations
+    // handed from layer to layer through distributed shared memory (no grid barrier, no round trip through the L2).
+    // Layer l uses slices_l = N_l / 32 column slices times ks_l parts of the reduction axis.
+    if (ok && kind == 2 && row_tiles == 1 && !c->opt.grid_wide_chain) {
+      bool fit = c->layers[0].M <= 64;
+      int max_slices = 0;
+      for (const LayerPlan& L : c->layers) {
+        fit = fit && L.use_tc && L.N % 32 == 0 && L.N / 32 <= 16 && L.epi.out_dtype == GC_F32 && !L.epi.acc_is_int;
+        max_slices = std::max(max_slices, L.N / 32);
+      }
+      const int C = max_slices > 8 ? 16 : 8;
+      const int rows_pad = (c->layers[0].M + 7) / 8 * 8;
+      std::vector<int> ks_l(c->layers.size(), 1), rows_per(c->layers.size(), rows_pad);
+      std::vector<uint32_t> w_off(c->layers.size(), 0);
+      uint32_t cw = 0;
+      int stages = 1, stage_rows = rows_pad;
+      for (size_t l = 0; fit && l < c->layers.size(); ++l) {
+        const LayerPlan& L = c->layers[l];
+        int ks = 1;
+        while (ks < 4 && 2 * ks * (L.N / 32) <= C && 2 * ks <= L.nkb) ks *= 2;
+        ks_l[l] = ks;
+        rows_per[l] = ((rows_pad + ks - 1) / ks + 7) / 8 * 8;
+        fit = rows_per[l] <= 64;                                  // two finishing threads per row, 128 of them
+        stage_rows = std::max(stage_rows, ks * rows_per[l]);
+        const int my_nkb = (L.nkb + ks - 1) / ks;
+        stages = std::max(stages, my_nkb);
+        w_off[l] = cw;
+        cw += static_cast<uint32_t>(my_nkb) * 32 * 128;
+      }
+      size_t csmem = 0;
+      if (fit) {
+        csmem = mlp_cluster_smem_bytes(cw, stages, stage_rows * 128);
+        fit = csmem <= static_cast<size_t>(prop.sharedMemPerBlockOptin);
+      }
+      if (fit && cuda_device != GC_DEVICE_PLAN_ONLY) {
+        int cur = -1;
+        cudaGetDevice(&cur);
+        if (cur != cuda_device) cudaSetDevice(cuda_device);
+        fit = mlp_cluster_max_clusters(C, csmem) >= 1;
+        if (cur >= 0 && cur != cuda_device) cudaSetDevice(cur);
+      }
+      if (fit) {
+        c->chain_cluster = C;
+        c->chain_ks_l = ks_l;
+        c->chain_rows_per = rows_per;
+        c->chain_w_off = w_off;
+        c->chain_w_smem = cw;
+        c->chain_a_stages = stages;
+        c->chain_a_stage_bytes = stage_rows * 128;
+        c->chain_grid = C;
+        c->chain_barriers = 0;
+        snprintf(line, sizeof(line), "  -> inside one cluster of %d CTAs instead: activations through distributed shared memory, %u KB of resident weight slices per CTA, no grid barrier\n",
+                 C, cw / 1024);
+        c->desc += line;
+      }
+    }
   }
   // Two consecutive large layers on CTA pairs: one launch with a tile schedule over both (see the kernel's header).
   if (c->pattern == PAT_MLP && !c->chain_fused && !c->opt.no_chain_fusion && !c->opt.force_generic) {
@@ -1149,6 +1208,10 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
       cl.epi.bias = L.bias_input >= 0 ? static_cast<const float*>(in[L.bias_input]) : nullptr;
       cl.epi.dqv = L.dqv_host.empty() ? nullptr : reinterpret_cast<const float*>(ws + L.dqv_off);
       cl.epi.comp = L.need_comp ? reinterpret_cast<const int*>(ws + L.comp_off) : nullptr;
+      if (c.chain_cluster) {
+        cl.ks_l = c.chain_ks_l[l];
+        cl.rows_per = c.chain_rows_per[l];
+      }
       if (L.use_tc) {
         const uint32_t afmt = L.a_dtype == GC_S8 ? 1u : 0u;
         cl.idesc = L.kind == 0   ? ((2u << 4) | (afmt << 7) | (1u << 10) | ((32u >> 3) << 17) | ((128u >> 4) << 24))
@@ -1169,7 +1232,10 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
       c.chain_a0_ptr = a0;
     }
     memcpy(cp.tmaps, c.chain_tmaps.data(), sizeof(cp.tmaps));
-    CUDA_TRY(launch_mlp_chain(c.chain_kind, cp, c.chain_grid, st));
+    if (c.chain_cluster)
+      CUDA_TRY(launch_mlp_cluster(cp, c.chain_cluster, st));
+    else
+      CUDA_TRY(launch_mlp_chain(c.chain_kind, cp, c.chain_grid, st));
     return GC_OK;
   }
   GemmTcParams pair_first = {};

@@ -121,6 +121,9 @@ struct ChainLayer {
   int64_t out_pitch;       // elements
   int out_elem;            // bytes per stored element
   Epilogue epi;
+  // one-cluster variant only (kernels_chain_cluster.cu): parts this layer's reduction axis is split into, and the rows
+  // of the tile each CTA of such a group finishes (a multiple of 8)
+  int ks_l, rows_per;
 };
 struct ChainParams {
   int n_layers;
@@ -148,6 +151,14 @@ size_t mlp_chain_smem_bytes(size_t w_smem_bytes, int a_stages, int a_stage_bytes
 cudaError_t launch_mlp_chain(int kind, const ChainParams& p, int grid, cudaStream_t s);
 // clusters of `ks` CTAs of the chain kernel that can be resident together on the current device (0 on error)
 int mlp_chain_max_clusters(int kind, int ks, size_t smem);
+
+// The same chain inside ONE thread-block cluster (fp32 / tf32 chains small enough for it): activations travel from
+// layer to layer through distributed shared memory, no grid barrier, no round trip through the L2.  Uses
+// ChainParams with a_stages = stages per A-operand region (two regions, alternating by layer) and the per-layer
+// ks_l / rows_per; `cluster` = CTAs of the launch = cluster size (8 or 16).
+size_t mlp_cluster_smem_bytes(size_t w_smem_bytes, int a_stages, int a_stage_bytes);
+cudaError_t launch_mlp_cluster(const ChainParams& p, int cluster, cudaStream_t s);
+int mlp_cluster_max_clusters(int cluster, size_t smem);
 
 // Raise a kernel's dynamic shared-memory limit to at least `smem` bytes on the current device.  The driver call is made
 // once per (kernel, device) and size, not on every launch.

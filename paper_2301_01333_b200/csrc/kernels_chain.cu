@@ -61,12 +61,16 @@ __device__ __forceinline__ bool grid_barrier(unsigned long long* ctr, unsigned l
     // TMA loads: proxy fence on the global space, then a releasing reduction (no return value to wait for)
     asm volatile("fence.proxy.async.global;" ::: "memory");
     asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(ctr), "l"(1ULL) : "memory");
-    const uint64_t t0 = globaltimer_ns();
+    uint64_t t0 = 0;                                            // the global timer is slow to read: only once polling drags on
     uint32_t i = 0;
     while (ld_acquire_u64(ctr) < target) {
-      if ((++i & 1023u) == 0 && globaltimer_ns() - t0 > 2000000000ull) {
-        ok = 0;
-        break;
+      if ((++i & 1023u) == 0) {
+        const uint64_t t = globaltimer_ns();
+        if (t0 == 0) t0 = t;
+        else if (t - t0 > 2000000000ull) {
+          ok = 0;
+          break;
+        }
       }
     }
     asm volatile("fence.proxy.async.global;" ::: "memory");
@@ -82,34 +86,6 @@ __device__ __forceinline__ float ch_load_f(const void* p, int64_t i, int dtype) 
 __device__ __forceinline__ int ch_load_i(const void* p, int64_t i, int dtype) {
   if (dtype == GC_U8) return static_cast<const uint8_t*>(p)[i];
   return static_cast<const int8_t*>(p)[i];
-}
-
-// Bulk copy from this CTA's shared memory into the shared memory of a CTA of the cluster; the copy reports its
-// bytes to that CTA's mbarrier (complete_tx).  Addresses and size are multiples of 16 bytes.
-__device__ __forceinline__ void bulk_copy_to_cluster(uint32_t dst_cluster_addr, uint32_t src_cta_addr, uint32_t bytes,
-                                                     uint32_t cluster_bar) {
-  asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                   dst_cluster_addr),
-               "r"(src_cta_addr), "r"(bytes), "r"(cluster_bar)
-               : "memory");
-}
-// Bounded wait on an mbarrier of this CTA that CTAs of the cluster arrive on: acquire at cluster scope, so the
-// remote shared-memory stores made before those arrivals are visible afterwards.
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity) {
-  const uint64_t t0 = globaltimer_ns();
-  for (uint32_t i = 0; i < (1u << 22); ++i) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred P;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 P, [%1], %2, %3;\n\t"
-        "selp.b32 %0, 1, 0, P;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity), "r"(20000u)
-        : "memory");
-    if (ok) return true;
-    if ((i & 15u) == 15u && globaltimer_ns() - t0 > 2000000000ull) break;
-  }
-  return false;
 }
 
 template <int KIND>

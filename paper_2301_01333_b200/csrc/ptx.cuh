@@ -68,10 +68,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity, uin
 // code in the status word and leaves its loop; nothing spins forever.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   if (mbar_try_wait(bar, parity, 1000u)) return true;
-  const uint64_t t0 = globaltimer_ns();
+  uint64_t t0 = 0;                                              // the global timer is slow to read: only once polling drags on
   for (uint32_t i = 0; i < (1u << 22); ++i) {
     if (mbar_try_wait(bar, parity, 20000u)) return true;
-    if ((i & 15u) == 15u && globaltimer_ns() - t0 > 2000000000ull) break;
+    if ((i & 15u) == 15u) {
+      const uint64_t t = globaltimer_ns();
+      if (t0 == 0) t0 = t;
+      else if (t - t0 > 2000000000ull) break;
+    }
   }
   return false;
 }
@@ -80,10 +84,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
 // another CTA (such waiters were seen to wake up to a microsecond late with the long hints).
 __device__ __forceinline__ bool mbar_wait_prompt(uint32_t bar, uint32_t parity) {
   if (mbar_try_wait(bar, parity, 100u)) return true;
-  const uint64_t t0 = globaltimer_ns();
+  uint64_t t0 = 0;
   for (uint32_t i = 0; i < (1u << 30); ++i) {
     if (mbar_try_wait(bar, parity, 100u)) return true;
-    if ((i & 255u) == 255u && globaltimer_ns() - t0 > 2000000000ull) break;
+    if ((i & 255u) == 255u) {
+      const uint64_t t = globaltimer_ns();
+      if (t0 == 0) t0 = t;
+      else if (t - t0 > 2000000000ull) break;
+    }
   }
   return false;
 }
@@ -287,6 +295,39 @@ __device__ __forceinline__ void mbar_arrive_cluster_nomem(uint32_t cluster_bar) 
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+
+// Bulk copy from this CTA's shared memory into the shared memory of a CTA of the cluster; the copy reports its
+// bytes to that CTA's mbarrier (complete_tx).  Addresses and size are multiples of 16 bytes.
+__device__ __forceinline__ void bulk_copy_to_cluster(uint32_t dst_cluster_addr, uint32_t src_cta_addr, uint32_t bytes,
+                                                     uint32_t cluster_bar) {
+  asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   dst_cluster_addr),
+               "r"(src_cta_addr), "r"(bytes), "r"(cluster_bar)
+               : "memory");
+}
+// Bounded wait on an mbarrier of this CTA that CTAs of the cluster arrive on: acquire at cluster scope, so the
+// remote shared-memory stores made before those arrivals are visible afterwards.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint64_t t0 = 0;                                              // the global timer is slow to read: only once polling drags on
+  for (uint32_t i = 0; i < (1u << 22); ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred P;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 P, [%1], %2, %3;\n\t"
+        "selp.b32 %0, 1, 0, P;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(20000u)
+        : "memory");
+    if (ok) return true;
+    if ((i & 15u) == 15u) {
+      const uint64_t t = globaltimer_ns();
+      if (t0 == 0) t0 = t;
+      else if (t - t0 > 2000000000ull) break;
+    }
+  }
+  return false;
+}
+
 __device__ __forceinline__ void tmem_alloc2(uint32_t smem_result, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(ncols)
                : "memory");
