@@ -448,8 +448,9 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
   // total between launches, which the start-value computation above relies on.  Relaxed: the next launch reads the
   // counter only after this one has completed, and a release here would hold the CTA back for over a thousand clocks.
   if (threadIdx.x == 0) asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(p.barrier), "l"(1ULL) : "memory");
-  // no CTA leaves while another one of its cluster may still write into its shared memory
-  if (KS > 1) cluster_sync_all();
+  // no CTA leaves while another one of its cluster may still write into its shared memory or read a copy out of it
+  // (every CTA has seen all copies addressed to it complete before it arrives here; nothing else is ordered)
+  if (KS > 1) cluster_sync_all_relaxed();
 }
 
 size_t mlp_chain_smem_bytes(size_t w_smem_bytes, int a_stages, int a_stage_bytes, int ks) {

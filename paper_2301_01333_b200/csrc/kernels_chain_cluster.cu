@@ -11,7 +11,7 @@
 //     (slices_l * ks_l <= C); CTA r works on slice r / ks_l, part r % ks_l, and is idle in layers with fewer parts;
 //   * per layer a CTA waits for its k-blocks of the A operand (first layer: TMA from global memory, or rows packed
 //     by the epilogue warps when TMA cannot address the row pitch; later layers: the bulk copies of the finishing
-//     CTAs), issues tcgen05.mma (tf32, M = 128, N = 32; the four 8-deep k-steps of a k-block go to four independent
+//     CTAs), issues tcgen05.mma (tf32, M = 64, N = 32; the four 8-deep k-steps of a k-block go to four independent
 //     accumulators), and its epilogue warps read the accumulators;
 //   * with ks_l > 1 the partial sums meet as in the grid-wide kernel: every CTA of a group finishes rows_per rows and
 //     receives those rows of the others' partial sums; they are added in a fixed order;
@@ -56,8 +56,8 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
   const int STAGE = p.a_stage_bytes;                              // bytes per A-operand stage (rows x 128)
   const int REGION = p.a_stages * STAGE;                          // one of the two A-operand regions
   uint8_t* sA = smem;                                             // 2 regions
-  // the weight slices (padded to at least 16 KB) follow, so the 128-row MMA reads of the last stages stay inside
-  // this CTA's shared memory
+  // the weight slices (padded to at least 16 KB) follow, so the 64-row MMA reads of the last stages (a stage may hold
+  // fewer rows) stay inside this CTA's shared memory
   uint8_t* sW = sA + ((2 * REGION + 1023) & ~1023);
   uint8_t* sRed = sW + (p.w_smem_bytes < 16384u ? 16384u : p.w_smem_bytes);   // partial sums from my group
   uint8_t* sSend = sRed + CC_RED_BYTES;                           // 2 x STAGE: my partial sums, staged for the copies
@@ -166,11 +166,13 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
           if (ok) {
             tc_fence_after();
             const uint32_t a0 = smem_u32(region), b0 = smem_u32(sW) + L.w_smem_off;
+            // at most 64 rows are ever finished: M = 64 (the M field of the descriptor is bits 24..28, in units of 16)
+            const uint32_t idesc = (L.idesc & ~(0x1Fu << 24)) | ((64u >> 4) << 24);
             for (int i = 0; i < my_nkb; ++i) {
 #pragma unroll
               for (int k = 0; k < 4; ++k)   // (each descriptor is built from its address, not stepped as an integer)
                 umma_ss<KIND_TF32>(tmem_base + k * CC_BLOCK_N, make_smem_desc(a0 + i * STAGE + 32 * k, 16, 1024, SWZ_128B),
-                                   make_smem_desc(b0 + i * (CC_BLOCK_N * 128) + 32 * k, 16, 1024, SWZ_128B), L.idesc, i != 0);
+                                   make_smem_desc(b0 + i * (CC_BLOCK_N * 128) + 32 * k, 16, 1024, SWZ_128B), idesc, i != 0);
             }
             umma_commit(bar_tfull);
           } else {
@@ -224,17 +226,33 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
       const int rows_all = KS * rows_per;                         // rows of the tile that are finished at all
       // expect my rows of the partial sums of the whole group (senders cannot be ahead of this by a whole layer)
       if (KS > 1 && et == 0) mbar_arrive_expect_tx(bar_red, static_cast<uint32_t>(rows_all * 128));
-      // thread et finishes row et / 2 of my rows, columns 16 (et % 2) .. + 16 of my slice
-      const int frow = et >> 1, half = et & 1;
-      const bool finisher = frow < rows_per;
-      const int fcol = slice * CC_BLOCK_N + 16 * half;
-      EpiCols16 fk;
-      if (finisher) epi_load_cols16(fk, fcol, L.epi);
+      // The M = 64 accumulator keeps tile row i in tensor-memory lane 32 (i / 16) + i % 16: warp q reads rows
+      // 16 q .. 16 q + 15 with its lanes 0 .. 15.
+      const int row = q * 16 + lane;                              // my accumulator row (lanes 0..15)
+      const bool has_row = lane < 16 && row < rows_all;
+      // split layers: thread et finishes row et / 2 of my rows, columns 16 (et % 2) .. + 16 of my slice;
+      // unsplit layers: the thread that read a row finishes all 32 columns of it
+      const int frow = KS > 1 ? (et >> 1) : row, half = et & 1;
+      const bool finisher = KS > 1 ? frow < rows_per : has_row;
+      const int ncol4 = KS > 1 ? 4 : 8;                           // float4 groups this thread finishes
+      const int fcol = slice * CC_BLOCK_N + (KS > 1 ? 16 * half : 0);
+      float4 bias4[8];
+      if (finisher && L.epi.bias) {
+        const float4* bp = reinterpret_cast<const float4*>(L.epi.bias + fcol);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          if (i < ncol4) bias4[i] = __ldg(bp + i);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) bias4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+      const int act = L.epi.act;
       bool ok = cc_epi_all(mbar_wait(bar_tfull, tphase));
+      float4 acc4[8];
       if (ok) {
         tc_fence_after();
         uint32_t r[32];
-        if (my_nkb > 0 && q * 32 < rows_all) {
+        if (my_nkb > 0 && q * 16 < rows_all) {
           uint32_t r1[32], r2[32], r3[32];
           const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
           tmem_ld32(t_row, r);
@@ -251,23 +269,21 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
           for (int i = 0; i < 32; ++i) r[i] = 0u;
         }
         tc_fence_before();
-        // my accumulator row goes to a staging buffer (16-byte chunks XOR-swizzled by the row); with a split
-        // reduction axis the rows then travel to the CTAs of my group that finish them, otherwise I finish them all
-        const int row = q * 32 + lane;
-        uint8_t* stage_buf = KS > 1 ? send : sRed;
-        if (row < rows_all) {
-          uint8_t* my = stage_buf + row * 128;
-#pragma unroll
-          for (int c = 0; c < 8; ++c)
-            *reinterpret_cast<uint4*>(my + ((c ^ (row & 7)) << 4)) = make_uint4(r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);
-        }
         if (KS > 1) {
+          // my accumulator row goes to the staging buffer (16-byte chunks XOR-swizzled by the row) and from there to
+          // the CTA of my group that finishes it
+          if (has_row) {
+            uint8_t* my = send + row * 128;
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+              *reinterpret_cast<uint4*>(my + ((c ^ (row & 7)) << 4)) = make_uint4(r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);
+          }
           fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) {
             const int base = rank - part;                         // first CTA of my group
             for (int d = 0; d < KS; ++d) {                        // rows [d rows_per, (d + 1) rows_per) belong to part d
-              const int ra = max(d * rows_per, q * 32), rb = min((d + 1) * rows_per, q * 32 + 32);
+              const int ra = max(d * rows_per, q * 16), rb = min((d + 1) * rows_per, q * 16 + 16);
               if (ra >= rb) continue;
               bulk_copy_to_cluster(mapa_shared(smem_u32(sRed) + static_cast<uint32_t>((part * rows_per + ra - d * rows_per) * 128), base + d),
                                    smem_u32(send) + static_cast<uint32_t>(ra * 128), static_cast<uint32_t>((rb - ra) * 128),
@@ -275,60 +291,74 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
             }
           }
           ok = cc_epi_all(mbar_wait_cluster(bar_red, rphase));
+          if (ok && finisher) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc4[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int s = 0; s < KS; ++s) {                        // fixed order: deterministic
+              const uint8_t* src = sRed + (s * rows_per + frow) * 128;
+#pragma unroll
+              for (int c = 0; c < 4; ++c) {
+                const float4 v = *reinterpret_cast<const float4*>(src + (((half * 4 + c) ^ (frow & 7)) << 4));
+                acc4[c].x += v.x; acc4[c].y += v.y; acc4[c].z += v.z; acc4[c].w += v.w;
+              }
+            }
+          }
         } else {
-          asm volatile("bar.sync 1, 128;" ::: "memory");          // all rows staged (epilogue warps only)
+#pragma unroll
+          for (int c = 0; c < 8; ++c)
+            acc4[c] = make_float4(__uint_as_float(r[4 * c]), __uint_as_float(r[4 * c + 1]), __uint_as_float(r[4 * c + 2]),
+                                  __uint_as_float(r[4 * c + 3]));
         }
       }
       if (ok) {
         if (finisher) {
-          uint32_t a[16];
+          // bias and activation (fp32 chains only: this kernel takes no other)
 #pragma unroll
-          for (int i = 0; i < 16; ++i) a[i] = 0u;
-          for (int s = 0; s < KS; ++s) {                          // fixed order: deterministic
-            const uint8_t* src = sRed + (s * rows_per + frow) * 128;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              const uint4 v = *reinterpret_cast<const uint4*>(src + (((half * 4 + c) ^ (frow & 7)) << 4));
-              a[4 * c] = __float_as_uint(__uint_as_float(a[4 * c]) + __uint_as_float(v.x));
-              a[4 * c + 1] = __float_as_uint(__uint_as_float(a[4 * c + 1]) + __uint_as_float(v.y));
-              a[4 * c + 2] = __float_as_uint(__uint_as_float(a[4 * c + 2]) + __uint_as_float(v.z));
-              a[4 * c + 3] = __float_as_uint(__uint_as_float(a[4 * c + 3]) + __uint_as_float(v.w));
+          for (int c = 0; c < 8; ++c) {
+            if (c < ncol4) {
+              float4 t = acc4[c];
+              t.x = __fadd_rn(t.x, bias4[c].x); t.y = __fadd_rn(t.y, bias4[c].y);
+              t.z = __fadd_rn(t.z, bias4[c].z); t.w = __fadd_rn(t.w, bias4[c].w);
+              if (act == ACT_RELU) {
+                t.x = fmaxf(t.x, 0.f); t.y = fmaxf(t.y, 0.f); t.z = fmaxf(t.z, 0.f); t.w = fmaxf(t.w, 0.f);
+              } else if (act != ACT_NONE) {
+                t.x = apply_act(t.x, act); t.y = apply_act(t.y, act); t.z = apply_act(t.z, act); t.w = apply_act(t.w, act);
+              }
+              acc4[c] = t;
             }
           }
           const int grow = part * rows_per + frow;                // row of the tile
           if (last) {
             if (grow < L.M) {
-              char* dst_row = static_cast<char*>(L.out) + static_cast<int64_t>(grow) * L.out_pitch * L.out_elem;
-              epi_store16_cols(a, dst_row, fcol, L.epi, fk);
+              float4* d = reinterpret_cast<float4*>(static_cast<float*>(L.out) + static_cast<int64_t>(grow) * L.out_pitch + fcol);
+#pragma unroll
+              for (int c = 0; c < 8; ++c)
+                if (c < ncol4) d[c] = acc4[c];
             }
           } else {
-            float t[16];
-            epi_values16(a, t, L.epi, fk);
             uint8_t* my = outb + frow * 128;
+            const int c0 = KS > 1 ? half * 4 : 0;
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
-              *reinterpret_cast<uint4*>(my + (((half * 4 + c) ^ (frow & 7)) << 4)) =
-                  make_uint4(__float_as_uint(t[4 * c]), __float_as_uint(t[4 * c + 1]), __float_as_uint(t[4 * c + 2]),
-                             __float_as_uint(t[4 * c + 3]));
+            for (int c = 0; c < 8; ++c)
+              if (c < ncol4) *reinterpret_cast<float4*>(my + (((c0 + c) ^ (frow & 7)) << 4)) = acc4[c];
           }
         }
         if (!last) {
           // my finished rows are rows [part rows_per, + rows_per) of k-block `slice` of the next layer's A operand:
-          // one copy to every CTA of that layer whose part of the reduction axis contains the k-block
+          // one copy to every CTA of that layer whose part of the reduction axis contains the k-block (each copy
+          // issued by a thread of its own)
           fence_proxy_async_smem();
           asm volatile("bar.sync 1, 128;" ::: "memory");
-          if (et == 0) {
-            const ChainLayer& Nx = p.L[l + 1];
+          const ChainLayer& Nx = p.L[l + 1];
+          const int nslices = Nx.N / CC_BLOCK_N;
+          if (et < nslices) {
             int np = 0;
             while (np + 1 < Nx.ks_l && (np + 1) * Nx.nkb / Nx.ks_l <= slice) ++np;     // the part that holds k-block `slice`
             const int st = slice - np * Nx.nkb / Nx.ks_l;                                // its stage there
             const uint32_t dst = smem_u32(sA) + static_cast<uint32_t>(((l + 1) & 1) * REGION + st * STAGE + part * rows_per * 128);
-            const int nslices = Nx.N / CC_BLOCK_N;
-            for (int s = 0; s < nslices; ++s) {
-              const int rc = s * Nx.ks_l + np;
-              bulk_copy_to_cluster(mapa_shared(dst, rc), smem_u32(outb), static_cast<uint32_t>(rows_per * 128),
-                                   mapa_shared(bar_a + 8 * (l + 1), rc));
-            }
+            const int rc = et * Nx.ks_l + np;
+            bulk_copy_to_cluster(mapa_shared(dst, rc), smem_u32(outb), static_cast<uint32_t>(rows_per * 128),
+                                 mapa_shared(bar_a + 8 * (l + 1), rc));
           }
         }
       } else {
@@ -347,8 +377,9 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
     tc_fence_after();
     tmem_dealloc(tmem_base, CC_NACC * CC_BLOCK_N);
   }
-  // no CTA leaves while another one of its cluster may still write into its shared memory
-  cluster_sync_all();
+  // no CTA leaves while another one of its cluster may still write into its shared memory or read a copy out of it
+  // (every CTA has seen all copies addressed to it complete before it arrives here; nothing else is ordered)
+  cluster_sync_all_relaxed();
 }
 
 size_t mlp_cluster_smem_bytes(size_t w_smem_bytes, int a_stages, int a_stage_bytes) {

@@ -295,6 +295,12 @@ __device__ __forceinline__ void mbar_arrive_cluster_nomem(uint32_t cluster_bar) 
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// The same as a pure execution barrier: no memory ordering, so the arrival does not wait for this CTA's outstanding
+// global stores (a releasing arrival does, a thousand clocks and more).  For the barrier before the exit that only
+// keeps a CTA's shared memory alive until its peers have stopped using it.
+__device__ __forceinline__ void cluster_sync_all_relaxed() {
+  asm volatile("barrier.cluster.arrive.relaxed.aligned;\n\tbarrier.cluster.wait.aligned;" ::: "memory");
+}
 
 // Bulk copy from this CTA's shared memory into the shared memory of a CTA of the cluster; the copy reports its
 // bytes to that CTA's mbarrier (complete_tx).  Addresses and size are multiples of 16 bytes.

@@ -198,10 +198,39 @@ def test_mlp_int8_chain_kernel_cluster_sizes_and_entry_reorder(B, batch, dims, k
 @pytest.mark.parametrize("batch,dims,ks", [(16, (160, 64, 32), 2), (100, (13, 1024, 48), 4), (128, (37, 32, 16), 1)])
 def test_mlp_f32_chain_kernel_cluster_sizes(B, batch, dims, ks):
     w = W.mlp_f32(batch=batch, dims=dims)
-    got, plan = run_gpu(B, w)
-    assert f"clusters of {ks}" in plan
+    got, plan = run_gpu(B, w, grid_wide_chain=True)
+    assert f"clusters of {ks}" in plan and "inside one cluster" not in plan
     ref = oracle(w)
     assert np.abs(got.astype(np.float64) - ref).max() <= 5e-3 * np.abs(ref).max()
+
+
+@pytest.mark.parametrize("batch,dims,cluster", [
+    (32, (13, 512, 256, 128), 16),        # config 1: 16 x 1, 8 x 2 and 4 x 4 (slices x parts of the reduction axis)
+    (64, (13, 512, 256, 128), 16),        # the most rows the kernel takes
+    (1, (32, 32, 32), 8),                 # one row, one slice
+    (17, (45, 96, 64), 8),                # ragged rows and a first layer whose row pitch TMA cannot address
+    (8, (64, 128, 64), 8),                # first layer fed by TMA
+    (24, (200, 160, 288, 32, 64), 16),    # five k-blocks over two parts, nine slices, a one-slice layer in the middle
+])
+def test_mlp_f32_chain_inside_one_cluster(B, batch, dims, cluster):
+    w = W.mlp_f32(batch=batch, dims=dims)
+    got, plan = run_gpu(B, w, n_runs=3)
+    assert f"inside one cluster of {cluster} CTAs" in plan
+    assert np.array_equal(got[0], got[1]) and np.array_equal(got[0], got[2])      # deterministic, no state carried over
+    ref = oracle(w)
+    assert np.abs(got[0].astype(np.float64) - ref).max() <= 5e-3 * np.abs(ref).max()
+    wide, plan_w = run_gpu(B, w, grid_wide_chain=True)
+    assert "inside one cluster" not in plan_w
+    assert np.abs(wide.astype(np.float64) - ref).max() <= 5e-3 * np.abs(ref).max()
+
+
+def test_mlp_f32_too_large_for_one_cluster_stays_grid_wide(B):
+    for batch, dims in ((65, (13, 512, 256, 128)), (32, (13, 1024, 64)), (40, (100, 256, 256, 128, 32))):
+        w = W.mlp_f32(batch=batch, dims=dims)
+        got, plan = run_gpu(B, w)
+        assert "fused chain" in plan and "inside one cluster" not in plan
+        ref = oracle(w)
+        assert np.abs(got.astype(np.float64) - ref).max() <= 5e-3 * np.abs(ref).max()
 
 
 def test_two_large_layers_in_one_launch_bf16(B):
