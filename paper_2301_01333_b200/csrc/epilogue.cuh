@@ -28,6 +28,10 @@ __device__ __forceinline__ float apply_act(float t, int act) {
   }
 }
 
+// The same out of line: for kernels whose code runs once per launch (the small-batch chain kernels), where every
+// inlined copy of the exponential / tanh sequences is instruction-cache misses and nothing else.
+static __device__ __noinline__ float apply_act_cold(float t, int act) { return apply_act(t, act); }
+
 // Value after dequantize / bias / activation.  `raw` holds the accumulator bits (s32 or f32).
 __device__ __forceinline__ float epi_value(uint32_t raw, int n, const Epilogue& e) {
   float t;

@@ -272,6 +272,7 @@ struct gc_compiled {
   bool chain_tmaps_valid = false;
   // the same chain inside one thread-block cluster (small fp32 chains)
   int chain_cluster = 0;                     // cluster size (0: the grid-wide kernel)
+  bool chain_recompute_first = false;
   std::vector<int> chain_ks_l, chain_rows_per;
   // host staging
   size_t staging_bytes = 0;
@@ -839,30 +840,47 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
     // handed from layer to layer through distributed shared memory (no grid barrier, no round trip through the L2).
     // Layer l uses slices_l = N_l / 32 column slices times ks_l parts of the reduction axis.
     if (ok && kind == 2 && row_tiles == 1 && !c->opt.grid_wide_chain) {
+      // A first layer with a short reduction axis is recomputed by the CTAs of the second layer (each produces the
+      // columns that form its own part of that layer's reduction axis) instead of being distributed and handed over.
+      const bool can_recompute = c->layers.size() >= 2 && c->layers[0].nkb <= 2;
+      for (int attempt = can_recompute ? 0 : 1; attempt < 2 && !c->chain_cluster; ++attempt) {   // (not re-indented)
+      const bool recompute = attempt == 0;
+      const size_t l_first = recompute ? 1 : 0;
       bool fit = c->layers[0].M <= 64;
-      int max_slices = 0;
-      for (const LayerPlan& L : c->layers) {
-        fit = fit && L.use_tc && L.N % 32 == 0 && L.N / 32 <= 16 && L.epi.out_dtype == GC_F32 && !L.epi.acc_is_int;
-        max_slices = std::max(max_slices, L.N / 32);
+      int want = 0;                                               // CTAs the widest distributed layer can use
+      for (size_t l = 0; l < c->layers.size(); ++l) {
+        const LayerPlan& L = c->layers[l];
+        fit = fit && L.use_tc && L.N % 32 == 0 && L.epi.out_dtype == GC_F32 && !L.epi.acc_is_int;
+        if (l >= l_first) want = std::max(want, (L.N / 32) * std::min(4, L.nkb));
       }
-      const int C = max_slices > 8 ? 16 : 8;
+      const int C = want > 8 ? 16 : 8;
       const int rows_pad = (c->layers[0].M + 7) / 8 * 8;
       std::vector<int> ks_l(c->layers.size(), 1), rows_per(c->layers.size(), rows_pad);
       std::vector<uint32_t> w_off(c->layers.size(), 0);
       uint32_t cw = 0;
       int stages = 1, stage_rows = rows_pad;
-      for (size_t l = 0; fit && l < c->layers.size(); ++l) {
+      for (size_t l = l_first; fit && l < c->layers.size(); ++l) {
         const LayerPlan& L = c->layers[l];
+        fit = L.N / 32 <= C;
         int ks = 1;
         while (ks < 4 && 2 * ks * (L.N / 32) <= C && 2 * ks <= L.nkb) ks *= 2;
         ks_l[l] = ks;
         rows_per[l] = ((rows_pad + ks - 1) / ks + 7) / 8 * 8;
-        fit = rows_per[l] <= 64;                                  // two finishing threads per row, 128 of them
+        fit = fit && rows_per[l] <= 64;                           // two finishing threads per row, 128 of them
         stage_rows = std::max(stage_rows, ks * rows_per[l]);
         const int my_nkb = (L.nkb + ks - 1) / ks;
         stages = std::max(stages, my_nkb);
         w_off[l] = cw;
         cw += static_cast<uint32_t>(my_nkb) * 32 * 128;
+      }
+      if (fit && recompute) {
+        const LayerPlan& L0 = c->layers[0];
+        const LayerPlan& L1 = c->layers[1];
+        const int n1 = (L1.nkb + ks_l[1] - 1) / ks_l[1];         // k-blocks of the second layer per CTA = 32-column groups to produce
+        fit = n1 * 32 <= 256;                                     // one accumulator, one MMA N
+        stages = std::max(stages, L0.nkb);
+        w_off[0] = cw;
+        cw += static_cast<uint32_t>(L0.nkb * n1) * 32 * 128;
       }
       size_t csmem = 0;
       if (fit) {
@@ -880,15 +898,17 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
         c->chain_cluster = C;
         c->chain_ks_l = ks_l;
         c->chain_rows_per = rows_per;
+        c->chain_recompute_first = recompute;
         c->chain_w_off = w_off;
         c->chain_w_smem = cw;
         c->chain_a_stages = stages;
         c->chain_a_stage_bytes = stage_rows * 128;
         c->chain_grid = C;
         c->chain_barriers = 0;
-        snprintf(line, sizeof(line), "  -> inside one cluster of %d CTAs instead: activations through distributed shared memory, %u KB of resident weight slices per CTA, no grid barrier\n",
-                 C, cw / 1024);
+        snprintf(line, sizeof(line), "  -> inside one cluster of %d CTAs instead: activations through distributed shared memory, %u KB of resident weight slices per CTA, no grid barrier%s\n",
+                 C, cw / 1024, recompute ? "; first layer recomputed by the CTAs of the second" : "");
         c->desc += line;
+      }
       }
     }
   }
@@ -1232,6 +1252,7 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
       c.chain_a0_ptr = a0;
     }
     memcpy(cp.tmaps, c.chain_tmaps.data(), sizeof(cp.tmaps));
+    cp.recompute_first = c.chain_recompute_first ? 1 : 0;
     if (c.chain_cluster)
       CUDA_TRY(launch_mlp_cluster(cp, c.chain_cluster, st));
     else

@@ -142,6 +142,8 @@ struct ChainParams {
   int slices;                               // 32-column slices per row tile: grid = row tiles x slices x ks
   int early_weights;                        // 1: the prepacked weights were written by an earlier call, so their loads
                                             // need not wait for the kernel that precedes this one on the stream
+  int recompute_first;                      // one-cluster variant: every CTA of the second layer computes the first
+                                            // layer's columns it needs itself (no hand-over between the two)
   uint32_t* status;
   // TMA descriptors travel in the kernel parameter space (fetched once, cached by the TMA unit); descriptors
   // kept in global memory cost a fetch of several hundred clocks on every load instruction.

@@ -18,6 +18,10 @@
 //   * a finished row of 32 fp32 values IS a 128-byte row of a k-block of the next layer's A operand (k-block = my
 //     slice index): it is written in the swizzled operand layout into a local buffer and copied to every CTA of the
 //     next layer whose part of the reduction axis contains that k-block; the last layer stores to global memory.
+//   * a first layer with a short reduction axis (at most two k-blocks) is not distributed at all: every CTA of the
+//     second layer multiplies the input by the first-layer weight columns that make up its own part of the second
+//     layer's reduction axis (N up to 256 in one accumulator) and writes the result, bias and activation applied,
+//     straight into its own A-operand stages - redundant arithmetic across the column slices, no exchange.
 // A-operand stages alternate between two regions by layer parity, and so do the staging buffers; every buffer is
 // reused two layers later, by which time the data dependence chain guarantees that all copies out of it and all MMAs
 // reading it have completed (a CTA can only reach layer l + 2 after every CTA has finished layer l).
@@ -34,6 +38,8 @@ constexpr int CC_BLOCK_N = 32;
 constexpr int CC_NACC = 4;
 constexpr int CC_K_ELEMS = 32;           // fp32 elements per 128-byte k-block
 constexpr int CC_RED_BYTES = 128 * 128;  // partial sums received: at most 128 rows of 128 bytes
+constexpr int CC_T0_COL = CC_NACC * CC_BLOCK_N;   // tensor-memory column of the recomputed first layer's accumulator
+constexpr int CC_T0_MAX = 256;                     // its widest form
 
 // AND of a flag over the 128 threads of the four epilogue warps (named barrier 1): after a bounded wait every one of
 // them takes the same branch, so the named barriers that follow are reached by all or by none.
@@ -48,6 +54,20 @@ __device__ __forceinline__ bool cc_epi_all(bool ok) {
       : "r"(ok ? 1u : 0u)
       : "memory");
   return r != 0;
+}
+
+// Bounded waits out of line: this kernel's code runs once per launch, so every inlined copy of a polling loop is
+// instruction-cache misses on the way to the code that matters.
+static __device__ __noinline__ bool cc_wait(uint32_t bar, uint32_t parity) { return mbar_wait_prompt(bar, parity); }
+static __device__ __noinline__ bool cc_wait_cluster(uint32_t bar, uint32_t parity) { return mbar_wait_cluster<100u>(bar, parity); }
+
+// One lane of the warp polls, the others wait for it at the warp barrier of the shuffle: 128 polling threads keep the
+// shared-memory pipeline busy that the working warp needs.
+template <typename F>
+__device__ __forceinline__ bool cc_lane0_wait(int lane, F wait) {
+  int ok = 1;
+  if (lane == 0) ok = wait() ? 1 : 0;
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
 __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid_constant__ ChainParams p) {
@@ -68,16 +88,26 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
   const uint32_t bar_tfull = bar_a + 8 * CHAIN_MAX_LAYERS;        // accumulators ready
   const uint32_t bar_red = bar_tfull + 8;                         // partial sums of my group have arrived
   const uint32_t bar_a0 = bar_red + 8;                            // first layer's A operand packed by the epilogue warps
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * CHAIN_MAX_LAYERS + 3);
+  const uint32_t bar_a1 = bar_a0 + 8;                             // second layer's A operand written by the epilogue warps
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * CHAIN_MAX_LAYERS + 4);
+  float* sBias0 = reinterpret_cast<float*>(bars + 2 * CHAIN_MAX_LAYERS + 6);   // [CC_T0_MAX] first-layer bias of my columns
+  float* sBias = sBias0 + CC_T0_MAX;                              // [CHAIN_MAX_LAYERS][32] bias of my slice of every layer
+  const bool recompute = p.recompute_first != 0;
+  const int tmem_cols = recompute ? 512 : CC_NACC * CC_BLOCK_N;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rank = static_cast<int>(cluster_ctarank());
 
   // my role in layer l
-  auto active = [&](const ChainLayer& L) { return rank < (L.N / CC_BLOCK_N) * L.ks_l; };
-  auto kb_lo = [&](const ChainLayer& L, int part) { return part * L.nkb / L.ks_l; };
+  // (ks_l is 1, 2 or 4: shifts and masks, not divisions - they sit between the layers of a latency chain)
+  auto ks_sh = [](const ChainLayer& L) { return __ffs(L.ks_l) - 1; };
+  auto active = [&](const ChainLayer& L) { return rank < ((L.N >> 5) << ks_sh(L)); };
+  auto kb_lo = [&](const ChainLayer& L, int part) { return (part * L.nkb) >> ks_sh(L); };
+  auto part_of = [&](const ChainLayer& L) { return rank & (L.ks_l - 1); };
+  auto slice_of = [&](const ChainLayer& L) { return rank >> ks_sh(L); };
   const bool manual_a = p.pack_rows > 0;
 
   if (threadIdx.x == 0) {
+#pragma unroll 1
     for (int l = 0; l < CHAIN_MAX_LAYERS; ++l) {
       mbar_init(bar_w + 8 * l, 1);
       mbar_init(bar_a + 8 * l, 1);
@@ -85,19 +115,21 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
     mbar_init(bar_tfull, 1);
     mbar_init(bar_red, 1);
     mbar_init(bar_a0, 4);                                         // one arrival per epilogue warp
+    mbar_init(bar_a1, 4);
     fence_mbar_init();
     // the bytes the finishing CTAs of layer l - 1 will copy into my stages of layer l: armed before anybody can send
-    for (int l = 1; l < p.n_layers; ++l) {
+#pragma unroll 1
+    for (int l = recompute ? 2 : 1; l < p.n_layers; ++l) {
       const ChainLayer& L = p.L[l];
       if (!active(L)) continue;
-      const int part = rank % L.ks_l;
+      const int part = part_of(L);
       const int my_nkb = kb_lo(L, part + 1) - kb_lo(L, part);
       const ChainLayer& P = p.L[l - 1];
       mbar_arrive_expect_tx(bar_a + 8 * l, static_cast<uint32_t>(my_nkb * P.ks_l * P.rows_per * 128));
     }
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(tmem_slot), CC_NACC * CC_BLOCK_N);
+    tmem_alloc(smem_u32(tmem_slot), tmem_cols);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -113,37 +145,69 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (!p.early_weights) asm volatile("griddepcontrol.wait;" ::: "memory");
   if (warp == 0 && lane == 0) {
-    for (int l = 0; l < p.n_layers; ++l) {
+    if (recompute && active(p.L[1])) {
+      // the first-layer weight rows (= output columns) that form my part of the second layer's reduction axis
+      const ChainLayer& L0 = p.L[0];
+      const ChainLayer& L1 = p.L[1];
+      const int part = part_of(L1);
+      const int lo1 = kb_lo(L1, part), n1 = kb_lo(L1, part + 1) - lo1;
+      mbar_arrive_expect_tx(bar_w, static_cast<uint32_t>(L0.nkb * n1) * (CC_BLOCK_N * 128));
+#pragma unroll 1
+      for (int kb = 0; kb < L0.nkb; ++kb)
+#pragma unroll 1
+        for (int j = 0; j < n1; ++j)
+          tma_load_2d(smem_u32(sW) + L0.w_smem_off + (kb * n1 + j) * (CC_BLOCK_N * 128), p.tmaps + L0.b_tm, kb * CC_K_ELEMS,
+                      (lo1 + j) * CC_BLOCK_N, bar_w);
+    }
+#pragma unroll 1
+    for (int l = recompute ? 1 : 0; l < p.n_layers; ++l) {
       const ChainLayer& L = p.L[l];
       if (!active(L)) continue;
-      const int slice = rank / L.ks_l, part = rank % L.ks_l;
+      const int slice = slice_of(L), part = part_of(L);
       const int lo = kb_lo(L, part), hi = kb_lo(L, part + 1);
       if (hi == lo) continue;
       mbar_arrive_expect_tx(bar_w + 8 * l, static_cast<uint32_t>(hi - lo) * (CC_BLOCK_N * 128));
+#pragma unroll 1
       for (int kb = lo; kb < hi; ++kb)
         tma_load_2d(smem_u32(sW) + L.w_smem_off + (kb - lo) * (CC_BLOCK_N * 128), p.tmaps + L.b_tm, kb * CC_K_ELEMS,
                     slice * CC_BLOCK_N, bar_w + 8 * l);
     }
   }
-  if (p.early_weights) asm volatile("griddepcontrol.wait;" ::: "memory");
-
-  // the per-column constants my epilogues will need: start them on their way from DRAM now
-  if (warp >= 2 && threadIdx.x - 64 < p.n_layers) {
-    const ChainLayer& L = p.L[threadIdx.x - 64];
-    if (active(L) && L.epi.bias) asm volatile("prefetch.global.L2 [%0];" ::"l"(L.epi.bias + (rank / L.ks_l) * CC_BLOCK_N));
+  // The per-column constants my epilogues will need are constants like the weights: start them on their way now (the
+  // recomputed first layer's bias into shared memory, the others into the L2).
+  if (warp >= 2) {
+#pragma unroll 1
+    for (int i = threadIdx.x - 64; i < p.n_layers * CC_BLOCK_N; i += 128) {
+      const ChainLayer& L = p.L[i >> 5];
+      if ((recompute && i < CC_BLOCK_N) || !active(L)) continue;
+      sBias[i] = L.epi.bias ? __ldg(L.epi.bias + slice_of(L) * CC_BLOCK_N + (i & 31)) : 0.f;
+    }
   }
+  if (recompute && warp >= 2 && active(p.L[1])) {
+    const ChainLayer& L1 = p.L[1];
+    const int part = part_of(L1);
+    const int lo1 = kb_lo(L1, part), ncol = (kb_lo(L1, part + 1) - lo1) * CC_BLOCK_N;
+#pragma unroll 1
+    for (int i = threadIdx.x - 64; i < ncol; i += 128) sBias0[i] = p.L[0].epi.bias ? __ldg(p.L[0].epi.bias + lo1 * CC_BLOCK_N + i) : 0.f;
+  }
+  if (p.early_weights) asm volatile("griddepcontrol.wait;" ::: "memory");
 
   bool failed = false;
   uint32_t tphase = 0;           // parity of the accumulator-ready barrier (one completion per layer I am active in)
   uint32_t rphase = 0;           // parity of the partial-sum barrier (one completion per such layer with ks_l > 1)
 
+#pragma unroll 1
   for (int l = 0; l < p.n_layers && !failed; ++l) {
     // (a by-value copy: fields read through a reference into the parameter space are re-fetched around every store)
     const ChainLayer L = p.L[l];
-    if (!active(L)) continue;
-    const int KS = L.ks_l, rows_per = L.rows_per;
-    const int slice = rank / KS, part = rank % KS;
-    const int lo = kb_lo(L, part), my_nkb = kb_lo(L, part + 1) - lo;
+    // a recomputed first layer is the business of the CTAs of the second layer, each with the whole reduction axis
+    const bool rc0 = recompute && l == 0;
+    if (!active(rc0 ? p.L[1] : L)) continue;
+    const int KS = rc0 ? 1 : L.ks_l, rows_per = L.rows_per;
+    const int slice = rc0 ? rank : slice_of(L), part = rc0 ? 0 : part_of(L);
+    const int lo = rc0 ? 0 : kb_lo(L, part), my_nkb = rc0 ? L.nkb : kb_lo(L, part + 1) - lo;
+    // (recomputed first layer: the k-blocks of the second layer that are mine, i.e. 32-column groups to produce)
+    const int n1 = rc0 ? kb_lo(p.L[1], part_of(p.L[1]) + 1) - kb_lo(p.L[1], part_of(p.L[1])) : 0;
     const bool last = l + 1 == p.n_layers;
     uint8_t* region = sA + (l & 1) * REGION;
     uint8_t* send = sSend + (l & 1) * STAGE;
@@ -153,6 +217,7 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
       if (lane == 0 && l == 0 && !manual_a && my_nkb > 0) {
         const uint32_t box_bytes = static_cast<uint32_t>((L.M < 128 ? (L.M + 7) / 8 * 8 : 128) * 128);
         mbar_arrive_expect_tx(bar_a, static_cast<uint32_t>(my_nkb) * box_bytes);
+#pragma unroll 1
         for (int i = 0; i < my_nkb; ++i)
           tma_load_2d(smem_u32(region) + i * STAGE, p.tmaps + L.a_tm, (lo + i) * CC_K_ELEMS, 0, bar_a);
       }
@@ -161,13 +226,29 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
         if (my_nkb == 0) {
           mbar_arrive(bar_tfull);                                 // nothing to multiply: my partial sums are zero
         } else {
-          bool ok = mbar_wait(bar_w + 8 * l, 0);
-          if (ok) ok = (l == 0 && manual_a) ? mbar_wait(bar_a0, 0) : mbar_wait_cluster(bar_a + 8 * l, 0);
-          if (ok) {
+          bool ok = cc_wait(bar_w + 8 * l, 0);
+          if (ok) ok = (l == 0 && manual_a) ? cc_wait(bar_a0, 0)
+                       : (l == 1 && recompute) ? cc_wait(bar_a1, 0) : cc_wait_cluster(bar_a + 8 * l, 0);
+          if (ok && rc0) {
+            tc_fence_after();
+            const uint32_t a0 = smem_u32(region), b0 = smem_u32(sW) + L.w_smem_off;
+            // M = 64, N = 32 n1 (N field: bits 17..22 in units of 8); one accumulator: the few MMAs form a chain
+            const uint32_t idesc = (L.idesc & ~((0x1Fu << 24) | (0x3Fu << 17))) | ((64u >> 4) << 24) |
+                                   ((static_cast<uint32_t>(n1 * CC_BLOCK_N) >> 3) << 17);
+#pragma unroll 1
+            for (int i = 0; i < my_nkb; ++i) {
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                umma_ss<KIND_TF32>(tmem_base + CC_T0_COL, make_smem_desc(a0 + i * STAGE + 32 * k, 16, 1024, SWZ_128B),
+                                   make_smem_desc(b0 + i * n1 * (CC_BLOCK_N * 128) + 32 * k, 16, 1024, SWZ_128B), idesc, (i | k) != 0);
+            }
+            umma_commit(bar_tfull);
+          } else if (ok) {
             tc_fence_after();
             const uint32_t a0 = smem_u32(region), b0 = smem_u32(sW) + L.w_smem_off;
             // at most 64 rows are ever finished: M = 64 (the M field of the descriptor is bits 24..28, in units of 16)
             const uint32_t idesc = (L.idesc & ~(0x1Fu << 24)) | ((64u >> 4) << 24);
+#pragma unroll 1
             for (int i = 0; i < my_nkb; ++i) {
 #pragma unroll
               for (int k = 0; k < 4; ++k)   // (each descriptor is built from its address, not stepped as an integer)
@@ -193,9 +274,10 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
         const int64_t kbytes = static_cast<int64_t>(L.K) * 4;
         const uint8_t* src_row = static_cast<const uint8_t*>(p.pack_src) + static_cast<int64_t>(r) * p.pack_src_pitch;
         if (r < a_rows) {
+#pragma unroll 1
           for (int i = 0; i < my_nkb; ++i) {
             uint8_t* dst = region + i * STAGE + (r >> 3) * 1024 + (r & 7) * 128;
-#pragma unroll
+#pragma unroll 1
             for (int c = 0; c < 8; ++c) {
               const int64_t off = static_cast<int64_t>(lo + i) * 128 + c * 16;
               int64_t nv = kbytes - off;
@@ -223,6 +305,55 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_a0);
       }
+      if (rc0) {
+        // Recomputed first layer: my accumulator row holds the 32 n1 columns that are my k-blocks of the second layer's
+        // A operand; bias and activation applied, each group of 32 goes to its stage as one swizzled 128-byte row.
+        const int row = q * 16 + lane;
+        const bool has_row = lane < 16 && row < STAGE / 128;
+        const int act = L.epi.act;
+        uint8_t* region1 = sA + REGION;
+        const bool ok = cc_epi_all(cc_lane0_wait(lane, [&]() { return cc_wait(bar_tfull, tphase); }));   // (also orders the writes of sBias0 before its reads)
+        if (ok) {
+          tc_fence_after();
+          const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + CC_T0_COL;
+#pragma unroll 1
+          for (int j = 0; j < n1; ++j) {
+            uint32_t r[32];
+            tmem_ld32(t_row + j * CC_BLOCK_N, r);
+            tmem_wait_ld();
+            if (has_row) {
+              // all loads, then all arithmetic, then all stores: a lone warp per scheduler lives on instruction-level
+              // parallelism, and a store into the stage may alias the bias for all the compiler knows
+              float4 t[8];
+#pragma unroll
+              for (int c = 0; c < 8; ++c) t[c] = *reinterpret_cast<const float4*>(sBias0 + j * CC_BLOCK_N + 4 * c);
+#pragma unroll
+              for (int c = 0; c < 8; ++c) {
+                t[c].x = __fadd_rn(__uint_as_float(r[4 * c]), t[c].x); t[c].y = __fadd_rn(__uint_as_float(r[4 * c + 1]), t[c].y);
+                t[c].z = __fadd_rn(__uint_as_float(r[4 * c + 2]), t[c].z); t[c].w = __fadd_rn(__uint_as_float(r[4 * c + 3]), t[c].w);
+                if (act == ACT_RELU) {
+                  t[c].x = fmaxf(t[c].x, 0.f); t[c].y = fmaxf(t[c].y, 0.f); t[c].z = fmaxf(t[c].z, 0.f); t[c].w = fmaxf(t[c].w, 0.f);
+                } else if (act != ACT_NONE) {
+                  t[c].x = apply_act_cold(t[c].x, act); t[c].y = apply_act_cold(t[c].y, act);
+                  t[c].z = apply_act_cold(t[c].z, act); t[c].w = apply_act_cold(t[c].w, act);
+                }
+              }
+              uint8_t* my = region1 + j * STAGE + (row >> 3) * 1024 + (row & 7) * 128;
+#pragma unroll
+              for (int c = 0; c < 8; ++c) *reinterpret_cast<float4*>(my + ((c ^ (row & 7)) << 4)) = t[c];
+            }
+          }
+          tc_fence_before();
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_a1);
+        } else {
+          report(p.status, DEV_TIMEOUT_EPILOGUE);
+          failed = true;
+        }
+        tphase ^= 1;
+        continue;
+      }
       const int rows_all = KS * rows_per;                         // rows of the tile that are finished at all
       // expect my rows of the partial sums of the whole group (senders cannot be ahead of this by a whole layer)
       if (KS > 1 && et == 0) mbar_arrive_expect_tx(bar_red, static_cast<uint32_t>(rows_all * 128));
@@ -236,18 +367,10 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
       const bool finisher = KS > 1 ? frow < rows_per : has_row;
       const int ncol4 = KS > 1 ? 4 : 8;                           // float4 groups this thread finishes
       const int fcol = slice * CC_BLOCK_N + (KS > 1 ? 16 * half : 0);
-      float4 bias4[8];
-      if (finisher && L.epi.bias) {
-        const float4* bp = reinterpret_cast<const float4*>(L.epi.bias + fcol);
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-          if (i < ncol4) bias4[i] = __ldg(bp + i);
-      } else {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) bias4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-      }
+      // (the bias of my slice sits in shared memory since the start of the kernel; the named barrier below orders it)
+      const float4* bias4 = reinterpret_cast<const float4*>(sBias + l * CC_BLOCK_N + (KS > 1 ? 16 * half : 0));
       const int act = L.epi.act;
-      bool ok = cc_epi_all(mbar_wait(bar_tfull, tphase));
+      bool ok = cc_epi_all(cc_lane0_wait(lane, [&]() { return cc_wait(bar_tfull, tphase); }));
       float4 acc4[8];
       if (ok) {
         tc_fence_after();
@@ -282,6 +405,7 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
           __syncwarp();
           if (lane == 0) {
             const int base = rank - part;                         // first CTA of my group
+#pragma unroll 1
             for (int d = 0; d < KS; ++d) {                        // rows [d rows_per, (d + 1) rows_per) belong to part d
               const int ra = max(d * rows_per, q * 16), rb = min((d + 1) * rows_per, q * 16 + 16);
               if (ra >= rb) continue;
@@ -290,10 +414,11 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
                                    mapa_shared(bar_red, base + d));
             }
           }
-          ok = cc_epi_all(mbar_wait_cluster(bar_red, rphase));
+          ok = cc_epi_all(cc_lane0_wait(lane, [&]() { return cc_wait_cluster(bar_red, rphase); }));
           if (ok && finisher) {
 #pragma unroll
             for (int c = 0; c < 4; ++c) acc4[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 1
             for (int s = 0; s < KS; ++s) {                        // fixed order: deterministic
               const uint8_t* src = sRed + (s * rows_per + frow) * 128;
 #pragma unroll
@@ -322,7 +447,7 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
               if (act == ACT_RELU) {
                 t.x = fmaxf(t.x, 0.f); t.y = fmaxf(t.y, 0.f); t.z = fmaxf(t.z, 0.f); t.w = fmaxf(t.w, 0.f);
               } else if (act != ACT_NONE) {
-                t.x = apply_act(t.x, act); t.y = apply_act(t.y, act); t.z = apply_act(t.z, act); t.w = apply_act(t.w, act);
+                t.x = apply_act_cold(t.x, act); t.y = apply_act_cold(t.y, act); t.z = apply_act_cold(t.z, act); t.w = apply_act_cold(t.w, act);
               }
               acc4[c] = t;
             }
@@ -353,8 +478,8 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
           const int nslices = Nx.N / CC_BLOCK_N;
           if (et < nslices) {
             int np = 0;
-            while (np + 1 < Nx.ks_l && (np + 1) * Nx.nkb / Nx.ks_l <= slice) ++np;     // the part that holds k-block `slice`
-            const int st = slice - np * Nx.nkb / Nx.ks_l;                                // its stage there
+            while (np + 1 < Nx.ks_l && kb_lo(Nx, np + 1) <= slice) ++np;                 // the part that holds k-block `slice`
+            const int st = slice - kb_lo(Nx, np);                                        // its stage there
             const uint32_t dst = smem_u32(sA) + static_cast<uint32_t>(((l + 1) & 1) * REGION + st * STAGE + part * rows_per * 128);
             const int rc = et * Nx.ks_l + np;
             bulk_copy_to_cluster(mapa_shared(dst, rc), smem_u32(outb), static_cast<uint32_t>(rows_per * 128),
@@ -375,7 +500,7 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, CC_NACC * CC_BLOCK_N);
+    tmem_dealloc(tmem_base, tmem_cols);
   }
   // no CTA leaves while another one of its cluster may still write into its shared memory or read a copy out of it
   // (every CTA has seen all copies addressed to it complete before it arrives here; nothing else is ordered)
@@ -383,8 +508,9 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
 }
 
 size_t mlp_cluster_smem_bytes(size_t w_smem_bytes, int a_stages, int a_stage_bytes) {
+  // (the last two terms: barriers and the two bias tables; slack for the 1024-byte alignment of the base)
   return ((2 * static_cast<size_t>(a_stages) * a_stage_bytes + 1023) & ~size_t(1023)) +
-         (w_smem_bytes < 16384 ? size_t(16384) : w_smem_bytes) + CC_RED_BYTES + 4 * static_cast<size_t>(a_stage_bytes) + 1024 + 1024;
+         (w_smem_bytes < 16384 ? size_t(16384) : w_smem_bytes) + CC_RED_BYTES + 4 * static_cast<size_t>(a_stage_bytes) + 3072 + 1024;
 }
 
 static cudaError_t cluster_kernel_ready(size_t smem) {

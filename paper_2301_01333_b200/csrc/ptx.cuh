@@ -313,19 +313,21 @@ __device__ __forceinline__ void bulk_copy_to_cluster(uint32_t dst_cluster_addr, 
 }
 // Bounded wait on an mbarrier of this CTA that CTAs of the cluster arrive on: acquire at cluster scope, so the
 // remote shared-memory stores made before those arrivals are visible afterwards.
+// (suspend_ns: the time hint of each try; waiters on the critical path were seen to wake late with long hints)
+template <uint32_t SUSPEND_NS = 20000u>
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity) {
   uint64_t t0 = 0;                                              // the global timer is slow to read: only once polling drags on
-  for (uint32_t i = 0; i < (1u << 22); ++i) {
+  for (uint32_t i = 0; i < (SUSPEND_NS >= 1000u ? (1u << 22) : (1u << 30)); ++i) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred P;\n\t"
         "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 P, [%1], %2, %3;\n\t"
         "selp.b32 %0, 1, 0, P;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity), "r"(20000u)
+        : "r"(bar), "r"(parity), "r"(SUSPEND_NS)
         : "memory");
     if (ok) return true;
-    if ((i & 15u) == 15u) {
+    if ((i & (SUSPEND_NS >= 1000u ? 15u : 1023u)) == 0u && i) {
       const uint64_t t = globaltimer_ns();
       if (t0 == 0) t0 = t;
       else if (t - t0 > 2000000000ull) break;

@@ -211,6 +211,9 @@ def test_mlp_f32_chain_kernel_cluster_sizes(B, batch, dims, ks):
     (17, (45, 96, 64), 8),                # ragged rows and a first layer whose row pitch TMA cannot address
     (8, (64, 128, 64), 8),                # first layer fed by TMA
     (24, (200, 160, 288, 32, 64), 16),    # five k-blocks over two parts, nine slices, a one-slice layer in the middle
+    (32, (13, 1024, 64), 8),              # recomputed first layer at its widest (256 columns per CTA)
+    (40, (100, 256, 256, 128, 32), 16),   # first layer too deep to recompute: distributed like the others
+    (32, (60, 64, 32), 8),                # recomputed first layer with two k-blocks
 ])
 def test_mlp_f32_chain_inside_one_cluster(B, batch, dims, cluster):
     w = W.mlp_f32(batch=batch, dims=dims)
@@ -225,7 +228,7 @@ def test_mlp_f32_chain_inside_one_cluster(B, batch, dims, cluster):
 
 
 def test_mlp_f32_too_large_for_one_cluster_stays_grid_wide(B):
-    for batch, dims in ((65, (13, 512, 256, 128)), (32, (13, 1024, 64)), (40, (100, 256, 256, 128, 32))):
+    for batch, dims in ((65, (13, 512, 256, 128)), (32, (13, 1024, 1024, 64)), (48, (300, 512, 512, 256, 128))):
         w = W.mlp_f32(batch=batch, dims=dims)
         got, plan = run_gpu(B, w)
         assert "fused chain" in plan and "inside one cluster" not in plan
