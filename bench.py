@@ -46,7 +46,7 @@ GRAPH_STEPS = {"c1": 256, "c2": 256, "c3": 256, "c4": 50, "c5": 50}     # execut
 TRAFFIC_BYTES_PER_LAUNCH = {"c5": 126.65e6, "c3": 18.9e6, "c4": 84.8e6}
 TRAFFIC_SOURCE = {"c5": "profiles/gemm_tc2_bf16_c5_ffn_one_launch.md (capture of the one-launch FFN, 70.0 MB read + 56.7 MB written)",
                   "c3": "profiles/sdpa_small_c3_attention.md (reads; the 6.3 MB of output were still in the L2 when the launch ended)", "c4": "profiles/sdpa_tc_c3_c4_attention.md"}
-DOMINANT_KERNEL = {"c1": "mlp_chain_kernel<tf32>", "c2": "mlp_chain_kernel<i8>", "c3": "sdpa_small_kernel (bf16, one unit per CTA)",
+DOMINANT_KERNEL = {"c1": "mlp_cluster_kernel (tf32, whole chain inside one thread-block cluster)", "c2": "mlp_chain_kernel<i8>", "c3": "sdpa_small_kernel (bf16, one unit per CTA)",
                    "c4": "sdpa_tc_kernel<int8>", "c5": "gemm_tc2_kernel<bf16, bf16 out> (both FFN GEMMs in one launch)"}
 
 
@@ -556,7 +556,11 @@ def main():
             # coarse-grain fusion ablation (Section VII, Fig. 8): the whole chain in one persistent launch, one
             # launch per layer (fine-grain fusion only), and the CUDA-core kernels
             abl = {"fused_chain": {"us_cold": us, "us_warm": res["us_per_subgraph_warm"], "launches": reps[0].c.launches}}
-            for label, opts in (("per_layer", {"no_chain_fusion": True}), ("cuda_core_per_layer", {"force_generic": True})):
+            variants = [("per_layer", {"no_chain_fusion": True}), ("cuda_core_per_layer", {"force_generic": True})]
+            if "inside one cluster" in reps[0].c.plan:
+                # the same chain spread over the whole GPU, activations through the L2 behind a grid barrier
+                variants.insert(0, ("grid_wide_chain", {"grid_wide_chain": True}))
+            for label, opts in variants:
                 _, areps, an = time_config(B, name, steps, args.warmup, local, **opts)
                 cold = max_over_ranks(run_timed(areps, an, steps, local, barrier)) * 1e3 / steps
                 warm = max_over_ranks(run_timed(areps[:1], 1, warm_steps, local, barrier)) * 1e3 / warm_steps
