@@ -738,7 +738,7 @@ def test_repeated_runs_are_bitwise_identical(B):
         assert np.array_equal(res[0], res[1]) and np.array_equal(res[0], res[2])
 
 
-@pytest.mark.parametrize("which", ["chain", "two_layers_one_launch", "attention"])
+@pytest.mark.parametrize("which", ["chain", "chain_in_one_cluster", "two_layers_one_launch", "attention"])
 def test_captured_executes_replay_correctly(B, which):
     # gc_execute after the first call is a pure sequence of kernel launches: captured into a CUDA graph and replayed,
     # it must give the same results, also for the kernels that synchronise through counters in global memory
@@ -746,11 +746,15 @@ def test_captured_executes_replay_correctly(B, which):
     import torch
     if which == "chain":
         w = W.mlp_int8(batch=128, dims=(479, 1024, 512, 32), final="none", per_channel=True, x_zp=3, act_zp=2)
+    elif which == "chain_in_one_cluster":
+        w = W.mlp_f32()
     elif which == "two_layers_one_launch":
         w = W.ffn_bf16(tokens=4900, d_model=1024, d_ff=1024)
     else:
         w = W.mha_int8(batch=2, heads=4, seq=384, head_dim=64)
     c = B.CompiledPartition(w.graph, 0)
+    if which == "chain_in_one_cluster":
+        assert "inside one cluster" in c.plan
     ins = B.device_inputs(w)
     outs = B.device_outputs(w.graph)
     s = torch.cuda.Stream()
@@ -784,6 +788,8 @@ def test_captured_executes_replay_correctly(B, which):
     ref = oracle(w)
     if which == "chain":
         assert np.array_equal(replayed, ref)
+    elif which == "chain_in_one_cluster":
+        assert np.abs(replayed.astype(np.float64) - ref).max() <= 5e-3 * np.abs(ref).max()
     elif which == "attention":
         check_int8_attention(replayed, ref)
     else:
