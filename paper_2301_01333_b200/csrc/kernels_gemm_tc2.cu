@@ -179,18 +179,13 @@ __global__ void __launch_bounds__(F2_THREADS, 1) gemm_tc2_kernel(const __grid_co
           if (l == 1 && kb % K_PER_TILE == 0) {
             const int j = kb / K_PER_TILE;
             if (j < p.L[0].n_tiles && (j >= 32 || !((known >> j) & 1u))) {
-              uint64_t t0 = 0;                                    // the global timer is slow to read: only once polling drags on
+              const uint64_t t0 = globaltimer_ns();
               uint32_t spins = 0;
               while (f2_ld_acquire(tile_ready + j) < tile_target) {
-                if ((++spins & 255u) == 0) {
-                  const uint64_t t = globaltimer_ns();
-                  if (t0 == 0) {
-                    t0 = t;
-                  } else if (t - t0 > 2000000000ull) {
-                    report(p.status, DEV_TIMEOUT_PRODUCER);
-                    failed = true;
-                    break;
-                  }
+                if ((++spins & 255u) == 0 && globaltimer_ns() - t0 > 2000000000ull) {
+                  report(p.status, DEV_TIMEOUT_PRODUCER);
+                  failed = true;
+                  break;
                 }
               }
               if (failed) break;
