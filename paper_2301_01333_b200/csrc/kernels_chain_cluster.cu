@@ -39,7 +39,8 @@ constexpr int CC_NACC = 4;
 constexpr int CC_K_ELEMS = 32;           // fp32 elements per 128-byte k-block
 constexpr int CC_RED_BYTES = 128 * 128;  // partial sums received: at most 128 rows of 128 bytes
 constexpr int CC_T0_COL = CC_NACC * CC_BLOCK_N;   // tensor-memory column of the recomputed first layer's accumulator
-constexpr int CC_T0_MAX = 256;                     // its widest form
+constexpr int CC_T0_MAX = 256;                     // its widest form (first-layer columns per CTA)
+constexpr int CC_T0_STRIDE = 64;                   // columns between its 128-row blocks (at most 64 batch rows)
 
 // AND of a flag over the 128 threads of the four epilogue warps (named barrier 1): after a bounded wait every one of
 // them takes the same branch, so the named barriers that follow are reached by all or by none.
@@ -93,7 +94,7 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
   float* sBias0 = reinterpret_cast<float*>(bars + 2 * CHAIN_MAX_LAYERS + 6);   // [CC_T0_MAX] first-layer bias of my columns
   float* sBias = sBias0 + CC_T0_MAX;                              // [CHAIN_MAX_LAYERS][32] bias of my slice of every layer
   const bool recompute = p.recompute_first != 0;
-  const int tmem_cols = recompute ? 512 : CC_NACC * CC_BLOCK_N;
+  const int tmem_cols = recompute ? 256 : CC_NACC * CC_BLOCK_N;     // (+ two blocks of CC_T0_STRIDE columns)
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rank = static_cast<int>(cluster_ctarank());
 
@@ -208,6 +209,7 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
     const int lo = rc0 ? 0 : kb_lo(L, part), my_nkb = rc0 ? L.nkb : kb_lo(L, part + 1) - lo;
     // (recomputed first layer: the k-blocks of the second layer that are mine, i.e. 32-column groups to produce)
     const int n1 = rc0 ? kb_lo(p.L[1], part_of(p.L[1]) + 1) - kb_lo(p.L[1], part_of(p.L[1])) : 0;
+    const int nb0 = min(64, (L.M + 15) / 16 * 16);               // batch rows as the N of the transposed first layer
     const bool last = l + 1 == p.n_layers;
     uint8_t* region = sA + (l & 1) * REGION;
     uint8_t* send = sSend + (l & 1) * STAGE;
@@ -231,16 +233,23 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
                        : (l == 1 && recompute) ? cc_wait(bar_a1, 0) : cc_wait_cluster(bar_a + 8 * l, 0);
           if (ok && rc0) {
             tc_fence_after();
-            const uint32_t a0 = smem_u32(region), b0 = smem_u32(sW) + L.w_smem_off;
-            // M = 64, N = 32 n1 (N field: bits 17..22 in units of 8); one accumulator: the few MMAs form a chain
-            const uint32_t idesc = (L.idesc & ~((0x1Fu << 24) | (0x3Fu << 17))) | ((64u >> 4) << 24) |
-                                   ((static_cast<uint32_t>(n1 * CC_BLOCK_N) >> 3) << 17);
+            const uint32_t x0 = smem_u32(region), w0 = smem_u32(sW) + L.w_smem_off;
+            // The product is taken transposed: the weight rows (= my 32 n1 first-layer columns, 128 per MMA) are the
+            // M side, the batch rows the N side, so that all 128 epilogue threads own an accumulator row (a column
+            // of the activation) instead of the 32 that would own a batch row.  M = 128, N = batch rows rounded up
+            // to 16 (N field: bits 17..22 in units of 8; M field: bits 24..28 in units of 16).
+            const uint32_t idesc = (L.idesc & ~((0x1Fu << 24) | (0x3Fu << 17))) | ((128u >> 4) << 24) |
+                                   ((static_cast<uint32_t>(nb0) >> 3) << 17);
 #pragma unroll 1
-            for (int i = 0; i < my_nkb; ++i) {
+            for (int m = 0; m * 128 < n1 * CC_BLOCK_N; ++m) {
+#pragma unroll 1
+              for (int i = 0; i < my_nkb; ++i) {
 #pragma unroll
-              for (int k = 0; k < 4; ++k)
-                umma_ss<KIND_TF32>(tmem_base + CC_T0_COL, make_smem_desc(a0 + i * STAGE + 32 * k, 16, 1024, SWZ_128B),
-                                   make_smem_desc(b0 + i * n1 * (CC_BLOCK_N * 128) + 32 * k, 16, 1024, SWZ_128B), idesc, (i | k) != 0);
+                for (int k = 0; k < 4; ++k)
+                  umma_ss<KIND_TF32>(tmem_base + CC_T0_COL + m * CC_T0_STRIDE,
+                                     make_smem_desc(w0 + i * n1 * (CC_BLOCK_N * 128) + m * (128 * 128) + 32 * k, 16, 1024, SWZ_128B),
+                                     make_smem_desc(x0 + i * STAGE + 32 * k, 16, 1024, SWZ_128B), idesc, (i | k) != 0);
+              }
             }
             umma_commit(bar_tfull);
           } else if (ok) {
@@ -273,7 +282,24 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
         const int a_rows = STAGE / 128;
         const int64_t kbytes = static_cast<int64_t>(L.K) * 4;
         const uint8_t* src_row = static_cast<const uint8_t*>(p.pack_src) + static_cast<int64_t>(r) * p.pack_src_pitch;
-        if (r < a_rows) {
+        const bool words_ok = ((reinterpret_cast<uintptr_t>(p.pack_src) | static_cast<uintptr_t>(p.pack_src_pitch)) & 3) == 0;
+        if (r < a_rows && words_ok) {
+          // rows of whole 32-bit words (every fp32 input): 32 independent predicated loads per k-block and not one
+          // branch (a lone warp pays about 30 clocks for each)
+          const uint32_t* src_w = reinterpret_cast<const uint32_t*>(src_row);
+          const int kmax = r < L.M ? L.K : 0;
+#pragma unroll 1
+          for (int i = 0; i < my_nkb; ++i) {
+            uint8_t* dst = region + i * STAGE + (r >> 3) * 1024 + (r & 7) * 128;
+            const int k0 = (lo + i) * CC_K_ELEMS;
+            uint32_t w[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) w[j] = (k0 + j < kmax) ? __ldg(src_w + k0 + j) : 0u;
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+              *reinterpret_cast<uint4*>(dst + ((c ^ (r & 7)) << 4)) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+          }
+        } else if (r < a_rows) {
 #pragma unroll 1
           for (int i = 0; i < my_nkb; ++i) {
             uint8_t* dst = region + i * STAGE + (r >> 3) * 1024 + (r & 7) * 128;
@@ -306,41 +332,50 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
         if (lane == 0) mbar_arrive(bar_a0);
       }
       if (rc0) {
-        // Recomputed first layer: my accumulator row holds the 32 n1 columns that are my k-blocks of the second layer's
-        // A operand; bias and activation applied, each group of 32 goes to its stage as one swizzled 128-byte row.
-        const int row = q * 16 + lane;
-        const bool has_row = lane < 16 && row < STAGE / 128;
+        // Recomputed first layer, computed transposed: accumulator row = one of my 32 n1 first-layer columns (warp q of
+        // block m owns columns 128 m + 32 q .. + 32, i.e. k-block 4 m + q of the second layer's A operand),
+        // accumulator column = batch row.  Bias and activation applied, the 32 lanes of a warp write one swizzled
+        // 128-byte operand row per batch row.
         const int act = L.epi.act;
+        const bool relu = act == ACT_RELU, other_act = act != ACT_NONE && !relu;
         uint8_t* region1 = sA + REGION;
+        const int rows_st = min(STAGE / 128, nb0);               // batch rows that exist in a stage
         const bool ok = cc_epi_all(cc_lane0_wait(lane, [&]() { return cc_wait(bar_tfull, tphase); }));   // (also orders the writes of sBias0 before its reads)
         if (ok) {
           tc_fence_after();
-          const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + CC_T0_COL;
 #pragma unroll 1
-          for (int j = 0; j < n1; ++j) {
-            uint32_t r[32];
-            tmem_ld32(t_row + j * CC_BLOCK_N, r);
-            tmem_wait_ld();
-            if (has_row) {
-              // all loads, then all arithmetic, then all stores: a lone warp per scheduler lives on instruction-level
-              // parallelism, and a store into the stage may alias the bias for all the compiler knows
-              float4 t[8];
+          for (int m = 0; m * 128 < n1 * CC_BLOCK_N; ++m) {
+            const int j = m * 4 + q;                              // my k-block of the second layer
+            if (j >= n1) break;                                   // (warp-uniform)
+            const float bias = sBias0[j * CC_BLOCK_N + lane];
+            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + CC_T0_COL + m * CC_T0_STRIDE;
+            uint8_t* st = region1 + j * STAGE + (lane & 3) * 4;
+#pragma unroll 1
+            for (int h = 0; h * 32 < rows_st; ++h) {
+              uint32_t r[32];
+              tmem_ld32(t_row + h * 32, r);
+              tmem_wait_ld();
 #pragma unroll
-              for (int c = 0; c < 8; ++c) t[c] = *reinterpret_cast<const float4*>(sBias0 + j * CC_BLOCK_N + 4 * c);
+              for (int i = 0; i < 32; ++i) {                      // (no branch per element: see the finishing step below)
+                const float t = __fadd_rn(__uint_as_float(r[i]), bias);
+                r[i] = __float_as_uint(relu ? fmaxf(t, 0.f) : t);
+              }
+              if (other_act) {
 #pragma unroll
-              for (int c = 0; c < 8; ++c) {
-                t[c].x = __fadd_rn(__uint_as_float(r[4 * c]), t[c].x); t[c].y = __fadd_rn(__uint_as_float(r[4 * c + 1]), t[c].y);
-                t[c].z = __fadd_rn(__uint_as_float(r[4 * c + 2]), t[c].z); t[c].w = __fadd_rn(__uint_as_float(r[4 * c + 3]), t[c].w);
-                if (act == ACT_RELU) {
-                  t[c].x = fmaxf(t[c].x, 0.f); t[c].y = fmaxf(t[c].y, 0.f); t[c].z = fmaxf(t[c].z, 0.f); t[c].w = fmaxf(t[c].w, 0.f);
-                } else if (act != ACT_NONE) {
-                  t[c].x = apply_act_cold(t[c].x, act); t[c].y = apply_act_cold(t[c].y, act);
-                  t[c].z = apply_act_cold(t[c].z, act); t[c].w = apply_act_cold(t[c].w, act);
+                for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(apply_act_cold(__uint_as_float(r[i]), act));
+              }
+              // row brow, 16-byte chunk (lane / 4) XOR (brow mod 8), word lane mod 4.  The rows of a stage come in groups
+              // of 8: one test per group, not one per row (a predicated store becomes a branch, and a lone warp pays
+              // about 30 clocks for each).
+#pragma unroll
+              for (int g8 = 0; g8 < 4; ++g8) {
+                if (h * 32 + g8 * 8 < rows_st) {
+#pragma unroll
+                  for (int i = 0; i < 8; ++i)
+                    *reinterpret_cast<float*>(st + (h * 4 + g8) * 1024 + i * 128 + (((lane >> 2) ^ i) << 4)) =
+                        __uint_as_float(r[g8 * 8 + i]);
                 }
               }
-              uint8_t* my = region1 + j * STAGE + (row >> 3) * 1024 + (row & 7) * 128;
-#pragma unroll
-              for (int c = 0; c < 8; ++c) *reinterpret_cast<float4*>(my + ((c ^ (row & 7)) << 4)) = t[c];
             }
           }
           tc_fence_before();
@@ -417,7 +452,7 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
           ok = cc_epi_all(cc_lane0_wait(lane, [&]() { return cc_wait_cluster(bar_red, rphase); }));
           if (ok && finisher) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) acc4[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int c = 0; c < 8; ++c) acc4[c] = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 1
             for (int s = 0; s < KS; ++s) {                        // fixed order: deterministic
               const uint8_t* src = sRed + (s * rows_per + frow) * 128;
@@ -437,19 +472,24 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
       }
       if (ok) {
         if (finisher) {
-          // bias and activation (fp32 chains only: this kernel takes no other)
+          // bias and activation (fp32 chains only: this kernel takes no other).  No branch per element: a lone warp
+          // pays dozens of clocks for every one, so ReLU / none is a select, and anything else one pass of its own
+          // behind a single branch.
+          const bool relu = act == ACT_RELU;
 #pragma unroll
           for (int c = 0; c < 8; ++c) {
-            if (c < ncol4) {
-              float4 t = acc4[c];
-              t.x = __fadd_rn(t.x, bias4[c].x); t.y = __fadd_rn(t.y, bias4[c].y);
-              t.z = __fadd_rn(t.z, bias4[c].z); t.w = __fadd_rn(t.w, bias4[c].w);
-              if (act == ACT_RELU) {
-                t.x = fmaxf(t.x, 0.f); t.y = fmaxf(t.y, 0.f); t.z = fmaxf(t.z, 0.f); t.w = fmaxf(t.w, 0.f);
-              } else if (act != ACT_NONE) {
-                t.x = apply_act_cold(t.x, act); t.y = apply_act_cold(t.y, act); t.z = apply_act_cold(t.z, act); t.w = apply_act_cold(t.w, act);
-              }
-              acc4[c] = t;
+            float4 t = acc4[c];
+            t.x = __fadd_rn(t.x, bias4[c & (ncol4 - 1)].x); t.y = __fadd_rn(t.y, bias4[c & (ncol4 - 1)].y);
+            t.z = __fadd_rn(t.z, bias4[c & (ncol4 - 1)].z); t.w = __fadd_rn(t.w, bias4[c & (ncol4 - 1)].w);
+            t.x = relu ? fmaxf(t.x, 0.f) : t.x; t.y = relu ? fmaxf(t.y, 0.f) : t.y;
+            t.z = relu ? fmaxf(t.z, 0.f) : t.z; t.w = relu ? fmaxf(t.w, 0.f) : t.w;
+            acc4[c] = t;
+          }
+          if (act != ACT_NONE && !relu) {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              acc4[c].x = apply_act_cold(acc4[c].x, act); acc4[c].y = apply_act_cold(acc4[c].y, act);
+              acc4[c].z = apply_act_cold(acc4[c].z, act); acc4[c].w = apply_act_cold(acc4[c].w, act);
             }
           }
           const int grow = part * rows_per + frow;                // row of the tile
