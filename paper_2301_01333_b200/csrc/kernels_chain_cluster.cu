@@ -438,28 +438,28 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
           }
           fence_proxy_async_smem();
           __syncwarp();
-          if (lane == 0) {
-            const int base = rank - part;                         // first CTA of my group
-#pragma unroll 1
-            for (int d = 0; d < KS; ++d) {                        // rows [d rows_per, (d + 1) rows_per) belong to part d
-              const int ra = max(d * rows_per, q * 16), rb = min((d + 1) * rows_per, q * 16 + 16);
-              if (ra >= rb) continue;
+          if (lane < KS) {                                        // lane d serves the CTA that finishes rows [d rows_per, + rows_per)
+            const int base = rank - part, d = lane;               // (base: first CTA of my group)
+            const int ra = max(d * rows_per, q * 16), rb = min((d + 1) * rows_per, q * 16 + 16);
+            if (ra < rb)
               bulk_copy_to_cluster(mapa_shared(smem_u32(sRed) + static_cast<uint32_t>((part * rows_per + ra - d * rows_per) * 128), base + d),
                                    smem_u32(send) + static_cast<uint32_t>(ra * 128), static_cast<uint32_t>((rb - ra) * 128),
                                    mapa_shared(bar_red, base + d));
-            }
           }
           ok = cc_epi_all(cc_lane0_wait(lane, [&]() { return cc_wait_cluster(bar_red, rphase); }));
           if (ok && finisher) {
 #pragma unroll
             for (int c = 0; c < 8; ++c) acc4[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 1
-            for (int s = 0; s < KS; ++s) {                        // fixed order: deterministic
+#pragma unroll
+            for (int s = 0; s < 4; ++s) {                         // fixed order: deterministic; parts beyond KS add zero
+              // (all four loads are issued - the rows exist in the buffer - and a select drops the surplus ones: no
+              // branch per part)
               const uint8_t* src = sRed + (s * rows_per + frow) * 128;
 #pragma unroll
               for (int c = 0; c < 4; ++c) {
-                const float4 v = *reinterpret_cast<const float4*>(src + (((half * 4 + c) ^ (frow & 7)) << 4));
-                acc4[c].x += v.x; acc4[c].y += v.y; acc4[c].z += v.z; acc4[c].w += v.w;
+                float4 v = *reinterpret_cast<const float4*>(src + (((half * 4 + c) ^ (frow & 7)) << 4));
+                const bool use = s < KS;
+                acc4[c].x += use ? v.x : 0.f; acc4[c].y += use ? v.y : 0.f; acc4[c].z += use ? v.z : 0.f; acc4[c].w += use ? v.w : 0.f;
               }
             }
           }
