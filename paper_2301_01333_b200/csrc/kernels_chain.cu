@@ -97,6 +97,9 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
   const int CH_STAGES = p.a_stages;
   const int CH_A_STAGE_BYTES = p.a_stage_bytes;
   const int KS = p.ks;                                            // CTAs per cluster = parts of the reduction axis
+  // (1, 2 or 4: shifts and masks instead of divisions, which cost a lone thread a hundred clocks each on the way from
+  // one layer to the next)
+  const int KS_SH = __ffs(KS) - 1;
   uint8_t* sA = smem;                                             // a_stages x a_stage_bytes
   // the weight slices (padded to at least 16 KB) follow the ring, so the 128-row MMA reads of the last stages
   // stay inside this CTA's shared memory
@@ -116,8 +119,8 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
   const int ksr = KS > 1 ? static_cast<int>(cluster_ctarank()) : 0;   // my part of the reduction axis
   // CTA index -> (row tile, 32-column slice, part of the reduction axis): batches above 128 rows are cut into row
   // tiles that run as independent CTAs (rows of a matmul are independent); only the grid barrier joins them
-  const int cta = (blockIdx.x / KS) % p.slices;                   // my 32-column slice
-  const int row0 = (blockIdx.x / KS) / p.slices * 128;            // first row of my row tile
+  const int cta = static_cast<int>(blockIdx.x >> KS_SH) % p.slices;   // my 32-column slice
+  const int row0 = static_cast<int>(blockIdx.x >> KS_SH) / p.slices * 128;   // first row of my row tile
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < CH_STAGES; ++s) {
@@ -148,8 +151,8 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
   if (!p.early_weights) asm volatile("griddepcontrol.wait;" ::: "memory");
 
   // my k-blocks of layer L: [kb_lo, kb_hi)
-  auto kb_lo = [&](const ChainLayer& L) { return ksr * L.nkb / KS; };
-  auto kb_hi = [&](const ChainLayer& L) { return (ksr + 1) * L.nkb / KS; };
+  auto kb_lo = [&](const ChainLayer& L) { return (ksr * L.nkb) >> KS_SH; };
+  auto kb_hi = [&](const ChainLayer& L) { return ((ksr + 1) * L.nkb) >> KS_SH; };
 
   // every layer's weight slice starts moving now (constants: they do not depend on earlier layers)
   if (warp == 0 && lane == 0) {
@@ -220,7 +223,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
       report(p.status, DEV_TIMEOUT_OTHER);
     }
   };
-  const int rows_per = 128 / KS; // rows of the tile this CTA finishes
+  const int rows_per = 128 >> KS_SH; // rows of the tile this CTA finishes
   for (int l = 0; l < p.n_layers && !failed; ++l) {
     // A by-value copy: fields read through a reference into the parameter space are re-fetched around every
     // store (possible aliasing) at a few hundred clocks each, which made a 16-element epilogue cost thousands.
@@ -283,14 +286,14 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
                   int64_t nv = kbytes - off;                                             // valid bytes of this chunk
                   nv = row0 + r < L.M ? (nv > 16 ? 16 : nv) : 0;
                   uint32_t o[4] = {0u, 0u, 0u, 0u};
-                  if (nv > 0) {
+                  {   // (no branch on nv: with nothing valid every load below is predicated off and every mask is zero)
                     const uintptr_t a = reinterpret_cast<uintptr_t>(src_row + off);
                     const uint32_t sh = static_cast<uint32_t>(a & 3);
                     const uint32_t* aw = reinterpret_cast<const uint32_t*>(a - sh);
                     uint32_t w[5];
 #pragma unroll
                     for (int j = 0; j < 5; ++j)   // word j holds chunk bytes [4j - sh, 4j - sh + 4): load it only if one is valid
-                      w[j] = (4 * j - static_cast<int>(sh) < nv) ? __ldg(aw + j) : 0u;
+                      w[j] = (nv > 0 && 4 * j - static_cast<int>(sh) < nv) ? __ldg(aw + j) : 0u;
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                       const uint32_t v = __funnelshift_r(w[j], w[j + 1], sh * 8);
@@ -351,7 +354,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
             } else {
               // my warp's 32 rows belong to CTA `dest` of the cluster: 128 bytes per row into its buffer
               const int row = q * 32 + lane;
-              const int dest = row / rows_per, lrow = row % rows_per;
+              const int dest = row >> (7 - KS_SH), lrow = row & (rows_per - 1);
               // stage the row locally (16-byte chunks XOR-swizzled by the row), then one bulk copy per warp: its 32
               // rows are contiguous here and in the owner's buffer
               uint8_t* my = sSend + row * 128;
@@ -370,18 +373,24 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
                   uint32_t a[16];
 #pragma unroll
                   for (int i = 0; i < 16; ++i) a[i] = 0u;
-                  for (int s = 0; s < KS; ++s) {
+                  // All four possible parts are loaded (what lies behind the buffer for KS < 4 is shared memory of this
+                  // CTA) and a select drops the surplus ones: no branch per part - a lone warp pays about 30 clocks for
+                  // each.  Fixed order: exact for s32, deterministic for fp32.
+#pragma unroll
+                  for (int s = 0; s < 4; ++s) {
                     const uint8_t* src = sRed + (s * rows_per + frow) * 128;
+                    const bool use = s < KS;
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                       const uint4 v = *reinterpret_cast<const uint4*>(src + (((half * 4 + c) ^ (frow & 7)) << 4));
                       if constexpr (KIND == KIND_I8) {
-                        a[4 * c] += v.x; a[4 * c + 1] += v.y; a[4 * c + 2] += v.z; a[4 * c + 3] += v.w;
+                        a[4 * c] += use ? v.x : 0u; a[4 * c + 1] += use ? v.y : 0u;
+                        a[4 * c + 2] += use ? v.z : 0u; a[4 * c + 3] += use ? v.w : 0u;
                       } else {
-                        a[4 * c] = __float_as_uint(__uint_as_float(a[4 * c]) + __uint_as_float(v.x));
-                        a[4 * c + 1] = __float_as_uint(__uint_as_float(a[4 * c + 1]) + __uint_as_float(v.y));
-                        a[4 * c + 2] = __float_as_uint(__uint_as_float(a[4 * c + 2]) + __uint_as_float(v.z));
-                        a[4 * c + 3] = __float_as_uint(__uint_as_float(a[4 * c + 3]) + __uint_as_float(v.w));
+                        a[4 * c] = __float_as_uint(__uint_as_float(a[4 * c]) + (use ? __uint_as_float(v.x) : 0.f));
+                        a[4 * c + 1] = __float_as_uint(__uint_as_float(a[4 * c + 1]) + (use ? __uint_as_float(v.y) : 0.f));
+                        a[4 * c + 2] = __float_as_uint(__uint_as_float(a[4 * c + 2]) + (use ? __uint_as_float(v.z) : 0.f));
+                        a[4 * c + 3] = __float_as_uint(__uint_as_float(a[4 * c + 3]) + (use ? __uint_as_float(v.w) : 0.f));
                       }
                     }
                   }
