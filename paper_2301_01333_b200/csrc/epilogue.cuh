@@ -184,4 +184,36 @@ __device__ __forceinline__ void epi_store1(uint32_t raw, void* dst_row, int n, c
   }
 }
 
+// ---- the graph-entry reorder as a pre-op (Section V: fused "only at the entry point of the graph") ----
+// One 128-byte k-block of one input row, read from an arbitrarily aligned source with aligned 32-bit loads and
+// written where TMA would have put it: row r of a 128B-swizzled K-major tile (8-row groups of 1024 bytes, 16-byte chunk
+// index XOR row mod 8).  `src` points at the k-block's first byte in the row, `nv` (0..128) is the number of valid
+// bytes from there (0 for rows beyond the matrix); the rest is zero filled.  Straight-line code: 33 predicated loads
+// that are independent of one another (one memory round trip), 32 funnel shifts, masks by selects - no branch, no
+// 64-bit arithmetic (the code runs once per launch in a warp that is alone on its scheduler, where a branch costs
+// about 30 clocks).
+__device__ __forceinline__ void pack_row_kblock(const uint8_t* src, int nv, uint8_t* dst_tile, int r) {
+  const uintptr_t a = reinterpret_cast<uintptr_t>(src);
+  const int sh = static_cast<int>(a & 3);
+  const uint32_t* aw = reinterpret_cast<const uint32_t*>(a - sh);
+  uint32_t w[33];
+#pragma unroll
+  for (int u = 0; u < 33; ++u)   // word u holds k-block bytes [4u - sh, 4u - sh + 4): load it only if one of them is valid
+    w[u] = (nv > 0 && 4 * u - sh < nv) ? __ldg(aw + u) : 0u;
+  uint8_t* dst = dst_tile + (r >> 3) * 1024 + (r & 7) * 128;
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int t = 4 * c + j;
+      const uint32_t v = __funnelshift_r(w[t], w[t + 1], static_cast<uint32_t>(sh) * 8u);
+      const int left = nv - 4 * t;                                // valid bytes of this word
+      const uint32_t part = (1u << (8 * (left & 3))) - 1u;        // (used for left = 1..3 only)
+      o[j] = left >= 4 ? v : (left <= 0 ? 0u : (v & part));
+    }
+    *reinterpret_cast<uint4*>(dst + ((c ^ (r & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
 }  // namespace gc

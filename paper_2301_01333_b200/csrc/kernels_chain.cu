@@ -61,7 +61,7 @@ __device__ __forceinline__ bool grid_barrier(unsigned long long* ctr, unsigned l
     // TMA loads: proxy fence on the global space, then a releasing reduction (no return value to wait for)
     asm volatile("fence.proxy.async.global;" ::: "memory");
     asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(ctr), "l"(1ULL) : "memory");
-    uint64_t t0 = 0;                                            // the global timer is slow to read: only once polling drags on
+    uint64_t t0 = 0;
     uint32_t i = 0;
     while (ld_acquire_u64(ctr) < target) {
       if ((++i & 1023u) == 0) {
@@ -269,40 +269,15 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
         } else {
           const int q = warp & 3;
           if (manual_a) {
-            // Row r of my k-blocks (thread per row): 16-byte chunks assembled from aligned 32-bit words of the
-            // (arbitrarily aligned) source row with funnel shifts, zero beyond the row's K bytes and beyond row M,
-            // stored where TMA would have put them (128-byte rows, 8-row groups of 1024 bytes, 16-byte chunk index
-            // XOR row mod 8).  All loads of a thread are independent, so one memory round trip covers them.
+            // Row r of my k-blocks (thread per row), realigned in registers and stored where TMA would have put it.
             const int r = q * 32 + lane;
             const int a_rows = CH_A_STAGE_BYTES / 128;
-            const int64_t kbytes = static_cast<int64_t>(L.K) * ESZ;
+            const int kbytes = row0 + r < L.M ? L.K * ESZ : 0;  // valid bytes of my row (none beyond the matrix)
             const uint8_t* src_row = static_cast<const uint8_t*>(p.pack_src) + static_cast<int64_t>(row0 + r) * p.pack_src_pitch;
             if (r < a_rows) {
               for (int i = 0; i < my_nkb; ++i) {
-                uint8_t* dst = sA + i * CH_A_STAGE_BYTES + (r >> 3) * 1024 + (r & 7) * 128;
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                  const int64_t off = static_cast<int64_t>(lo + i) * 128 + c * 16;     // byte offset inside the row
-                  int64_t nv = kbytes - off;                                             // valid bytes of this chunk
-                  nv = row0 + r < L.M ? (nv > 16 ? 16 : nv) : 0;
-                  uint32_t o[4] = {0u, 0u, 0u, 0u};
-                  {   // (no branch on nv: with nothing valid every load below is predicated off and every mask is zero)
-                    const uintptr_t a = reinterpret_cast<uintptr_t>(src_row + off);
-                    const uint32_t sh = static_cast<uint32_t>(a & 3);
-                    const uint32_t* aw = reinterpret_cast<const uint32_t*>(a - sh);
-                    uint32_t w[5];
-#pragma unroll
-                    for (int j = 0; j < 5; ++j)   // word j holds chunk bytes [4j - sh, 4j - sh + 4): load it only if one is valid
-                      w[j] = (nv > 0 && 4 * j - static_cast<int>(sh) < nv) ? __ldg(aw + j) : 0u;
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                      const uint32_t v = __funnelshift_r(w[j], w[j + 1], sh * 8);
-                      const int64_t left = nv - 4 * j;
-                      o[j] = left >= 4 ? v : (left <= 0 ? 0u : (v & ((1u << (8 * static_cast<int>(left))) - 1u)));
-                    }
-                  }
-                  *reinterpret_cast<uint4*>(dst + ((c ^ (r & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
-                }
+                const int off = (lo + i) * 128;                  // byte offset of the k-block inside the row
+                pack_row_kblock(src_row + off, min(max(kbytes - off, 0), 128), sA + i * CH_A_STAGE_BYTES, r);
               }
             }
             fence_proxy_async_smem();

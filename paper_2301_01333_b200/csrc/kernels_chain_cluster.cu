@@ -275,9 +275,8 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
       const int q = warp & 3;
       const int et = threadIdx.x - 64;                            // 0..127
       if (l == 0 && manual_a) {
-        // Row r of my k-blocks (thread per row): 16-byte chunks assembled from aligned 32-bit words of the
-        // (arbitrarily aligned) source row with funnel shifts, zero beyond the row's K bytes and beyond row M, stored
-        // where TMA would have put them (128-byte rows, 8-row groups of 1024 bytes, chunk index XOR row mod 8).
+        // Row r of my k-blocks (thread per row), zero beyond the row's K bytes and beyond row M, stored where TMA would
+        // have put them (128-byte rows, 8-row groups of 1024 bytes, chunk index XOR row mod 8).
         const int r = et;
         const int a_rows = STAGE / 128;
         const int64_t kbytes = static_cast<int64_t>(L.K) * 4;
@@ -300,31 +299,11 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
               *reinterpret_cast<uint4*>(dst + ((c ^ (r & 7)) << 4)) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
           }
         } else if (r < a_rows) {
+          const int kb_bytes = r < L.M ? static_cast<int>(kbytes) : 0;
 #pragma unroll 1
           for (int i = 0; i < my_nkb; ++i) {
-            uint8_t* dst = region + i * STAGE + (r >> 3) * 1024 + (r & 7) * 128;
-#pragma unroll 1
-            for (int c = 0; c < 8; ++c) {
-              const int64_t off = static_cast<int64_t>(lo + i) * 128 + c * 16;
-              int64_t nv = kbytes - off;
-              nv = r < L.M ? (nv > 16 ? 16 : nv) : 0;
-              uint32_t o[4] = {0u, 0u, 0u, 0u};
-              if (nv > 0) {
-                const uintptr_t a = reinterpret_cast<uintptr_t>(src_row + off);
-                const uint32_t sh = static_cast<uint32_t>(a & 3);
-                const uint32_t* aw = reinterpret_cast<const uint32_t*>(a - sh);
-                uint32_t w[5];
-#pragma unroll
-                for (int j = 0; j < 5; ++j) w[j] = (4 * j - static_cast<int>(sh) < nv) ? __ldg(aw + j) : 0u;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  const uint32_t v = __funnelshift_r(w[j], w[j + 1], sh * 8);
-                  const int64_t left = nv - 4 * j;
-                  o[j] = left >= 4 ? v : (left <= 0 ? 0u : (v & ((1u << (8 * static_cast<int>(left))) - 1u)));
-                }
-              }
-              *reinterpret_cast<uint4*>(dst + ((c ^ (r & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
-            }
+            const int off = (lo + i) * 128;
+            pack_row_kblock(src_row + off, min(max(kb_bytes - off, 0), 128), region + i * STAGE, r);
           }
         }
         fence_proxy_async_smem();
