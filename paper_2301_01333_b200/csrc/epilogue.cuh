@@ -52,112 +52,128 @@ __device__ __forceinline__ int quantize_value(float t, float inv, int zp, int lo
   return min(max(r + zp, lo), hi);
 }
 
-// Per-column constants of 16 consecutive output columns (bias, dequantisation scale, zero-point compensation).
-// Loading them is separated from using them so that a kernel can issue the loads before it waits for its
-// accumulators.
-struct EpiCols16 {
-  float b[16];
-  float dq[16];
-  int c[16];
+// Per-column constants of NC (8 or 16) consecutive output columns (bias, dequantisation scale, zero-point
+// compensation).  Loading them is separated from using them so that a kernel can issue the loads before it waits for
+// its accumulators.
+template <int NC>
+struct EpiColsT {
+  float b[NC];
+  float dq[NC];
+  int c[NC];
 };
+using EpiCols16 = EpiColsT<16>;
 
-__device__ __forceinline__ void epi_load_cols16(EpiCols16& k, int n0, const Epilogue& e) {
+template <int NC>
+__device__ __forceinline__ void epi_load_cols(EpiColsT<NC>& k, int n0, const Epilogue& e) {
   if (e.comp) {
     const int4* cp = reinterpret_cast<const int4*>(e.comp + n0);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < NC / 4; ++i) {
       const int4 v = __ldg(cp + i);
       k.c[4 * i] = v.x; k.c[4 * i + 1] = v.y; k.c[4 * i + 2] = v.z; k.c[4 * i + 3] = v.w;
     }
   } else {
 #pragma unroll
-    for (int i = 0; i < 16; ++i) k.c[i] = 0;
+    for (int i = 0; i < NC; ++i) k.c[i] = 0;
   }
   if (e.bias) {
     const float4* bp = reinterpret_cast<const float4*>(e.bias + n0);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < NC / 4; ++i) {
       const float4 v = __ldg(bp + i);
       k.b[4 * i] = v.x; k.b[4 * i + 1] = v.y; k.b[4 * i + 2] = v.z; k.b[4 * i + 3] = v.w;
     }
   } else {
 #pragma unroll
-    for (int i = 0; i < 16; ++i) k.b[i] = 0.f;
+    for (int i = 0; i < NC; ++i) k.b[i] = 0.f;
   }
   if (e.dqv) {
     const float4* dp = reinterpret_cast<const float4*>(e.dqv + n0);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < NC / 4; ++i) {
       const float4 v = __ldg(dp + i);
       k.dq[4 * i] = v.x; k.dq[4 * i + 1] = v.y; k.dq[4 * i + 2] = v.z; k.dq[4 * i + 3] = v.w;
     }
   } else {
 #pragma unroll
-    for (int i = 0; i < 16; ++i) k.dq[i] = e.dq;
+    for (int i = 0; i < NC; ++i) k.dq[i] = e.dq;
   }
 }
+__device__ __forceinline__ void epi_load_cols16(EpiCols16& k, int n0, const Epilogue& e) { epi_load_cols<16>(k, n0, e); }
 
-// The 16 values after dequantisation, bias and activation (fp32, before any conversion to the output type).
-__device__ __forceinline__ void epi_values16(const uint32_t* raw, float (&t)[16], const Epilogue& e, const EpiCols16& k) {
+// The NC values after dequantisation, bias and activation (fp32, before any conversion to the output type).
+template <int NC>
+__device__ __forceinline__ void epi_values(const uint32_t* raw, float (&t)[NC], const Epilogue& e, const EpiColsT<NC>& k) {
   const bool has_bias = e.bias != nullptr, acc_int = e.acc_is_int != 0;
   const int act = e.act;
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
+  for (int i = 0; i < NC; ++i) {
     float x = acc_int ? __fmul_rn(__int2float_rn(static_cast<int>(raw[i]) - k.c[i]), k.dq[i]) : __uint_as_float(raw[i]);
     x = has_bias ? __fadd_rn(x, k.b[i]) : x;      // separately rounded: exact on the integer path
     t[i] = x;
   }
   if (act == ACT_RELU) {
 #pragma unroll
-    for (int i = 0; i < 16; ++i) t[i] = fmaxf(t[i], 0.0f);
+    for (int i = 0; i < NC; ++i) t[i] = fmaxf(t[i], 0.0f);
   } else if (act != ACT_NONE) {
 #pragma unroll
-    for (int i = 0; i < 16; ++i) t[i] = apply_act(t[i], act);
+    for (int i = 0; i < NC; ++i) t[i] = apply_act(t[i], act);
   }
 }
+__device__ __forceinline__ void epi_values16(const uint32_t* raw, float (&t)[16], const Epilogue& e, const EpiCols16& k) {
+  epi_values<16>(raw, t, e, k);
+}
 
-// Store 16 consecutive outputs of one row (columns n0..n0+15) from 16 raw accumulator words.
-// `dst_row` points at column 0 of the row; n0 is a multiple of 16 and the row pitch keeps 16-byte
-// alignment of (dst_row + n0) for every supported dtype.
-__device__ __forceinline__ void epi_store16_cols(const uint32_t* raw, void* dst_row, int n0, const Epilogue& e,
-                                                 const EpiCols16& k) {
+// Store NC consecutive outputs of one row (columns n0..n0+NC-1) from NC raw accumulator words.
+// `dst_row` points at column 0 of the row; n0 is a multiple of NC and the row pitch keeps the alignment of
+// (dst_row + n0) that the vector stores need (NC output elements) for every supported dtype.
+template <int NC>
+__device__ __forceinline__ void epi_store_cols(const uint32_t* raw, void* dst_row, int n0, const Epilogue& e,
+                                               const EpiColsT<NC>& k) {
   if (e.acc_is_int && !e.has_dq) {   // raw s32 accumulators (zero-point compensation is exact in s32)
     int4* d = reinterpret_cast<int4*>(static_cast<int*>(dst_row) + n0);
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < NC / 4; ++i)
       d[i] = make_int4(static_cast<int>(raw[4 * i]) - k.c[4 * i], static_cast<int>(raw[4 * i + 1]) - k.c[4 * i + 1],
                        static_cast<int>(raw[4 * i + 2]) - k.c[4 * i + 2], static_cast<int>(raw[4 * i + 3]) - k.c[4 * i + 3]);
     return;
   }
-  float t[16];
-  epi_values16(raw, t, e, k);
+  float t[NC];
+  epi_values<NC>(raw, t, e, k);
   if (e.out_dtype == GC_F32) {
     float4* d = reinterpret_cast<float4*>(static_cast<float*>(dst_row) + n0);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) d[i] = make_float4(t[4 * i], t[4 * i + 1], t[4 * i + 2], t[4 * i + 3]);
+    for (int i = 0; i < NC / 4; ++i) d[i] = make_float4(t[4 * i], t[4 * i + 1], t[4 * i + 2], t[4 * i + 3]);
   } else if (e.out_dtype == GC_BF16) {
-    uint32_t w[8];
+    uint32_t w[NC / 2];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
+    for (int i = 0; i < NC / 2; ++i) {
       __nv_bfloat162 h = __floats2bfloat162_rn(t[2 * i], t[2 * i + 1]);
       w[i] = *reinterpret_cast<uint32_t*>(&h);
     }
     uint4* d = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(dst_row) + n0);
-    d[0] = make_uint4(w[0], w[1], w[2], w[3]);
-    d[1] = make_uint4(w[4], w[5], w[6], w[7]);
+#pragma unroll
+    for (int i = 0; i < NC / 8; ++i) d[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
   } else {
     const int lo = e.out_dtype == GC_U8 ? 0 : -128, hi = e.out_dtype == GC_U8 ? 255 : 127;
-    uint32_t w[4];
+    uint32_t w[NC / 4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < NC / 4; ++i) {
       uint32_t b0 = quantize_value(t[4 * i + 0], e.inv, e.zp, lo, hi) & 0xFF;
       uint32_t b1 = quantize_value(t[4 * i + 1], e.inv, e.zp, lo, hi) & 0xFF;
       uint32_t b2 = quantize_value(t[4 * i + 2], e.inv, e.zp, lo, hi) & 0xFF;
       uint32_t b3 = quantize_value(t[4 * i + 3], e.inv, e.zp, lo, hi) & 0xFF;
       w[i] = b0 | (b1 << 8) | (b2 << 16) | (b3 << 24);
     }
-    *reinterpret_cast<uint4*>(static_cast<uint8_t*>(dst_row) + n0) = make_uint4(w[0], w[1], w[2], w[3]);
+    if constexpr (NC == 16)
+      *reinterpret_cast<uint4*>(static_cast<uint8_t*>(dst_row) + n0) = make_uint4(w[0], w[1], w[2], w[3]);
+    else
+      *reinterpret_cast<uint2*>(static_cast<uint8_t*>(dst_row) + n0) = make_uint2(w[0], w[1]);
   }
+}
+__device__ __forceinline__ void epi_store16_cols(const uint32_t* raw, void* dst_row, int n0, const Epilogue& e,
+                                                 const EpiCols16& k) {
+  epi_store_cols<16>(raw, dst_row, n0, e, k);
 }
 
 __device__ __forceinline__ void epi_store16(const uint32_t* raw, void* dst_row, int n0, const Epilogue& e) {

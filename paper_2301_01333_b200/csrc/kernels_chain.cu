@@ -88,6 +88,37 @@ __device__ __forceinline__ int ch_load_i(const void* p, int64_t i, int dtype) {
   return static_cast<const int8_t*>(p)[i];
 }
 
+// One finishing thread: add the KS partial sums of NC consecutive columns of one row (column group `cgrp` of the 32
+// the CTA owns) and store them with the post-ops applied.  All four possible parts are loaded (what lies behind the
+// buffer for KS < 4 is shared memory of this CTA) and a select drops the surplus ones: no branch per part - a lone
+// warp pays about 30 clocks for each.  Fixed order: exact for s32, deterministic for fp32.
+template <int KIND, int NC>
+__device__ __forceinline__ void chain_finish(const uint8_t* sRed, int rows_per, int KS, int frow, int cgrp, void* dst_row,
+                                             int fcol, const Epilogue& epi, const EpiColsT<NC>& fk) {
+  uint32_t a[NC];
+#pragma unroll
+  for (int i = 0; i < NC; ++i) a[i] = 0u;
+#pragma unroll
+  for (int s = 0; s < 4; ++s) {
+    const uint8_t* src = sRed + (s * rows_per + frow) * 128;
+    const bool use = s < KS;
+#pragma unroll
+    for (int c = 0; c < NC / 4; ++c) {
+      const uint4 v = *reinterpret_cast<const uint4*>(src + (((cgrp * (NC / 4) + c) ^ (frow & 7)) << 4));
+      if constexpr (KIND == KIND_I8) {
+        a[4 * c] += use ? v.x : 0u; a[4 * c + 1] += use ? v.y : 0u;
+        a[4 * c + 2] += use ? v.z : 0u; a[4 * c + 3] += use ? v.w : 0u;
+      } else {
+        a[4 * c] = __float_as_uint(__uint_as_float(a[4 * c]) + (use ? __uint_as_float(v.x) : 0.f));
+        a[4 * c + 1] = __float_as_uint(__uint_as_float(a[4 * c + 1]) + (use ? __uint_as_float(v.y) : 0.f));
+        a[4 * c + 2] = __float_as_uint(__uint_as_float(a[4 * c + 2]) + (use ? __uint_as_float(v.z) : 0.f));
+        a[4 * c + 3] = __float_as_uint(__uint_as_float(a[4 * c + 3]) + (use ? __uint_as_float(v.w) : 0.f));
+      }
+    }
+  }
+  epi_store_cols<NC>(a, dst_row, fcol, epi, fk);
+}
+
 template <int KIND>
 __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_constant__ ChainParams p) {
   constexpr int K_ELEMS = KIND == KIND_I8 ? 128 : (KIND == KIND_BF16 ? 64 : 32);
@@ -287,11 +318,19 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
           // expect the partial sums of the whole cluster for my rows of the tile (senders may be ahead of this)
           if (KS > 1 && threadIdx.x == 64) mbar_arrive_expect_tx(bar_red, CH_RED_BYTES);
           // the per-column constants of the outputs this thread will finish: fetched now, used after the waits
+          // With four parts every CTA finishes 32 rows: four threads per row, 8 columns each, so that all 128 epilogue
+          // threads share the work; with two parts (64 rows) two threads per row, 16 columns each.
           const int ft = threadIdx.x - 64;
-          const int fcol = cta * CH_BLOCK_N + 16 * (ft & 1);
-          const bool finisher = KS > 1 && ft < 2 * rows_per && fcol < L.N;
-          EpiCols16 fk;
-          if (finisher) epi_load_cols16(fk, fcol, L.epi);
+          const bool fine = KS == 4;
+          const int frow = fine ? ft >> 2 : ft >> 1, cgrp = fine ? ft & 3 : ft & 1;
+          const int fcol = cta * CH_BLOCK_N + (fine ? 8 : 16) * cgrp;
+          const bool finisher = KS > 1 && frow < rows_per && fcol < L.N;
+          EpiColsT<16> fk16;
+          EpiColsT<8> fk8;
+          if (finisher) {
+            if (fine) epi_load_cols<8>(fk8, fcol, L.epi);
+            else epi_load_cols<16>(fk16, fcol, L.epi);
+          }
           if (KS == 1 && L.epi.bias && lane < 2 && cta * CH_BLOCK_N + 16 * lane < L.N)
             asm volatile("prefetch.global.L1 [%0];" ::"l"(L.epi.bias + cta * CH_BLOCK_N + 16 * lane));
           if (mbar_wait(bar_tfull, tphase)) {
@@ -341,38 +380,14 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
               if (lane == 0)
                 bulk_copy_to_cluster(mapa_shared(smem_u32(sRed) + static_cast<uint32_t>((ksr * rows_per + lrow) * 128), dest),
                                      smem_u32(sSend) + static_cast<uint32_t>(row * 128), 32 * 128, mapa_shared(bar_red, dest));
-              // finish my rows of the tile: thread t handles row t / 2, columns 16 (t % 2) .. + 16
+              // finish my rows of the tile
               if (mbar_wait_cluster(bar_red, tphase)) {
                 if (finisher) {
-                  const int frow = ft >> 1, half = ft & 1;
-                  uint32_t a[16];
-#pragma unroll
-                  for (int i = 0; i < 16; ++i) a[i] = 0u;
-                  // All four possible parts are loaded (what lies behind the buffer for KS < 4 is shared memory of this
-                  // CTA) and a select drops the surplus ones: no branch per part - a lone warp pays about 30 clocks for
-                  // each.  Fixed order: exact for s32, deterministic for fp32.
-#pragma unroll
-                  for (int s = 0; s < 4; ++s) {
-                    const uint8_t* src = sRed + (s * rows_per + frow) * 128;
-                    const bool use = s < KS;
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                      const uint4 v = *reinterpret_cast<const uint4*>(src + (((half * 4 + c) ^ (frow & 7)) << 4));
-                      if constexpr (KIND == KIND_I8) {
-                        a[4 * c] += use ? v.x : 0u; a[4 * c + 1] += use ? v.y : 0u;
-                        a[4 * c + 2] += use ? v.z : 0u; a[4 * c + 3] += use ? v.w : 0u;
-                      } else {
-                        a[4 * c] = __float_as_uint(__uint_as_float(a[4 * c]) + (use ? __uint_as_float(v.x) : 0.f));
-                        a[4 * c + 1] = __float_as_uint(__uint_as_float(a[4 * c + 1]) + (use ? __uint_as_float(v.y) : 0.f));
-                        a[4 * c + 2] = __float_as_uint(__uint_as_float(a[4 * c + 2]) + (use ? __uint_as_float(v.z) : 0.f));
-                        a[4 * c + 3] = __float_as_uint(__uint_as_float(a[4 * c + 3]) + (use ? __uint_as_float(v.w) : 0.f));
-                      }
-                    }
-                  }
                   const int grow = row0 + ksr * rows_per + frow;
                   if (grow < L.M) {
                     char* dst_row = static_cast<char*>(L.out) + static_cast<int64_t>(grow) * L.out_pitch * L.out_elem;
-                    epi_store16_cols(a, dst_row, fcol, L.epi, fk);
+                    if (fine) chain_finish<KIND, 8>(sRed, rows_per, KS, frow, cgrp, dst_row, fcol, L.epi, fk8);
+                    else chain_finish<KIND, 16>(sRed, rows_per, KS, frow, cgrp, dst_row, fcol, L.epi, fk16);
                   }
                 }
               } else {
