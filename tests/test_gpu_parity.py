@@ -333,6 +333,8 @@ def _mlp_variant(kind, batch, dims, bias=True, act="relu", transposed=False, hid
     ("bf16", 96, (256, 512, 128), dict(bias=False, act="gelu_tanh")),
     ("bf16", 5000, (1024, 1024, 1024), dict(transposed=True, act="gelu_tanh")),
     ("f32", 32, (100, 256, 64), dict(act="sigmoid")),
+    ("f32", 16, (40, 128, 64, 32), dict(act="gelu_tanh")),        # one cluster, first layer recomputed, out-of-line activation
+    ("f32", 8, (20, 64, 32), dict(bias=False, act="sigmoid")),
     ("f32", 600, (64, 512, 128), dict(bias=False, transposed=True))])
 @pytest.mark.parametrize("opts", [{}, {"no_chain_fusion": True}])
 def test_mlp_graph_variants(B, kind, batch, dims, kw, opts):
