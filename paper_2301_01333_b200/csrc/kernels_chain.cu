@@ -36,10 +36,11 @@ namespace gc {
 constexpr int CH_THREADS = 192;          // warp 0 producer, warp 1 MMA, warps 2-5 epilogue
 constexpr int CH_MAX_STAGES = 32;
 constexpr int CH_BLOCK_N = 32;
-// Consecutive MMAs into one accumulator form a dependent chain of roughly 130 clocks per instruction however
-// narrow the tile is, so the four 32-byte k-steps of a k-block go to four independent 32-column accumulators
-// that the epilogue adds up (exact for s32; a fixed summation order for fp32).
-constexpr int CH_NACC = 4;
+// One 32-column accumulator.  Dealing the four k-steps of a k-block onto four independent accumulators was tried and
+// kept for a while: it takes the MMAs from about 130 to about 118 clocks each, but the epilogue then reads four times
+// the tensor memory and adds it up, which costs a lone warp more than the MMAs gain (config 2: 21.06 us with four
+// accumulators, 20.42 us with one).
+constexpr int CH_NACC = 1;
 constexpr int CH_RED_BYTES = 128 * 32 * 4;   // partial-sum exchange buffer: 128 rows x 32 columns x 4 bytes
 
 __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
@@ -287,7 +288,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
                 const uint64_t a_desc = a_desc0 + static_cast<uint64_t>(manual_a ? i : stage) * a_step;
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
-                  umma_ss<KIND>(tmem_base + k * CH_BLOCK_N, a_desc + 2 * k, b_desc + 2 * k, idesc, i != 0);
+                  umma_ss<KIND>(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (i | k) != 0);
                 if (!manual_a && ++stage == CH_STAGES) {
                   stage = 0;
                   phase ^= 1;
@@ -337,21 +338,9 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
             tc_fence_after();
             uint32_t r[32];
             if (my_nkb > 0) {
-              uint32_t r1[32], r2[32], r3[32];
               const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
               tmem_ld32(t_row, r);
-              tmem_ld32(t_row + CH_BLOCK_N, r1);
-              tmem_ld32(t_row + 2 * CH_BLOCK_N, r2);
-              tmem_ld32(t_row + 3 * CH_BLOCK_N, r3);
               tmem_wait_ld();
-#pragma unroll
-              for (int i = 0; i < 32; ++i) {
-                if constexpr (KIND == KIND_I8)
-                  r[i] = (r[i] + r1[i]) + (r2[i] + r3[i]);
-                else
-                  r[i] = __float_as_uint((__uint_as_float(r[i]) + __uint_as_float(r1[i])) +
-                                         (__uint_as_float(r2[i]) + __uint_as_float(r3[i])));
-              }
             } else {
 #pragma unroll
               for (int i = 0; i < 32; ++i) r[i] = 0u;

@@ -11,8 +11,8 @@
 //     (slices_l * ks_l <= C); CTA r works on slice r / ks_l, part r % ks_l, and is idle in layers with fewer parts;
 //   * per layer a CTA waits for its k-blocks of the A operand (first layer: TMA from global memory, or rows packed
 //     by the epilogue warps when TMA cannot address the row pitch; later layers: the bulk copies of the finishing
-//     CTAs), issues tcgen05.mma (tf32, M = 64, N = 32; the four 8-deep k-steps of a k-block go to four independent
-//     accumulators), and its epilogue warps read the accumulators;
+//     CTAs), issues tcgen05.mma (tf32, M = 64, N = 32, four 8-deep k-steps per k-block, one accumulator), and its
+//     epilogue warps read the accumulator;
 //   * with ks_l > 1 the partial sums meet as in the grid-wide kernel: every CTA of a group finishes rows_per rows and
 //     receives those rows of the others' partial sums; they are added in a fixed order;
 //   * a finished row of 32 fp32 values IS a 128-byte row of a k-block of the next layer's A operand (k-block = my
@@ -35,10 +35,10 @@ namespace gc {
 
 constexpr int CC_THREADS = 192;          // warp 0 producer, warp 1 MMA, warps 2-5 epilogue
 constexpr int CC_BLOCK_N = 32;
-constexpr int CC_NACC = 4;
+constexpr int CC_NACC = 1;           // one accumulator: four did not overlap the MMAs and cost the epilogue three more loads
 constexpr int CC_K_ELEMS = 32;           // fp32 elements per 128-byte k-block
 constexpr int CC_RED_BYTES = 128 * 128;  // partial sums received: at most 128 rows of 128 bytes
-constexpr int CC_T0_COL = CC_NACC * CC_BLOCK_N;   // tensor-memory column of the recomputed first layer's accumulator
+constexpr int CC_T0_COL = 128;                     // tensor-memory column of the recomputed first layer's accumulator
 constexpr int CC_T0_MAX = 256;                     // its widest form (first-layer columns per CTA)
 constexpr int CC_T0_STRIDE = 64;                   // columns between its 128-row blocks (at most 64 batch rows)
 
@@ -94,7 +94,7 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
   float* sBias0 = reinterpret_cast<float*>(bars + 2 * CHAIN_MAX_LAYERS + 6);   // [CC_T0_MAX] first-layer bias of my columns
   float* sBias = sBias0 + CC_T0_MAX;                              // [CHAIN_MAX_LAYERS][32] bias of my slice of every layer
   const bool recompute = p.recompute_first != 0;
-  const int tmem_cols = recompute ? 256 : CC_NACC * CC_BLOCK_N;     // (+ two blocks of CC_T0_STRIDE columns)
+  const int tmem_cols = recompute ? 256 : 32;                     // (128 + two blocks of CC_T0_STRIDE columns)
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rank = static_cast<int>(cluster_ctarank());
 
@@ -261,8 +261,8 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
             for (int i = 0; i < my_nkb; ++i) {
 #pragma unroll
               for (int k = 0; k < 4; ++k)   // (each descriptor is built from its address, not stepped as an integer)
-                umma_ss<KIND_TF32>(tmem_base + k * CC_BLOCK_N, make_smem_desc(a0 + i * STAGE + 32 * k, 16, 1024, SWZ_128B),
-                                   make_smem_desc(b0 + i * (CC_BLOCK_N * 128) + 32 * k, 16, 1024, SWZ_128B), idesc, i != 0);
+                umma_ss<KIND_TF32>(tmem_base, make_smem_desc(a0 + i * STAGE + 32 * k, 16, 1024, SWZ_128B),
+                                   make_smem_desc(b0 + i * (CC_BLOCK_N * 128) + 32 * k, 16, 1024, SWZ_128B), idesc, (i | k) != 0);
             }
             umma_commit(bar_tfull);
           } else {
@@ -390,17 +390,9 @@ __global__ void __launch_bounds__(CC_THREADS, 1) mlp_cluster_kernel(const __grid
         tc_fence_after();
         uint32_t r[32];
         if (my_nkb > 0 && q * 16 < rows_all) {
-          uint32_t r1[32], r2[32], r3[32];
           const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
           tmem_ld32(t_row, r);
-          tmem_ld32(t_row + CC_BLOCK_N, r1);
-          tmem_ld32(t_row + 2 * CC_BLOCK_N, r2);
-          tmem_ld32(t_row + 3 * CC_BLOCK_N, r3);
           tmem_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            r[i] = __float_as_uint((__uint_as_float(r[i]) + __uint_as_float(r1[i])) +
-                                   (__uint_as_float(r2[i]) + __uint_as_float(r3[i])));
         } else {
 #pragma unroll
           for (int i = 0; i < 32; ++i) r[i] = 0u;
