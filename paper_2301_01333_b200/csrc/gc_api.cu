@@ -270,6 +270,8 @@ struct gc_compiled {
   std::vector<CUtensorMap> chain_tmaps;      // host copy of the tensor-map array
   const void* chain_a0_ptr = nullptr;        // first-layer A pointer the array was built for
   bool chain_tmaps_valid = false;
+  bool chain_fold_tail = false;              // the one-column last layer is folded into the layer before it
+  size_t chain_tail_off = 0;                 // workspace offset of its per-row sums and counters (2 x 4 bytes x M)
   // the same chain inside one thread-block cluster (small fp32 chains)
   int chain_cluster = 0;                     // cluster size (0: the grid-wide kernel)
   bool chain_recompute_first = false;
@@ -831,6 +833,22 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
       c->chain_barriers = static_cast<int>(c->layers.size()) - 1;   // one grid barrier between consecutive layers
       c->chain_tmap_off = ws;
       ws = align_up(ws + 2 * CHAIN_MAX_LAYERS * sizeof(CUtensorMap), 1024);
+      // An 8-bit chain that ends in a single output column (the 256 -> 1 tail of a recommender's top MLP): that
+      // column is a dot product over the row the layer before it has just finished, so its finishing threads add
+      // their part of it per row instead of storing the row, and the barrier and the separate layer go away.
+      {
+        const size_t nl = c->layers.size();
+        const LayerPlan& T = c->layers[nl - 1];
+        const LayerPlan& P = c->layers[nl - 2];
+        if (kind == 0 && ks > 1 && !T.use_tc && T.N == 1 && P.use_tc && P.out_pos < 0 && T.K == P.N && P.N % 32 == 0 &&
+            (P.epi.out_dtype == GC_U8 || P.epi.out_dtype == GC_S8) && T.w_dtype == GC_S8 && !T.need_comp) {
+          c->chain_fold_tail = true;
+          c->chain_barriers -= 1;
+          c->chain_tail_off = ws;
+          ws = align_up(ws + 2 * sizeof(int) * static_cast<size_t>(T.M), 1024);
+          c->desc += "  the one-column last layer is folded into the finishing step of the layer before it\n";
+        }
+      }
       c->launches = 1;
       snprintf(line, sizeof(line), "  fused chain: one persistent kernel, %d CTAs in clusters of %d (split reduction axis), %u KB of resident weight slices per CTA, %d grid barriers\n",
                max_ctas * ks * row_tiles, ks, w_smem / 1024, c->chain_barriers);
@@ -1253,6 +1271,9 @@ static gc_status_t run_mlp(gc_compiled& c, cudaStream_t st, const void* const* i
     }
     memcpy(cp.tmaps, c.chain_tmaps.data(), sizeof(cp.tmaps));
     cp.recompute_first = c.chain_recompute_first ? 1 : 0;
+    cp.fold_tail = (c.chain_fold_tail && !c.chain_cluster) ? 1 : 0;
+    cp.tail_acc = reinterpret_cast<int*>(ws + c.chain_tail_off);
+    cp.tail_cnt = reinterpret_cast<unsigned int*>(ws + c.chain_tail_off) + c.layers.back().M;
     if (c.chain_cluster)
       CUDA_TRY(launch_mlp_cluster(cp, c.chain_cluster, st));
     else
@@ -1432,6 +1453,8 @@ static gc_status_t run_sdpa(gc_compiled& c, cudaStream_t st, const void* const* 
 // the counters of every fused two-layer launch.
 static gc_status_t reset_device_state(gc_compiled& c, cudaStream_t st) {
   CUDA_TRY(cudaMemsetAsync(c.ws, 0, 256, st));
+  if (c.chain_fold_tail)
+    CUDA_TRY(cudaMemsetAsync(static_cast<char*>(c.ws) + c.chain_tail_off, 0, 2 * sizeof(int) * static_cast<size_t>(c.layers.back().M), st));
   for (auto& L : c.layers)
     if (L.fused_first)
       CUDA_TRY(cudaMemsetAsync(static_cast<char*>(c.ws) + L.pair_ready_off, 0, L.pair_ready_words * sizeof(unsigned long long), st));
@@ -1459,6 +1482,8 @@ extern "C" gc_status_t gc_execute(gc_compiled_t* c, void* cuda_stream, const voi
   if (cur != c->device) CUDA_TRY(cudaSetDevice(c->device));
   if (!c->status_cleared) {
     CUDA_TRY(cudaMemsetAsync(c->ws, 0, 256, st));
+    if (c->chain_fold_tail)
+      CUDA_TRY(cudaMemsetAsync(static_cast<char*>(c->ws) + c->chain_tail_off, 0, 2 * sizeof(int) * static_cast<size_t>(c->layers.back().M), st));
     c->status_cleared = true;
   }
   gc_status_t r;

@@ -142,6 +142,11 @@ struct ChainParams {
   int slices;                               // 32-column slices per row tile: grid = row tiles x slices x ks
   int early_weights;                        // 1: the prepacked weights were written by an earlier call, so their loads
                                             // need not wait for the kernel that precedes this one on the stream
+  int fold_tail;                            // grid-wide variant: the last layer has one output column and is folded into
+                                            // the finishing step of the layer before it (partial dot products added
+                                            // per row with atomics; the last contributor of a row applies the post-ops)
+  int* tail_acc;                            // [M] s32 sums, zero between launches
+  unsigned int* tail_cnt;                   // [M] contributions counted so far, zero between launches
   int recompute_first;                      // one-cluster variant: every CTA of the second layer computes the first
                                             // layer's columns it needs itself (no hand-over between the two)
   uint32_t* status;

@@ -120,6 +120,34 @@ __device__ __forceinline__ void chain_finish(const uint8_t* sRed, int rows_per, 
   epi_store_cols<NC>(a, dst_row, fcol, epi, fk);
 }
 
+// The same for the layer before a folded one-column last layer: the NC finished values are quantised as they would
+// have been stored, and what leaves is their part of the last layer's dot product, sum (code - zero point) x weight.
+template <int KIND, int NC>
+__device__ __forceinline__ int chain_finish_dot(const uint8_t* sRed, int rows_per, int KS, int frow, int cgrp, const Epilogue& epi,
+                                                const EpiColsT<NC>& fk, const int (&wt)[NC], int a_zp) {
+  uint32_t a[NC];
+#pragma unroll
+  for (int i = 0; i < NC; ++i) a[i] = 0u;
+#pragma unroll
+  for (int s = 0; s < 4; ++s) {
+    const uint8_t* src = sRed + (s * rows_per + frow) * 128;
+    const bool use = s < KS;
+#pragma unroll
+    for (int c = 0; c < NC / 4; ++c) {
+      const uint4 v = *reinterpret_cast<const uint4*>(src + (((cgrp * (NC / 4) + c) ^ (frow & 7)) << 4));
+      a[4 * c] += use ? v.x : 0u; a[4 * c + 1] += use ? v.y : 0u;
+      a[4 * c + 2] += use ? v.z : 0u; a[4 * c + 3] += use ? v.w : 0u;
+    }
+  }
+  float t[NC];
+  epi_values<NC>(a, t, epi, fk);
+  const int lo = epi.out_dtype == GC_U8 ? 0 : -128, hi = epi.out_dtype == GC_U8 ? 255 : 127;
+  int d = 0;
+#pragma unroll
+  for (int i = 0; i < NC; ++i) d += (quantize_value(t[i], epi.inv, epi.zp, lo, hi) - a_zp) * wt[i];
+  return d;
+}
+
 template <int KIND>
 __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_constant__ ChainParams p) {
   constexpr int K_ELEMS = KIND == KIND_I8 ? 128 : (KIND == KIND_BF16 ? 64 : 32);
@@ -256,7 +284,8 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
     }
   };
   const int rows_per = 128 >> KS_SH; // rows of the tile this CTA finishes
-  for (int l = 0; l < p.n_layers && !failed; ++l) {
+  const int n_run = p.fold_tail ? p.n_layers - 1 : p.n_layers;   // layers that run as layers
+  for (int l = 0; l < n_run && !failed; ++l) {
     // A by-value copy: fields read through a reference into the parameter space are re-fetched around every
     // store (possible aliasing) at a few hundred clocks each, which made a 16-element epilogue cost thousands.
     const ChainLayer L = p.L[l];
@@ -332,6 +361,14 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
             if (fine) epi_load_cols<8>(fk8, fcol, L.epi);
             else epi_load_cols<16>(fk16, fcol, L.epi);
           }
+          // the layer before a folded last layer: my columns' weights of that layer (s8, one output column)
+          const bool fold = KIND == KIND_I8 && p.fold_tail && l == n_run - 1;
+          int wt16[16];
+          if (fold && finisher) {
+            const int8_t* wp = static_cast<const int8_t*>(p.L[n_run].wt_ptr) + fcol;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) wt16[i] = (fine && i >= 8) ? 0 : static_cast<int>(wp[i]);
+          }
           if (KS == 1 && L.epi.bias && lane < 2 && cta * CH_BLOCK_N + 16 * lane < L.N)
             asm volatile("prefetch.global.L1 [%0];" ::"l"(L.epi.bias + cta * CH_BLOCK_N + 16 * lane));
           if (mbar_wait(bar_tfull, tphase)) {
@@ -370,13 +407,43 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
                 bulk_copy_to_cluster(mapa_shared(smem_u32(sRed) + static_cast<uint32_t>((ksr * rows_per + lrow) * 128), dest),
                                      smem_u32(sSend) + static_cast<uint32_t>(row * 128), 32 * 128, mapa_shared(bar_red, dest));
               // finish my rows of the tile
-              if (mbar_wait_cluster(bar_red, tphase)) {
-                if (finisher) {
-                  const int grow = row0 + ksr * rows_per + frow;
-                  if (grow < L.M) {
+              if (__all_sync(0xffffffffu, mbar_wait_cluster(bar_red, tphase) ? 1 : 0)) {   // (warp-uniform: shuffles follow)
+                const int grow = row0 + ksr * rows_per + frow;
+                if (!fold) {
+                  if (finisher && grow < L.M) {
                     char* dst_row = static_cast<char*>(L.out) + static_cast<int64_t>(grow) * L.out_pitch * L.out_elem;
                     if (fine) chain_finish<KIND, 8>(sRed, rows_per, KS, frow, cgrp, dst_row, fcol, L.epi, fk8);
                     else chain_finish<KIND, 16>(sRed, rows_per, KS, frow, cgrp, dst_row, fcol, L.epi, fk16);
+                  }
+                } else if constexpr (KIND == KIND_I8) {
+                  // Folded last layer: the row is not stored.  The 2 or 4 threads of a row (neighbouring lanes) add
+                  // up their parts of the dot product; the first of them adds the CTA's part to the row's sum in
+                  // global memory and counts the row; whoever counts last takes the sum (leaving zero behind for the
+                  // next launch), applies the last layer's post-ops and stores the one output of the row.
+                  const ChainLayer& T = p.L[n_run];
+                  int d = 0;
+                  if (finisher && grow < L.M) {
+                    if (fine) {
+                      int w8[8];
+#pragma unroll
+                      for (int i = 0; i < 8; ++i) w8[i] = wt16[i];
+                      d = chain_finish_dot<KIND, 8>(sRed, rows_per, KS, frow, cgrp, L.epi, fk8, w8, T.a_zp);
+                    } else {
+                      d = chain_finish_dot<KIND, 16>(sRed, rows_per, KS, frow, cgrp, L.epi, fk16, wt16, T.a_zp);
+                    }
+                  }
+                  d += __shfl_xor_sync(0xffffffffu, d, 1);
+                  if (fine) d += __shfl_xor_sync(0xffffffffu, d, 2);
+                  if (cgrp == 0 && frow < rows_per && grow < L.M) {
+                    asm volatile("red.relaxed.gpu.global.add.s32 [%0], %1;" ::"l"(p.tail_acc + grow), "r"(d) : "memory");
+                    unsigned int seen;
+                    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(seen) : "l"(p.tail_cnt + grow), "r"(1u) : "memory");
+                    if (seen == static_cast<unsigned int>(L.active_ctas) - 1u) {
+                      const int sum = atomicExch(p.tail_acc + grow, 0);
+                      p.tail_cnt[grow] = 0u;
+                      char* dst_row = static_cast<char*>(T.out) + static_cast<int64_t>(grow) * T.out_pitch * T.out_elem;
+                      epi_store1(static_cast<uint32_t>(sum), dst_row, 0, T.epi);
+                    }
                   }
                 }
               } else {
@@ -423,7 +490,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) mlp_chain_kernel(const __grid_c
         }
       }
     }
-    if (l + 1 < p.n_layers) next_barrier(l + 1);
+    if (l + 1 < n_run) next_barrier(l + 1);
   }
 
   tc_fence_before();

@@ -195,6 +195,27 @@ def test_mlp_int8_chain_kernel_cluster_sizes_and_entry_reorder(B, batch, dims, k
     assert np.array_equal(got, oracle(w))
 
 
+@pytest.mark.parametrize("batch,dims,ks,final", [
+    (128, (479, 1024, 1024, 512, 256, 1), 4, "sigmoid"),   # config 2: four threads per finished row
+    (300, (600, 512, 64, 1), 2, "none"),                   # two threads per row, three row tiles, the last one ragged
+    (512, (1024, 256, 1), 4, "sigmoid"),                   # four row tiles: 32 slices x 4 x 4 CTAs would not fit -> ks shrinks
+    (7, (700, 96, 32, 1), 2, "none"),                      # a handful of rows, one slice in the folded layer
+])
+def test_mlp_int8_one_column_tail_folded_into_the_layer_before(B, batch, dims, ks, final):
+    w = W.mlp_int8(batch=batch, dims=dims, final=final, per_channel=True, x_zp=3, act_zp=7)
+    got, plan = run_gpu(B, w, n_runs=3)
+    assert "folded into the finishing step" in plan, plan
+    assert np.array_equal(got[0], got[1]) and np.array_equal(got[0], got[2])      # sums and counters are left at zero
+    ref = oracle(w)
+    if final == "none":
+        assert np.array_equal(got[0], ref)
+    else:
+        assert np.abs(got[0].astype(np.float64) - ref).max() <= 2e-6
+    sep, plan2 = run_gpu(B, w, no_chain_fusion=True)
+    assert "folded" not in plan2
+    assert np.array_equal(sep, got[0]) if final == "none" else np.abs(sep.astype(np.float64) - ref).max() <= 2e-6
+
+
 @pytest.mark.parametrize("batch,dims,ks", [(16, (160, 64, 32), 2), (100, (13, 1024, 48), 4), (128, (37, 32, 16), 1)])
 def test_mlp_f32_chain_kernel_cluster_sizes(B, batch, dims, ks):
     w = W.mlp_f32(batch=batch, dims=dims)
@@ -740,7 +761,7 @@ def test_repeated_runs_are_bitwise_identical(B):
         assert np.array_equal(res[0], res[1]) and np.array_equal(res[0], res[2])
 
 
-@pytest.mark.parametrize("which", ["chain", "chain_in_one_cluster", "two_layers_one_launch", "attention"])
+@pytest.mark.parametrize("which", ["chain", "chain_folded_tail", "chain_in_one_cluster", "two_layers_one_launch", "attention"])
 def test_captured_executes_replay_correctly(B, which):
     # gc_execute after the first call is a pure sequence of kernel launches: captured into a CUDA graph and replayed,
     # it must give the same results, also for the kernels that synchronise through counters in global memory
@@ -750,6 +771,8 @@ def test_captured_executes_replay_correctly(B, which):
         w = W.mlp_int8(batch=128, dims=(479, 1024, 512, 32), final="none", per_channel=True, x_zp=3, act_zp=2)
     elif which == "chain_in_one_cluster":
         w = W.mlp_f32()
+    elif which == "chain_folded_tail":
+        w = W.mlp_int8(batch=128, dims=(479, 1024, 256, 1), final="none", per_channel=True, x_zp=3, act_zp=2)
     elif which == "two_layers_one_launch":
         w = W.ffn_bf16(tokens=4900, d_model=1024, d_ff=1024)
     else:
@@ -757,6 +780,8 @@ def test_captured_executes_replay_correctly(B, which):
     c = B.CompiledPartition(w.graph, 0)
     if which == "chain_in_one_cluster":
         assert "inside one cluster" in c.plan
+    if which == "chain_folded_tail":
+        assert "folded into the finishing step" in c.plan
     ins = B.device_inputs(w)
     outs = B.device_outputs(w.graph)
     s = torch.cuda.Stream()
@@ -788,7 +813,7 @@ def test_captured_executes_replay_correctly(B, which):
     assert not np.array_equal(replayed, first)
     w.feeds[x_id] = new_x
     ref = oracle(w)
-    if which == "chain":
+    if which in ("chain", "chain_folded_tail"):
         assert np.array_equal(replayed, ref)
     elif which == "chain_in_one_cluster":
         assert np.abs(replayed.astype(np.float64) - ref).max() <= 5e-3 * np.abs(ref).max()
