@@ -20,8 +20,13 @@
 //     next layer whose part of the reduction axis contains that k-block; the last layer stores to global memory.
 //   * a first layer with a short reduction axis (at most two k-blocks) is not distributed at all: every CTA of the
 //     second layer multiplies the input by the first-layer weight columns that make up its own part of the second
-//     layer's reduction axis (N up to 256 in one accumulator) and writes the result, bias and activation applied,
-//     straight into its own A-operand stages - redundant arithmetic across the column slices, no exchange.
+//     layer's reduction axis (up to 256 of them) and writes the result, bias and activation applied, straight into
+//     its own A-operand stages - redundant arithmetic across the column slices, no exchange.  That product is taken
+//     transposed (weight rows on the M side, 128 per MMA; batch rows on the N side), so that every one of the 128
+//     epilogue threads owns an accumulator row.
+// The code between the waits runs once per launch in warps that are alone on their schedulers: every branch costs such
+// a warp about 30 clocks and every integer division a hundred, so the epilogues use selects, shifts and tests per
+// group of rows instead, loops with run-time trip counts stay rolled, and waits and rare activations are out of line.
 // A-operand stages alternate between two regions by layer parity, and so do the staging buffers; every buffer is
 // reused two layers later, by which time the data dependence chain guarantees that all copies out of it and all MMAs
 // reading it have completed (a CTA can only reach layer l + 2 after every CTA has finished layer l).
@@ -35,7 +40,7 @@ namespace gc {
 
 constexpr int CC_THREADS = 192;          // warp 0 producer, warp 1 MMA, warps 2-5 epilogue
 constexpr int CC_BLOCK_N = 32;
-constexpr int CC_NACC = 1;           // one accumulator: four did not overlap the MMAs and cost the epilogue three more loads
+constexpr int CC_NACC = 1;               // one accumulator: four did not overlap the MMAs and cost the epilogue three more loads
 constexpr int CC_K_ELEMS = 32;           // fp32 elements per 128-byte k-block
 constexpr int CC_RED_BYTES = 128 * 128;  // partial sums received: at most 128 rows of 128 bytes
 constexpr int CC_T0_COL = 128;                     // tensor-memory column of the recomputed first layer's accumulator
