@@ -19,12 +19,18 @@
 //     sends its 32 rows to the CTA that owns them and signals that CTA's mbarrier; the owner adds the KS partials
 //     in a fixed order (exact for s32, deterministic for fp32), applies the post-ops and stores;
 //   * a grid-wide barrier (epoch-counted atomic in global memory, bounded spin) separates the layers;
-//   * layers the tensor-core path does not take (N not a multiple of 16, e.g. the 256 -> 1 tail) run on
-//     CUDA cores inside the same kernel, one warp per output;
+//   * layers the tensor-core path does not take (N not a multiple of 16) run on CUDA cores inside the same kernel,
+//     one warp per output - except the one-column last layer of an 8-bit chain (the 256 -> 1 tail of a recommender's
+//     top MLP), which is folded into the finishing step of the layer before it: the finishing threads add their part
+//     of the dot product per row with a global atomic instead of storing the row, and whoever counts a row last
+//     applies the last layer's post-ops; that takes a grid barrier and a layer out of the chain;
 //   * an input whose row pitch TMA cannot address (the graph-entry reorder, Section V: pre-op fusion "only at the
 //     entry point of the graph") is read with plain loads by the four epilogue warps, which are idle at that point,
 //     realigned in registers and written straight into the swizzled A-operand stages of the first layer.
 // At most one CTA per SM, and the host checks that all clusters of the grid can be resident together.
+// The code between the waits runs once per launch in warps that are alone on their schedulers, where a branch costs
+// about 30 clocks and an integer division a hundred: hence the shifts by log2(KS), the selects instead of per-part
+// and per-chunk tests, and the finishing step spread over all 128 epilogue threads.
 #include <cuda_bf16.h>
 
 #include "epilogue.cuh"
