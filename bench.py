@@ -159,6 +159,41 @@ def run_timed(reps, n_rep, steps, device, barrier):
     return e0.elapsed_time(e1)          # ms
 
 
+def library_two_gemms_us(w, n_rep, steps, device):
+    """Context for the FFN config, not a baseline of the path: the two GEMMs of the block as plain library calls
+    (torch.matmul = cuBLAS, bf16, no bias, no GELU, hidden tensor through memory), on random data of the same shapes,
+    rotating through as many buffer sets as the timed run rotates replicas, timed the same way."""
+    import torch
+    g = w.graph
+    shapes = [g.tensors[t].dims for t in g.inputs]
+    tokens, d_model = shapes[0]
+    d_ff = [s for s in shapes[1:] if len(s) == 2][0]
+    d_ff = d_ff[1] if d_ff[0] == d_model else d_ff[0]
+    dev = f"cuda:{device}"
+    sets = []
+    for _ in range(n_rep):
+        sets.append((torch.randn(tokens, d_model, device=dev, dtype=torch.bfloat16),
+                     torch.randn(d_model, d_ff, device=dev, dtype=torch.bfloat16) * 0.03,
+                     torch.randn(d_ff, d_model, device=dev, dtype=torch.bfloat16) * 0.03,
+                     torch.empty(tokens, d_ff, device=dev, dtype=torch.bfloat16),
+                     torch.empty(tokens, d_model, device=dev, dtype=torch.bfloat16)))
+    def step(i):
+        x, w1, w2, h, y = sets[i % n_rep]
+        torch.matmul(x, w1, out=h)
+        torch.matmul(h, w2, out=y)
+    for i in range(max(3, n_rep)):
+        step(i)
+    torch.cuda.synchronize(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        step(i)
+    e1.record()
+    torch.cuda.synchronize(device)
+    del sets
+    return e0.elapsed_time(e1) * 1e3 / steps
+
+
 def launch_floor_us(B, device, steps=2000):
     """Back-to-back launches of the smallest partition (a 16x16x16 matmul on one CTA): the per-launch cost that
     bounds the small-batch configs from below however fast their kernels are."""
@@ -552,6 +587,14 @@ def main():
         res["us_per_subgraph_warm"] = max_over_ranks(run_timed(reps[:1], 1, warm_steps, local, barrier)) * 1e3 / warm_steps
         if not args.only:
             res["us_per_subgraph_graph"] = run_graph_replay(reps, n_rep, min(steps, GRAPH_STEPS[name]), local)
+        if name == "c5" and rank == 0 and not args.only and not args.split:
+            try:
+                res["library_two_gemms_us"] = library_two_gemms_us(w, n_rep, min(steps, 200), local)
+                res["library_two_gemms_note"] = ("torch.matmul (cuBLAS) on the two GEMMs alone, same shapes and replica "
+                                                 "rotation, no bias and no GELU: context, not part of the path")
+            except Exception as exc:                    # context only: never fail the bench over it
+                res["library_two_gemms_us"] = None
+                res["library_two_gemms_note"] = f"not measured: {exc}"
         if name in ("c1", "c2") and not args.only:
             # coarse-grain fusion ablation (Section VII, Fig. 8): the whole chain in one persistent launch, one
             # launch per layer (fine-grain fusion only), and the CUDA-core kernels
@@ -640,6 +683,10 @@ def main():
                 "algorithmic_flops_per_launch": head_w.ops / n_launch,
                 "frac_of_burst_peak": achieved / (peaks.get("bf16_tflops", 1590.0) * KIND_RATIO[head]),
                 "frac_of_nominal": achieved / (NOMINAL["bf16_tflops"] * KIND_RATIO[head])}
+        if hr.get("library_two_gemms_us"):
+            # context: the library's two bare GEMMs on these very shapes (the peak above is its 8192^3 figure)
+            roof["library_two_gemms_same_shapes_us"] = hr["library_two_gemms_us"]
+            roof["vs_library_two_gemms"] = hr["library_two_gemms_us"] / us
     else:
         achieved = head_w.bytes / (us * 1e-6) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
