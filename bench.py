@@ -194,6 +194,38 @@ def library_two_gemms_us(w, n_rep, steps, device):
     return e0.elapsed_time(e1) * 1e3 / steps
 
 
+def library_sdpa_us(w, n_rep, steps, device):
+    """Context for the bf16 attention config, not a baseline of the path: torch's scaled_dot_product_attention (whatever
+    fused library kernel it selects) on random data of the same shapes with an additive mask of the same form, rotating
+    through as many buffer sets as the timed run rotates replicas, timed the same way."""
+    import torch
+    import torch.nn.functional as F
+    g = w.graph
+    q_dims = g.tensors[g.inputs[0]].dims                     # [B, H, S, D]
+    Bn, H, S, D = q_dims
+    dev = f"cuda:{device}"
+    sets = []
+    for _ in range(n_rep):
+        q, k, v = (torch.randn(Bn, H, S, D, device=dev, dtype=torch.bfloat16) for _ in range(3))
+        mask = torch.zeros(Bn, 1, 1, S, device=dev, dtype=torch.bfloat16)
+        mask[:, :, :, S - S // 8:] = float("-inf")
+        sets.append((q, k, v, mask))
+    def step(i):
+        q, k, v, mask = sets[i % n_rep]
+        return F.scaled_dot_product_attention(q, k, v, attn_mask=mask, scale=0.125)
+    for i in range(max(3, n_rep)):
+        step(i)
+    torch.cuda.synchronize(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        step(i)
+    e1.record()
+    torch.cuda.synchronize(device)
+    del sets
+    return e0.elapsed_time(e1) * 1e3 / steps
+
+
 def launch_floor_us(B, device, steps=2000):
     """Back-to-back launches of the smallest partition (a 16x16x16 matmul on one CTA): the per-launch cost that
     bounds the small-batch configs from below however fast their kernels are."""
@@ -595,6 +627,14 @@ def main():
             except Exception as exc:                    # context only: never fail the bench over it
                 res["library_two_gemms_us"] = None
                 res["library_two_gemms_note"] = f"not measured: {exc}"
+        if name == "c3" and rank == 0 and not args.only and not args.split:
+            try:
+                res["library_sdpa_us"] = library_sdpa_us(w, n_rep, min(steps, 500), local)
+                res["library_sdpa_note"] = ("torch.nn.functional.scaled_dot_product_attention (the fused library kernel it "
+                                            "selects), same shapes, mask form and replica rotation: context, not part of the path")
+            except Exception as exc:                    # context only: never fail the bench over it
+                res["library_sdpa_us"] = None
+                res["library_sdpa_note"] = f"not measured: {exc}"
         if name in ("c1", "c2") and not args.only:
             # coarse-grain fusion ablation (Section VII, Fig. 8): the whole chain in one persistent launch, one
             # launch per layer (fine-grain fusion only), and the CUDA-core kernels
