@@ -621,7 +621,7 @@ def main():
             res["us_per_subgraph_graph"] = run_graph_replay(reps, n_rep, min(steps, GRAPH_STEPS[name]), local)
         if name == "c5" and rank == 0 and not args.only and not args.split:
             try:
-                res["library_two_gemms_us"] = library_two_gemms_us(w, n_rep, min(steps, 200), local)
+                res["library_two_gemms_us"] = library_two_gemms_us(w, n_rep, steps, local)   # same steps: same power regime
                 res["library_two_gemms_note"] = ("torch.matmul (cuBLAS) on the two GEMMs alone, same shapes and replica "
                                                  "rotation, no bias and no GELU: context, not part of the path")
             except Exception as exc:                    # context only: never fail the bench over it
