@@ -805,10 +805,6 @@ extern "C" gc_status_t gc_compile(const gc_partition_t* p, int32_t cuda_device, 
       a_stages = (max_nkb + ks - 1) / ks;
       const size_t smem = mlp_chain_smem_bytes(w_smem, a_stages, a_stage_bytes, ks);
       bool fits = a_stages <= 32 && max_ctas * ks * row_tiles <= c->num_sms && smem <= static_cast<size_t>(prop.sharedMemPerBlockOptin);
-      // When the row tiles leave the grid no room to split the reduction axis at all, a CTA that has to walk more
-      // than four k-blocks per layer on its own is slower than one launch per layer (measured: 479-1024-1024-512-
-      // 256-1 at batch 512, 42 against 33 microseconds).
-      if (row_tiles > 1 && ks == 1 && a_stages > 4) fits = false;
       // all clusters must be resident together (the layers are separated by a grid-wide barrier)
       if (fits && cuda_device != GC_DEVICE_PLAN_ONLY) {
         int cur = -1;
