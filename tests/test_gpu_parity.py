@@ -902,6 +902,27 @@ def test_overlapped_host_entry_point_batches_in_flight(B):
     torch.cuda.synchronize()
 
 
+def test_overlapped_host_entry_point_with_pageable_buffers_and_attention(B):
+    # pageable numpy buffers (the copies are then synchronous inside the call, the results the same) on the attention
+    # pattern: every slot in flight at once, each with its own Q
+    import torch
+    ws = [W.mha_bf16(batch=2, heads=3, seed=s) for s in (1, 2, 3)]
+    g = ws[0].graph
+    c = B.CompiledPartition(g, 0)
+    ns = c.HOST_SLOTS
+    ins = [[np.ascontiguousarray(w.feeds[t]) for t in g.inputs] for w in ws[:ns]]
+    outs = [np.zeros(g.tensors[g.outputs[0]].dims, dtype=np.uint16) for _ in range(ns)]
+    for k in range(ns):
+        c.execute_host_async(k, ins[k], [outs[k]])
+    for k in range(ns):
+        c.host_wait(k)
+        ref = interp.run(ws[k].graph, ws[k].feeds)[ws[k].graph.outputs[0]]
+        assert np.abs(bf16_to_f64(outs[k]) - ref).max() <= 2e-2
+    c.host_wait(0)                                          # waiting for an idle slot returns at once
+    c.close()
+    torch.cuda.synchronize()
+
+
 def test_host_buffer_entry_point_picks_up_a_constant_at_a_new_host_address(B):
     # a constant that arrives at a new host address is copied to the same staging address: the weights must be
     # preprocessed again, not only the bias re-read
